@@ -1,0 +1,267 @@
+"""ctypes front end of the CPU oracle (``snip_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the benchmark's
+cpu_baseline / reference arm.  It never touches the CUDA library and holds no arithmetic of its
+own beyond composing the C routines in the order the paper states them (Sec. 2.2, Fig. 5:
+quantize the operands, multiply, keep the product in BF16; Sec. 3.1: Frobenius norms of the
+tensors and of their quantization errors).
+
+bf16 tensors travel as ``numpy.uint16`` arrays holding the raw bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 0, 1, 2
+BLOCK_ROW, BLOCK_COL, BLOCK_BLK = 0, 1, 2
+TILE = 128
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "snip_oracle.c")
+_LIB = os.path.join(_HERE, "libsnip_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (strict IEEE flags: no contraction, no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-shared",
+               "-fPIC", "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i64, i32, vp, dbl = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_double
+        L.orc_fpx_max.restype = dbl
+        L.orc_fpx_max.argtypes = [i32]
+        L.orc_bf16_to_float.restype = ctypes.c_float
+        L.orc_bf16_to_float.argtypes = [ctypes.c_uint16]
+        L.orc_double_to_bf16.restype = ctypes.c_uint16
+        L.orc_double_to_bf16.argtypes = [dbl]
+        L.orc_decode_code.restype = dbl
+        L.orc_decode_code.argtypes = [i32, ctypes.c_uint8]
+        L.orc_encode_e4m3.restype = ctypes.c_uint8
+        L.orc_encode_e4m3.argtypes = [ctypes.c_float]
+        L.orc_encode_e2m1.restype = ctypes.c_uint8
+        L.orc_encode_e2m1.argtypes = [ctypes.c_float]
+        L.orc_tile_scale.restype = ctypes.c_float
+        L.orc_tile_scale.argtypes = [i32, ctypes.c_float]
+        L.orc_scale_shape.restype = None
+        L.orc_scale_shape.argtypes = [i64, i64, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.orc_quantize.restype = i32
+        L.orc_quantize.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp]
+        L.orc_dequantize.restype = i32
+        L.orc_dequantize.argtypes = [vp, vp, i64, i64, i32, i32, vp]
+        L.orc_pack_codes.restype = i32
+        L.orc_pack_codes.argtypes = [vp, i64, i64, i32, i32, vp]
+        for name in ("orc_gemm_fwd", "orc_gemm_dgrad", "orc_gemm_wgrad"):
+            fn = getattr(L, name)
+            fn.restype = None
+            fn.argtypes = [vp, vp, vp, i64, i64, i64]
+        L.orc_round_to_bf16.restype = None
+        L.orc_round_to_bf16.argtypes = [vp, i64, vp]
+        L.orc_sumsq_bf16.restype = dbl
+        L.orc_sumsq_bf16.argtypes = [vp, i64]
+        L.orc_num_threads.restype = i32
+        L.orc_num_threads.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def fpx_max(fmt: int) -> float:
+    return float(lib().orc_fpx_max(fmt))
+
+
+def decode_code(fmt: int, code: int) -> float:
+    return float(lib().orc_decode_code(fmt, code))
+
+
+def encode(fmt: int, t: float) -> int:
+    t32 = np.float32(t)
+    if fmt == FMT_FP8_E4M3:
+        return int(lib().orc_encode_e4m3(t32))
+    if fmt == FMT_FP4_E2M1:
+        return int(lib().orc_encode_e2m1(t32))
+    raise ValueError("fmt")
+
+
+def tile_scale(fmt: int, amax: float) -> np.float32:
+    return np.float32(lib().orc_tile_scale(fmt, np.float32(amax)))
+
+
+def bf16_to_float(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to float64."""
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    with np.errstate(invalid="ignore"):
+        return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def round_to_bf16(v: np.ndarray) -> np.ndarray:
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    out = np.empty(v.shape, dtype=np.uint16)
+    lib().orc_round_to_bf16(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def scale_shape(rows: int, cols: int, block: int):
+    d0, d1 = ctypes.c_int64(), ctypes.c_int64()
+    lib().orc_scale_shape(rows, cols, block, ctypes.byref(d0), ctypes.byref(d1))
+    return int(d0.value), int(d1.value)
+
+
+@dataclass
+class Quantized:
+    """Result of quantizing one bf16 matrix (Sec. 2.3)."""
+    fmt: int
+    block: int
+    rows: int
+    cols: int
+    codes: np.ndarray | None      # uint8 [rows, cols], one code per byte; None for BF16
+    scales: np.ndarray | None     # float32, shape given by scale_shape(); None for BF16
+    xhat: np.ndarray              # float64 [rows, cols], dequantized values
+    sumsq_x: float                # sum of x^2
+    sumsq_err: float              # sum of (x - xhat)^2
+    row_sumsq_x: np.ndarray       # float64 [rows]
+    row_sumsq_err: np.ndarray     # float64 [rows]
+
+    def packed(self, transposed: bool = False) -> np.ndarray:
+        """Codes in the library's storage layout (FP4: two per byte, even index low)."""
+        return pack_codes(self.codes, self.fmt, transposed)
+
+
+def quantize(x_bits: np.ndarray, fmt: int, block: int) -> Quantized:
+    x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    assert x.ndim == 2
+    rows, cols = x.shape
+    quantized = fmt != FMT_BF16
+    codes = np.zeros((rows, cols), dtype=np.uint8) if quantized else None
+    scales = np.zeros(scale_shape(rows, cols, block), dtype=np.float32) if quantized else None
+    xhat = np.empty((rows, cols), dtype=np.float64)
+    sumsq = np.zeros(2, dtype=np.float64)
+    row_sumsq = np.zeros((rows, 2), dtype=np.float64)
+    rc = lib().orc_quantize(_ptr(x), rows, cols, fmt, block, _ptr(codes), _ptr(scales),
+                            _ptr(xhat), _ptr(sumsq), _ptr(row_sumsq))
+    if rc != 0:
+        raise ValueError("orc_quantize: bad argument")
+    return Quantized(fmt, block, rows, cols, codes, scales, xhat, float(sumsq[0]),
+                     float(sumsq[1]), row_sumsq[:, 0].copy(), row_sumsq[:, 1].copy())
+
+
+def dequantize(codes: np.ndarray, scales: np.ndarray, fmt: int, block: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.float32)
+    rows, cols = codes.shape
+    out = np.empty((rows, cols), dtype=np.float64)
+    rc = lib().orc_dequantize(_ptr(codes), _ptr(scales), rows, cols, fmt, block, _ptr(out))
+    if rc != 0:
+        raise ValueError("orc_dequantize: bad argument")
+    return out
+
+
+def pack_codes(codes: np.ndarray, fmt: int, transposed: bool = False) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    rows, cols = codes.shape
+    outer, inner = (cols, rows) if transposed else (rows, cols)
+    per_byte = 2 if fmt == FMT_FP4_E2M1 else 1
+    out = np.zeros((outer, inner // per_byte), dtype=np.uint8)
+    rc = lib().orc_pack_codes(_ptr(codes), rows, cols, fmt, int(transposed), _ptr(out))
+    if rc != 0:
+        raise ValueError("orc_pack_codes: bad argument")
+    return out
+
+
+def _gemm(name, a, b, out_shape, M, N, K):
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    b = np.ascontiguousarray(b, dtype=np.float64)
+    out = np.empty(out_shape, dtype=np.float64)
+    getattr(lib(), name)(_ptr(a), _ptr(b), _ptr(out), M, N, K)
+    return out
+
+
+def gemm_fwd(xhat: np.ndarray, what: np.ndarray) -> np.ndarray:
+    """Y[M,N] = X[M,K] . W[N,K]^T in float64."""
+    M, K = xhat.shape
+    N, K2 = what.shape
+    assert K == K2
+    return _gemm("orc_gemm_fwd", xhat, what, (M, N), M, N, K)
+
+
+def gemm_dgrad(dyhat: np.ndarray, what: np.ndarray) -> np.ndarray:
+    """dX[M,K] = dY[M,N] . W[N,K] in float64."""
+    M, N = dyhat.shape
+    N2, K = what.shape
+    assert N == N2
+    return _gemm("orc_gemm_dgrad", dyhat, what, (M, K), M, N, K)
+
+
+def gemm_wgrad(dyhat: np.ndarray, xhat: np.ndarray) -> np.ndarray:
+    """dW[N,K] = dY[M,N]^T . X[M,K] in float64."""
+    M, N = dyhat.shape
+    M2, K = xhat.shape
+    assert M == M2
+    return _gemm("orc_gemm_wgrad", dyhat, xhat, (N, K), M, N, K)
+
+
+# ---- the three GEMMs of one linear layer under a precision choice (Fig. 5) -------------------
+
+def linear_fwd(x_bits, w_bits, fmt_x, fmt_w):
+    """Quantize X with 1x128 tiles along K and W with 128x128 blocks, then Y = Xhat What^T."""
+    qx = quantize(x_bits, fmt_x, BLOCK_ROW)
+    qw = quantize(w_bits, fmt_w, BLOCK_BLK)
+    return gemm_fwd(qx.xhat, qw.xhat), qx, qw
+
+
+def linear_dgrad(dy_bits, w_bits, fmt_dy, fmt_w):
+    """Quantize dY with 1x128 tiles along N and W with 128x128 blocks, then dX = dYhat What."""
+    qdy = quantize(dy_bits, fmt_dy, BLOCK_ROW)
+    qw = quantize(w_bits, fmt_w, BLOCK_BLK)
+    return gemm_dgrad(qdy.xhat, qw.xhat), qdy, qw
+
+
+def linear_wgrad(dy_bits, x_bits, fmt_dy, fmt_x):
+    """Quantize dY and X with 128x1 tiles along M (the contraction), then dW = dYhat^T Xhat."""
+    qdy = quantize(dy_bits, fmt_dy, BLOCK_COL)
+    qx = quantize(x_bits, fmt_x, BLOCK_COL)
+    return gemm_wgrad(qdy.xhat, qx.xhat), qdy, qx
+
+
+def sumsq_bf16(bits: np.ndarray) -> float:
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return float(lib().orc_sumsq_bf16(_ptr(b), b.size))
+
+
+def layer_stats(x_bits, w_bits, y_bits, dy_bits, dx_bits, dw_bits):
+    """Step-1 statistics of one linear layer (Sec. 3.1): the plain sum of squares of the six
+    tensors, and the error sum of squares of X, W, dY under each candidate format and each tile
+    kind the tensor is consumed with.  Any tensor may be None."""
+    out = {"sumsq": {}, "sumsq_err": {}}
+    named = {"X": x_bits, "W": w_bits, "Y": y_bits, "dY": dy_bits, "dX": dx_bits, "dW": dw_bits}
+    for name, t in named.items():
+        if t is not None:
+            out["sumsq"][name] = sumsq_bf16(t)
+    kinds = {"X": (BLOCK_ROW, BLOCK_COL), "W": (BLOCK_BLK,), "dY": (BLOCK_ROW, BLOCK_COL)}
+    for name, blocks in kinds.items():
+        t = named[name]
+        if t is None:
+            continue
+        for fmt in (FMT_FP8_E4M3, FMT_FP4_E2M1):
+            for block in blocks:
+                out["sumsq_err"][(name, fmt, block)] = quantize(t, fmt, block).sumsq_err
+    return out
