@@ -1,0 +1,227 @@
+/*
+ * snip.h -- C ABI of the B200 (sm_100a) library for SNIP's layerwise mixed-precision linear
+ * layer: per-block-scaled BF16 -> FP8 E4M3 / FP4 E2M1 quantizers with fused error-norm
+ * statistics, and the forward / input-gradient / weight-gradient GEMMs on the tcgen05 tensor
+ * cores with FP32 accumulation.
+ *
+ * Conventions
+ *   - Every function returns a snip_status_t (0 = SNIP_OK).  Nothing throws, nothing allocates,
+ *     nothing synchronizes the host: all device work is enqueued on the caller's stream.
+ *   - The caller owns every buffer.  Pointers are DEVICE pointers unless the name ends in
+ *     `_host`.  Device pointers must be 16-byte aligned.  Outputs are fully overwritten.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Matrices are row-major.  M = tokens, K = in-features, N = out-features;
+ *     X[M,K], W[N,K], Y[M,N], dY[M,N], dX[M,K], dW[N,K]  (paper Sec. 4.2, 4.3).
+ *   - All matrix dimensions must be positive multiples of 64 (SNIP_ERR_SHAPE otherwise); a
+ *     dimension that is not a multiple of 128 ends in one 64-wide tile.
+ *   - bf16 data is passed as raw 16-bit words (void* / uint16_t*).
+ *   - Errors: SNIP_ERR_ARG (null pointer, bad enum), SNIP_ERR_SHAPE, SNIP_ERR_ALIGN,
+ *     SNIP_ERR_UNSUPPORTED (precision pair, layout, or a device that is not sm_100),
+ *     SNIP_ERR_WORKSPACE (workspace too small), SNIP_ERR_CUDA (a CUDA call failed; see
+ *     snip_last_cuda_error), SNIP_ERR_TIMEOUT (a device-side bounded wait ran out; reported by
+ *     snip_poll_status).  On any error before launch nothing is enqueued.
+ */
+#ifndef SNIP_H_
+#define SNIP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SNIP_OK = 0,
+    SNIP_ERR_ARG = 1,
+    SNIP_ERR_SHAPE = 2,
+    SNIP_ERR_ALIGN = 3,
+    SNIP_ERR_UNSUPPORTED = 4,
+    SNIP_ERR_WORKSPACE = 5,
+    SNIP_ERR_CUDA = 6,
+    SNIP_ERR_TIMEOUT = 7
+} snip_status_t;
+
+/* Element formats (paper Sec. 2.3 "Quantization Format"): BF16 is the unquantized baseline,
+ * FP8 is E4M3 (max 448), FP4 is E2M1 of the MX specification (max 6). */
+typedef enum { SNIP_FMT_BF16 = 0, SNIP_FMT_FP8_E4M3 = 1, SNIP_FMT_FP4_E2M1 = 2 } snip_fmt_t;
+
+/* Scaling granularity (paper Sec. 2.3 "Quantization granularity"): 1x128 tiles for activations
+ * and gradients, 128x128 blocks for weights.  A 1x128 tile runs along the contraction dimension
+ * of the GEMM that consumes the operand: ROW = along the contiguous (column) index,
+ * COL = along the row index (128 consecutive rows of one column). */
+typedef enum { SNIP_BLOCK_ROW_1x128 = 0, SNIP_BLOCK_COL_128x1 = 1, SNIP_BLOCK_BLK_128x128 = 2 } snip_block_t;
+
+/* Output element type of a GEMM.  BF16 is the paper's choice (Sec. 2.2: "the output of the
+ * GEMM operator remains in BF16"); FP32 exposes the accumulator for parity checks and for
+ * weight-gradient accumulation. */
+typedef enum { SNIP_OUT_BF16 = 0, SNIP_OUT_FP32 = 1 } snip_out_t;
+
+typedef enum { SNIP_OP_FWD = 0, SNIP_OP_DGRAD = 1, SNIP_OP_WGRAD = 2 } snip_op_t;
+
+/* snip_quantize flags */
+#define SNIP_Q_TRANSPOSED 0x1u /* store the codes as the transpose: element (r,c) at [c][r]   */
+#define SNIP_Q_STATS      0x2u /* write *stats (needs a workspace)                            */
+#define SNIP_Q_NO_CODES   0x4u /* statistics only: codes and scales are not written           */
+
+/* Error-norm statistics of one tensor (paper Sec. 3.1, Step 1: Frobenius norm of a tensor and
+ * of its quantization error; Sec. 4.1: error = x - q(x)).  Lives in device memory.
+ * Norms are the square roots of the two sums. */
+typedef struct {
+    double sumsq_x;   /* sum of x^2                                  */
+    double sumsq_err; /* sum of (x - dequant(quant(x)))^2            */
+    float amax;       /* max |x| over the whole tensor               */
+    uint32_t reserved;
+} snip_stats_t;
+
+/* A quantized matrix, described to the GEMM.  No ownership is taken.
+ *   rows, cols : logical shape of the matrix that was quantized
+ *   codes      : FP8: one byte per element; FP4: two per byte, even index of the contiguous
+ *                dimension in bits [3:0], odd in [7:4]; BF16: the original bf16 words.
+ *                Stored [rows][cols] or, if `transposed`, [cols][rows].
+ *   scales     : FP32 scale S = FPX_MAX / amax of each tile (paper Sec. 2.3), NULL for BF16:
+ *                ROW  [ceil(cols/128)][rows],  COL  [ceil(rows/128)][cols],
+ *                BLK  [ceil(rows/128)][ceil(cols/128)].
+ */
+typedef struct {
+    const void *codes;
+    const float *scales;
+    int64_t rows, cols;
+    int32_t fmt;        /* snip_fmt_t   */
+    int32_t block;      /* snip_block_t */
+    int32_t transposed; /* 0 or 1       */
+    int32_t reserved;
+} snip_qtensor_t;
+
+/* Tensors of one linear layer for snip_layer_stats; any pointer may be NULL (skipped). */
+typedef struct {
+    const void *X, *W, *Y, *dY, *dX, *dW; /* bf16, shapes as in the header comment */
+    int64_t M, N, K;
+} snip_layer_tensors_t;
+
+/* Result of snip_layer_stats (device memory).  Indices: tensor 0..5 = X, W, Y, dY, dX, dW.
+ * sumsq_err[t][f][b]: t in {0:X, 1:W, 2:dY}, f in {0:FP8, 1:FP4}, b = snip_block_t.  Filled for
+ * the tile kinds the tensor is consumed with (X, dY: ROW and COL; W: BLK); others are 0. */
+typedef struct {
+    double sumsq[6];
+    double sumsq_err[3][2][3];
+} snip_layer_stats_t;
+
+/* ---- library information ----------------------------------------------------------------- */
+
+/* Version of this ABI as major*10000 + minor*100 + patch.  (No counterpart in the paper.) */
+int snip_version(void);
+/* Static, NUL-terminated name of a status code.  (No counterpart in the paper.) */
+const char *snip_status_string(int status);
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char *snip_last_cuda_error(void);
+
+/* ---- quantizer (paper Sec. 2.3: scale = FPX_MAX / max|x|, y = Op(Quant(x*scale))/scale) ---- */
+
+/*
+ * Byte sizes of the outputs and of the workspace that snip_quantize needs for a rows x cols
+ * input.  Host-only.  Any of the three output pointers may be NULL.
+ * codes_bytes: rows*cols (FP8), rows*cols/2 (FP4), 0 (BF16 or NO_CODES).
+ * scales_bytes: 4 * number of tiles (0 for BF16 or NO_CODES).
+ * ws_bytes: 0 unless SNIP_Q_STATS is set or row_stats will be requested (the value returned
+ * covers both).
+ */
+int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int block, uint32_t flags,
+                        size_t *codes_bytes_host, size_t *scales_bytes_host, size_t *ws_bytes_host);
+
+/*
+ * Quantize a row-major bf16 matrix x[rows][ld] (ld >= cols, in elements, multiple of 8).
+ * Per tile: amax = max|x|; S = FPX_MAX/amax as an IEEE binary32 quotient (S = 1 for an all-zero
+ * tile, clamped to FLT_MAX on overflow); code = round-to-nearest-even, saturating, of the
+ * binary32 product x*S.  Codes and scales are written in the layouts of snip_qtensor_t
+ * (codes transposed if SNIP_Q_TRANSPOSED).  With SNIP_Q_STATS the two sums and the global amax
+ * go to *stats in the same pass; with row_stats != NULL, row_stats[2*r] and [2*r+1] receive the
+ * per-row sums (paper Sec. 6.2: the row-wise form keeps one value per row).
+ * fmt = BF16 is the identity: nothing is encoded, the error sum is 0; only statistics are
+ * produced.  ws / ws_bytes: scratch of at least the size snip_quantize_sizes reports (may be
+ * NULL / 0 when that size is 0); its contents are undefined afterwards.
+ * Inputs must be finite.  One statistics kernel follows the main kernel on the same stream.
+ */
+int snip_quantize(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,
+                  uint32_t flags, void *codes, float *scales, snip_stats_t *stats,
+                  double *row_stats, void *ws, size_t ws_bytes, void *stream);
+
+/* ---- GEMMs (paper Fig. 5; Sec. 2.2: GEMM in FPX, output in BF16) -------------------------- */
+
+/*
+ * Workspace bytes for one GEMM call of the given op and shape, and for the snip_linear_* call
+ * of the same op (which also holds the quantized operands).  Host-only.
+ */
+int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b,
+                        size_t *gemm_bytes_host, size_t *linear_bytes_host);
+
+/*
+ * GEMM over already-quantized operands (lets W be quantized once per optimizer step).
+ *   FWD   : out[M,N] = A.B^T, A = X  (ROW tiles, codes [M,K]),            B = W (BLK, [N,K])
+ *   DGRAD : out[M,K] = A.B^T, A = dY (ROW tiles, codes [M,N]),            B = W (BLK, codes
+ *           stored transposed, i.e. [K,N])
+ *   WGRAD : out[N,K] = A.B^T, A = dY (COL tiles, codes transposed [N,M]), B = X (COL tiles,
+ *           codes transposed [K,M])
+ * i.e. both operands always have the contraction index contiguous.  Each 128-long chunk of the
+ * contraction is multiplied on the tensor cores (FP32 accumulation), then scaled by
+ * 1/(S_a*S_b) of that chunk in FP32 and added to an FP32 accumulator ("the output is scaled
+ * back by dividing by the same scaling factor", Sec. 2.3); the result is rounded to nearest-even
+ * to bf16 or stored as FP32.  accumulate != 0 adds to the existing contents of out (FP32 output
+ * only).  Operand formats: (BF16,BF16), (FP8,FP8), (FP4,FP4), (FP8,FP4), (FP4,FP8); pairs
+ * that mix BF16 with a quantized operand return SNIP_ERR_UNSUPPORTED.
+ * ws must hold at least gemm_bytes of snip_workspace_size; its first word is the device status
+ * word read by snip_poll_status.
+ */
+int snip_gemm_quantized(int op, const snip_qtensor_t *a_host, const snip_qtensor_t *b_host,
+                        void *out, int out_dtype, int accumulate, void *ws, size_t ws_bytes,
+                        void *stream);
+
+/*
+ * One linear layer's forward GEMM under a precision choice: quantize X (1x128 tiles along K)
+ * and W (128x128 blocks) into the workspace, then Y = Xq.Wq^T.  stats_x / stats_w may be NULL;
+ * if given they receive the statistics of the two quantizations.  (Fig. 5, forward pass.)
+ */
+int snip_linear_fwd(const void *X, const void *W, void *Y, int64_t M, int64_t N, int64_t K,
+                    int fmt_x, int fmt_w, int out_dtype, snip_stats_t *stats_x,
+                    snip_stats_t *stats_w, void *ws, size_t ws_bytes, void *stream);
+
+/* Input gradient: quantize dY (1x128 tiles along N) and W (128x128 blocks), dX = dYq.Wq.
+ * (Fig. 5, backward pass; Sec. 4.3.) */
+int snip_linear_dgrad(const void *dY, const void *W, void *dX, int64_t M, int64_t N, int64_t K,
+                      int fmt_dy, int fmt_w, int out_dtype, snip_stats_t *stats_dy,
+                      snip_stats_t *stats_w, void *ws, size_t ws_bytes, void *stream);
+
+/* Weight gradient: quantize dY and X with 128x1 tiles along M (the contraction),
+ * dW = dYq^T.Xq.  accumulate != 0 adds to dW (FP32 output only).  (Fig. 5; Sec. 4.3.) */
+int snip_linear_wgrad(const void *dY, const void *X, void *dW, int64_t M, int64_t N, int64_t K,
+                      int fmt_dy, int fmt_x, int out_dtype, int accumulate,
+                      snip_stats_t *stats_dy, snip_stats_t *stats_x, void *ws, size_t ws_bytes,
+                      void *stream);
+
+/* ---- statistics (paper Sec. 3.1, Step 1) -------------------------------------------------- */
+
+/*
+ * Frobenius-norm statistics of one linear layer: sum of squares of each given tensor, and the
+ * quantization-error sum of squares of X, W and dY under every format selected in fmt_mask
+ * (bit 1 = FP8, bit 2 = FP4) and every tile kind the tensor is consumed with, one read per
+ * tensor.  These are the quantities the loss- and weight-divergence estimates are built from
+ * (Sec. 4.2, 4.3).  ws_bytes must be at least snip_layer_stats_workspace().
+ */
+int snip_layer_stats(const snip_layer_tensors_t *t_host, uint32_t fmt_mask,
+                     snip_layer_stats_t *out, void *ws, size_t ws_bytes, void *stream);
+int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes_host);
+
+/* ---- device status ------------------------------------------------------------------------ */
+
+/*
+ * Read the device status word of a GEMM workspace.  Call after the stream has been
+ * synchronized.  *status_host becomes SNIP_OK or SNIP_ERR_TIMEOUT (a bounded device-side wait
+ * expired and the kernel returned early; outputs are then invalid).  Performs a small
+ * device-to-host copy.  (No counterpart in the paper.)
+ */
+int snip_poll_status(const void *ws, int *status_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNIP_H_ */

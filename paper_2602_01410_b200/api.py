@@ -1,0 +1,234 @@
+"""Thin Python binding of the C-ABI library declared in include/snip.h.
+
+Argument marshalling only: every function takes torch CUDA tensors (used here purely as device
+memory) and forwards raw pointers and sizes to the entry point of the same name.  All work runs
+in the library's CUDA kernels on torch's current stream.  There is no fallback: if the shared
+library is missing or fails to load, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 0, 1, 2
+BLOCK_ROW, BLOCK_COL, BLOCK_BLK = 0, 1, 2
+OUT_BF16, OUT_FP32 = 0, 1
+OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
+Q_TRANSPOSED, Q_STATS, Q_NO_CODES = 1, 2, 4
+OK = 0
+ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(1, 8)
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsnip_b200.so")
+
+EXPORTS = (
+    "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
+    "snip_quantize", "snip_workspace_size", "snip_gemm_quantized", "snip_linear_fwd",
+    "snip_linear_dgrad", "snip_linear_wgrad", "snip_layer_stats", "snip_layer_stats_workspace",
+    "snip_poll_status",
+)
+
+
+class SnipError(RuntimeError):
+    def __init__(self, fn, status):
+        self.status = status
+        name = _lib.snip_status_string(status).decode()
+        detail = _lib.snip_last_cuda_error().decode() if status == ERR_CUDA else ""
+        super().__init__(f"{fn} failed: {name} {detail}".strip())
+
+
+class QTensor(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("rows", ctypes.c_int64),
+                ("cols", ctypes.c_int64), ("fmt", ctypes.c_int32), ("block", ctypes.c_int32),
+                ("transposed", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class LayerTensors(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("X", "W", "Y", "dY", "dX", "dW")] + \
+               [(n, ctypes.c_int64) for n in ("M", "N", "K")]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2602_01410_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    i32, i64, u32, vp, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_size_t
+    psz = ctypes.POINTER(sz)
+    lib.snip_version.restype = i32
+    lib.snip_status_string.restype = ctypes.c_char_p
+    lib.snip_status_string.argtypes = [i32]
+    lib.snip_last_cuda_error.restype = ctypes.c_char_p
+    lib.snip_quantize_sizes.argtypes = [i64, i64, i32, i32, u32, psz, psz, psz]
+    lib.snip_quantize.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
+    lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
+    lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
+    lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.snip_linear_fwd.argtypes = lin
+    lib.snip_linear_dgrad.argtypes = lin
+    lib.snip_linear_wgrad.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.snip_layer_stats.argtypes = [ctypes.POINTER(LayerTensors), u32, vp, vp, sz, vp]
+    lib.snip_layer_stats_workspace.argtypes = [i64, i64, i64, psz]
+    lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int and name not in ("snip_version",):
+            fn.restype = i32
+    return lib
+
+
+_lib = _load()
+
+
+def _check(fn, status):
+    if status != OK:
+        raise SnipError(fn, status)
+
+
+def _p(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def snip_version() -> int:
+    return int(_lib.snip_version())
+
+
+def snip_status_string(status: int) -> str:
+    return _lib.snip_status_string(status).decode()
+
+
+def snip_quantize_sizes(rows, cols, fmt, block, flags=0):
+    cb, sb, wb = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+    _check("snip_quantize_sizes", _lib.snip_quantize_sizes(rows, cols, fmt, block, flags, ctypes.byref(cb),
+                                                            ctypes.byref(sb), ctypes.byref(wb)))
+    return cb.value, sb.value, wb.value
+
+
+def stats_to_host(stats: torch.Tensor) -> dict:
+    """Decode a snip_stats_t held in a 24-byte uint8 tensor (synchronizes)."""
+    raw = stats.cpu().numpy().tobytes()
+    import struct
+    sx, se, am, _ = struct.unpack("<ddfI", raw[:24])
+    return {"sumsq_x": sx, "sumsq_err": se, "amax": am}
+
+
+def snip_quantize(x: torch.Tensor, fmt: int, block: int, flags: int = 0, *, codes=None, scales=None,
+                  stats=None, row_stats=None, ws=None, want_row_stats=False):
+    """x: bf16 CUDA tensor [rows, cols] (row stride = x.stride(0)).  Allocates any output not
+    supplied, through torch, and returns (codes, scales, stats, row_stats) as uint8 / float32 /
+    uint8[24] / float64[rows,2] tensors (None where not produced)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    cb, sb, wb = snip_quantize_sizes(rows, cols, fmt, block, flags)
+    dev = x.device
+    if cb and codes is None:
+        codes = torch.empty(cb, dtype=torch.uint8, device=dev)
+    if sb and scales is None:
+        scales = torch.empty(sb // 4, dtype=torch.float32, device=dev)
+    if (flags & Q_STATS) and stats is None:
+        stats = torch.empty(24, dtype=torch.uint8, device=dev)
+    if want_row_stats and row_stats is None:
+        row_stats = torch.empty((rows, 2), dtype=torch.float64, device=dev)
+    if ws is None and ((flags & Q_STATS) or row_stats is not None):
+        ws = torch.empty(wb, dtype=torch.uint8, device=dev)
+    _check("snip_quantize", _lib.snip_quantize(_p(x), rows, cols, x.stride(0), fmt, block, flags, _p(codes), _p(scales),
+                                               _p(stats), _p(row_stats), _p(ws), 0 if ws is None else ws.numel(), _stream()))
+    return codes, scales, stats, row_stats
+
+
+def snip_workspace_size(op, M, N, K, fmt_a, fmt_b):
+    g, l = ctypes.c_size_t(), ctypes.c_size_t()
+    _check("snip_workspace_size", _lib.snip_workspace_size(op, M, N, K, fmt_a, fmt_b, ctypes.byref(g), ctypes.byref(l)))
+    return g.value, l.value
+
+
+def make_qtensor(codes, scales, rows, cols, fmt, block, transposed=False) -> QTensor:
+    return QTensor(codes.data_ptr(), 0 if scales is None else scales.data_ptr(), rows, cols, fmt, block,
+                   int(transposed), 0)
+
+
+def _out(shape, out_dtype, device, out):
+    if out is not None:
+        return out
+    return torch.empty(shape, dtype=torch.bfloat16 if out_dtype == OUT_BF16 else torch.float32, device=device)
+
+
+def snip_gemm_quantized(op, a: QTensor, b: QTensor, out_shape, out_dtype=OUT_BF16, accumulate=False, *, out=None,
+                        ws=None, device="cuda"):
+    out = _out(out_shape, out_dtype, device, out)
+    if ws is None:
+        M, N = out_shape
+        g, _ = snip_workspace_size(op, *_mnk(op, a, b), a.fmt, b.fmt)
+        ws = torch.zeros(g, dtype=torch.uint8, device=out.device)
+    _check("snip_gemm_quantized", _lib.snip_gemm_quantized(op, ctypes.byref(a), ctypes.byref(b), _p(out), out_dtype,
+                                                           int(accumulate), _p(ws), ws.numel(), _stream()))
+    return out
+
+
+def _mnk(op, a: QTensor, b: QTensor):
+    if op == OP_FWD:      # a = X[M,K], b = W[N,K]
+        return a.rows, b.rows, a.cols
+    if op == OP_DGRAD:    # a = dY[M,N], b = W[N,K]
+        return a.rows, a.cols, b.cols
+    return a.rows, a.cols, b.cols  # wgrad: a = dY[M,N], b = X[M,K]
+
+
+def _linear(fn_name, A, B, out_shape, M, N, K, fmt_a, fmt_b, out_dtype, op, out, ws, want_stats, extra=()):
+    out = _out(out_shape, out_dtype, A.device, out)
+    if ws is None:
+        _, l = snip_workspace_size(op, M, N, K, fmt_a, fmt_b)
+        ws = torch.zeros(l, dtype=torch.uint8, device=A.device)
+    sa = torch.empty(24, dtype=torch.uint8, device=A.device) if want_stats else None
+    sb = torch.empty(24, dtype=torch.uint8, device=A.device) if want_stats else None
+    fn = getattr(_lib, fn_name)
+    _check(fn_name, fn(_p(A), _p(B), _p(out), M, N, K, fmt_a, fmt_b, out_dtype, *extra, _p(sa), _p(sb), _p(ws),
+                       ws.numel(), _stream()))
+    return out, sa, sb
+
+
+def snip_linear_fwd(X, W, fmt_x, fmt_w, out_dtype=OUT_BF16, *, out=None, ws=None, want_stats=False):
+    M, K = X.shape
+    N = W.shape[0]
+    return _linear("snip_linear_fwd", X, W, (M, N), M, N, K, fmt_x, fmt_w, out_dtype, OP_FWD, out, ws, want_stats)
+
+
+def snip_linear_dgrad(dY, W, fmt_dy, fmt_w, out_dtype=OUT_BF16, *, out=None, ws=None, want_stats=False):
+    M, N = dY.shape
+    K = W.shape[1]
+    return _linear("snip_linear_dgrad", dY, W, (M, K), M, N, K, fmt_dy, fmt_w, out_dtype, OP_DGRAD, out, ws, want_stats)
+
+
+def snip_linear_wgrad(dY, X, fmt_dy, fmt_x, out_dtype=OUT_BF16, accumulate=False, *, out=None, ws=None,
+                      want_stats=False):
+    M, N = dY.shape
+    K = X.shape[1]
+    return _linear("snip_linear_wgrad", dY, X, (N, K), M, N, K, fmt_dy, fmt_x, out_dtype, OP_WGRAD, out, ws,
+                   want_stats, extra=(int(accumulate),))
+
+
+def snip_layer_stats_workspace(M, N, K):
+    w = ctypes.c_size_t()
+    _check("snip_layer_stats_workspace", _lib.snip_layer_stats_workspace(M, N, K, ctypes.byref(w)))
+    return w.value
+
+
+def snip_layer_stats(X=None, W=None, Y=None, dY=None, dX=None, dW=None, *, M, N, K, fmt_mask=0b110, out=None, ws=None):
+    """Returns a float64 CUDA tensor of 24 values: sumsq[6] then sumsq_err[3][2][3]."""
+    dev = next(t for t in (X, W, Y, dY, dX, dW) if t is not None).device
+    lt = LayerTensors(*[0 if t is None else t.data_ptr() for t in (X, W, Y, dY, dX, dW)], M, N, K)
+    if out is None:
+        out = torch.zeros(24, dtype=torch.float64, device=dev)
+    if ws is None:
+        ws = torch.empty(snip_layer_stats_workspace(M, N, K), dtype=torch.uint8, device=dev)
+    _check("snip_layer_stats", _lib.snip_layer_stats(ctypes.byref(lt), fmt_mask, _p(out), _p(ws), ws.numel(), _stream()))
+    return out
+
+
+def snip_poll_status(ws: torch.Tensor) -> int:
+    st = ctypes.c_int(0)
+    _check("snip_poll_status", _lib.snip_poll_status(_p(ws), ctypes.byref(st)))
+    return st.value

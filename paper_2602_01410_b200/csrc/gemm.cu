@@ -1,0 +1,571 @@
+// Block-scaled GEMMs on the tcgen05 tensor cores:  out[Mo,No] = A[Mo,Kc] . B[No,Kc]^T with both
+// operands contraction-major, FP32 accumulation in tensor memory, and the paper's FP32 tile
+// scales applied per 128-long chunk of the contraction (Sec. 2.3: "the output is scaled back by
+// dividing by the same scaling factor"; Fig. 5 for the three GEMMs of a linear layer).
+//
+// Structure of one CTA (persistent, one per SM, 384 threads):
+//   warp 0      : TMA producer - streams 128-byte-wide operand tiles into a shared-memory ring
+//   warp 1      : MMA issuer   - one thread issues tcgen05.mma; owns the tensor-memory allocation
+//   warps 2..3  : idle (they only give their registers to the epilogue warps)
+//   warps 4..11 : promotion / epilogue - pull each chunk's partial sums out of tensor memory,
+//                 multiply by 1/(S_a*S_b) of that chunk and add into FP32 register accumulators
+//                 (so the scaling overlaps the next chunk's MMAs, which write the other
+//                 tensor-memory buffer), then round and store the tile.
+// All hand-offs use mbarriers with bounded waits; on a timeout the CTA raises a status word and
+// leaves cleanly (tensor memory is always released).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "sm100.cuh"
+
+namespace snip {
+
+using namespace sm100;
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int kGemmThreads = 384;  // warps 0-3: producer, MMA issuer, 2 idle; warps 4-11: epilogue
+constexpr int kNumEpiWarps = 8;
+constexpr int kSfCols = 32;  // tensor-memory columns holding constant scale factors (kind::mxf4)
+
+enum ScaleMode { SCALE_NONE = 0, SCALE_BLOCK_B = 1, SCALE_VEC_B = 2 };
+
+struct GemmArgs {
+    int32_t Mo, No, Kc;        // output rows / cols, contraction length in elements
+    const float *sa;           // A scales [chunks][Mo]
+    int64_t sa_chunk_stride;
+    const float *sb;           // B scales: SCALE_BLOCK_B [blk*sb_blk_stride + chunk*sb_chunk_stride]
+    int64_t sb_chunk_stride;   //           SCALE_VEC_B   [chunk*sb_chunk_stride + n]
+    int64_t sb_blk_stride;
+    void *out;
+    int64_t ldo;
+    int32_t accumulate;
+    uint32_t *status;
+};
+
+template <MmaKind KIND, int BN>
+struct Cfg {
+    static constexpr int kStageElemsX = (KIND == MmaKind::F16) ? 64 : 128;   // TMA x step per stage
+    static constexpr int kChunkElems = 128;                                  // scale granularity
+    static constexpr int kStageK = (KIND == MmaKind::F16) ? 64 : (KIND == MmaKind::F8F6F4 ? 128 : 256);
+    static constexpr int kChunksPerStage = (KIND == MmaKind::MXF4) ? 2 : 1;
+    static constexpr int kABytes = BM * 128;
+    static constexpr int kBBytes = BN * 128;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStages = (BN >= 256) ? 4 : 5;
+    static constexpr int kSbInvBytes = kNumEpiWarps * (BN / 2) * 4;  // per-warp reciprocal B scales (wgrad)
+    static constexpr int kSmemBytes = kStages * kStageBytes + kSbInvBytes + 256 + 1024;  // + barriers + alignment slack
+    static constexpr int kAccCols = 2 * BN;
+    static constexpr int kSfCol0 = kAccCols;
+    static constexpr int kTmemCols = 512;
+    static_assert(kAccCols + (KIND == MmaKind::MXF4 ? kSfCols : 0) <= 512, "tensor memory budget");
+};
+
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int &m_idx, int &n_idx)
+{
+    // groups of 16 row-tiles share their B panels in L2 while they are resident together
+    constexpr int kGroupM = 16;
+    const int group_size = kGroupM * num_n;
+    const int g = t / group_size;
+    const int first_m = g * kGroupM;
+    const int gm = min(num_m - first_m, kGroupM);
+    const int r = t - g * group_size;
+    m_idx = first_m + r % gm;
+    n_idx = r / gm;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Store 32 consecutive output values of one row.
+template <bool OUT_F32>
+__device__ __forceinline__ void store32(const GemmArgs &g, int64_t row, int col, const float *v)
+{
+    if (OUT_F32) {
+        float *dst = static_cast<float *>(g.out) + row * g.ldo + col;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            if (col + i < g.No) {
+                float4 o = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                if (g.accumulate) {
+                    const float4 p = *reinterpret_cast<const float4 *>(dst + i);
+                    o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+                }
+                *reinterpret_cast<float4 *>(dst + i) = o;
+            }
+        }
+    } else {
+        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(g.out) + row * g.ldo + col;
+#pragma unroll
+        for (int i = 0; i < 32; i += 8) {
+            if (col + i < g.No) {
+                uint4 o = make_uint4(pack_bf16x2(v[i], v[i + 1]), pack_bf16x2(v[i + 2], v[i + 3]),
+                                     pack_bf16x2(v[i + 4], v[i + 5]), pack_bf16x2(v[i + 6], v[i + 7]));
+                *reinterpret_cast<uint4 *>(dst + i) = o;
+            }
+        }
+    }
+}
+
+template <MmaKind KIND, int BN, int SCALE, bool OUT_F32>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g,
+            const uint32_t idesc)
+{
+    using C = Cfg<KIND, BN>;
+    constexpr int S = C::kStages;
+    constexpr int G = BN / 64;       // 32-column groups handled by one epilogue warp
+    constexpr int HALF = BN / 2;     // columns handled by one epilogue warp
+
+    extern __shared__ uint8_t smem_raw[];
+    // operand tiles need 1024-byte alignment for the 128-byte swizzle
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t smem_a0 = smem_base;
+    const uint32_t smem_b0 = smem_base + S * C::kABytes;
+    float *sb_inv = reinterpret_cast<float *>(smem_gen + S * C::kStageBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_gen + S * C::kStageBytes + C::kSbInvBytes);
+    const uint32_t bar0 = smem_base + S * C::kStageBytes + C::kSbInvBytes;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * S + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * S + 2 + a); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 4);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_m = (g.Mo + BM - 1) / BM, num_n = (g.No + BN - 1) / BN;
+    const int num_tiles = num_m * num_n;
+    const int num_chunks = (g.Kc + C::kChunkElems - 1) / C::kChunkElems;
+    const int num_kstages = (g.Kc + C::kStageK - 1) / C::kStageK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kNumEpiWarps); }
+        *abort_flag = 0u;
+        fence_barrier_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (KIND == MmaKind::MXF4) {
+        // constant scale factors 2^0 (UE8M0 byte 127) for every row of A and B
+        if (warp >= 4 && warp < 8) {
+            const uint32_t q = warp & 3;
+            for (int c = 0; c < kSfCols; ++c) tmem_st1(tmem_base + ((q * 32u) << 16) + C::kSfCol0 + c, 0x7F7F7F7Fu);
+            tmem_st_wait();
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+    }
+
+    if (warp < 4) {
+      reg_dealloc<48>();  // frees (168-48)*128 = 15360 registers
+      if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                int m_idx, n_idx;
+                tile_coords(t, num_m, num_n, m_idx, n_idx);
+                for (int ks = 0; ks < num_kstages; ++ks, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (it / S) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(full_bar(s), C::kStageBytes);
+                    tma_load_2d(smem_a0 + s * C::kABytes, &tmA, full_bar(s), ks * C::kStageElemsX, m_idx * BM);
+                    tma_load_2d(smem_b0 + s * C::kBBytes, &tmB, full_bar(s), ks * C::kStageElemsX, n_idx * BN);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            uint32_t it = 0, cc = 0;
+            bool ok = true;
+            const uint32_t sfa = tmem_base + C::kSfCol0, sfb = tmem_base + C::kSfCol0 + 16;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                for (int ks = 0; ks < num_kstages && ok; ++ks, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (it / S) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint64_t adesc = make_smem_desc_k128(smem_a0 + s * C::kABytes);
+                    const uint64_t bdesc = make_smem_desc_k128(smem_b0 + s * C::kBBytes);
+                    if (KIND == MmaKind::F16) {
+                        const uint32_t a = cc & 1u;
+                        if (ks == 0) {
+                            if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                            tc_fence_after_sync();
+                        }
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_ss<KIND>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u, 0, 0);
+                        tc_commit(empty_bar(s));
+                        if (ks == num_kstages - 1) { tc_commit(tfull_bar(a)); ++cc; }
+                    } else if (KIND == MmaKind::F8F6F4) {
+                        const uint32_t a = cc & 1u;
+                        if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_ss<KIND>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, k > 0 ? 1u : 0u, 0, 0);
+                        tc_commit(empty_bar(s));
+                        tc_commit(tfull_bar(a));
+                        ++cc;
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (2 * ks + h < num_chunks) {
+                                const uint32_t a = cc & 1u;
+                                if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                                tc_fence_after_sync();
+#pragma unroll
+                                for (int k = 0; k < 2; ++k)
+                                    mma_ss<KIND>(tmem_base + a * BN, adesc + 2 * (2 * h + k), bdesc + 2 * (2 * h + k), idesc,
+                                                 k > 0 ? 1u : 0u, sfa, sfb);
+                                tc_commit(tfull_bar(a));
+                                ++cc;
+                            }
+                        }
+                        tc_commit(empty_bar(s));
+                    }
+                }
+            }
+        }
+      }
+    } else {
+        reg_alloc<224>();    // needs (224-168)*256 = 14336 <= 15360 (an unsatisfiable request would block forever)
+        // ================= promotion / epilogue warps =================
+        const int e = warp - 4;          // 0..7
+        const int q = warp & 3;          // tensor-memory lane quarter this warp may access
+        const int h = e >> 2;            // column half
+        uint32_t cc = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            int m_idx, n_idx;
+            tile_coords(t, num_m, num_n, m_idx, n_idx);
+            const int row = m_idx * BM + q * 32 + lane;
+            const int col0 = n_idx * BN + h * HALF;
+            const bool row_ok = row < g.Mo;
+            const int nacc = (KIND == MmaKind::F16) ? 1 : num_chunks;
+            float acc[SCALE == SCALE_NONE ? 1 : HALF];
+            if (SCALE != SCALE_NONE) {
+#pragma unroll
+                for (int i = 0; i < HALF; ++i) acc[i] = 0.0f;
+            }
+            for (int c = 0; c < nacc; ++c, ++cc) {
+                const uint32_t a = cc & 1u;
+                float f[G];
+                if (SCALE == SCALE_BLOCK_B) {
+                    const float sa = row_ok ? g.sa[(int64_t)c * g.sa_chunk_stride + row] : 1.0f;
+                    const float ia = __fdiv_rn(1.0f, sa);
+#pragma unroll
+                    for (int gi = 0; gi < G; ++gi) {
+                        const int col = min(col0 + 32 * gi, g.No - 1);
+                        const float sb = g.sb[(int64_t)(col >> 7) * g.sb_blk_stride + (int64_t)c * g.sb_chunk_stride];
+                        f[gi] = ia * __fdiv_rn(1.0f, sb);
+                    }
+                } else if (SCALE == SCALE_VEC_B) {
+                    const float sa = row_ok ? g.sa[(int64_t)c * g.sa_chunk_stride + row] : 1.0f;
+                    f[0] = __fdiv_rn(1.0f, sa);
+                    // reciprocal B scales of this chunk for this warp's HALF output columns; each warp
+                    // keeps a private copy so that no cross-warp barrier is needed
+#pragma unroll
+                    for (int i = lane; i < HALF; i += 32) {
+                        const int n = col0 + i;
+                        const float sb = n < g.No ? g.sb[(int64_t)c * g.sb_chunk_stride + n] : 1.0f;
+                        sb_inv[e * HALF + i] = __fdiv_rn(1.0f, sb);
+                    }
+                    __syncwarp();
+                }
+                const bool got = mbar_wait(tfull_bar(a), (cc >> 1) & 1u, abort_flag);
+                if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
+#pragma unroll
+                for (int gi = 0; gi < G; ++gi) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + 32 * gi, v);
+                    tmem_ld_wait(v);
+                    if (SCALE == SCALE_NONE) {
+                        float o[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+                        if (row_ok) store32<OUT_F32>(g, row, col0 + 32 * gi, o);
+                    } else if (SCALE == SCALE_BLOCK_B) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc[32 * gi + i] = fmaf(__uint_as_float(v[i]), f[gi], acc[32 * gi + i]);
+                    } else {
+                        const float4 *sbv = reinterpret_cast<const float4 *>(sb_inv + e * HALF + 32 * gi);
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            const float4 s4 = sbv[i >> 2];
+                            acc[32 * gi + i + 0] = fmaf(__uint_as_float(v[i + 0]) * s4.x, f[0], acc[32 * gi + i + 0]);
+                            acc[32 * gi + i + 1] = fmaf(__uint_as_float(v[i + 1]) * s4.y, f[0], acc[32 * gi + i + 1]);
+                            acc[32 * gi + i + 2] = fmaf(__uint_as_float(v[i + 2]) * s4.z, f[0], acc[32 * gi + i + 2]);
+                            acc[32 * gi + i + 3] = fmaf(__uint_as_float(v[i + 3]) * s4.w, f[0], acc[32 * gi + i + 3]);
+                        }
+                    }
+                }
+                // this warp's reads of buffer `a` are complete: hand it back to the MMA warp
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(a));
+            }
+            if (SCALE != SCALE_NONE && ok && row_ok) {
+#pragma unroll
+                for (int gi = 0; gi < G; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, acc + 32 * gi);
+            }
+        }
+    }
+
+    // ---- teardown: every role ends here, tensor memory is always released ------------------
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies and MMAs still in flight time to land before the CTA's resources go away
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        if (threadIdx.x == 0) atomicExch(g.status, (uint32_t)SNIP_ERR_TIMEOUT);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+// Simple bf16 transpose (used only for BF16-tagged dgrad / wgrad operands).
+__global__ void transpose_bf16_kernel(const uint16_t *__restrict__ in, uint16_t *__restrict__ out, int64_t rows, int64_t cols)
+{
+    __shared__ uint16_t tile[64][66];
+    const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+        const int64_t r = r0 + i, c = c0 + threadIdx.x * 2;
+        if (r < rows && c < cols) {
+            const uint32_t v = *reinterpret_cast<const uint32_t *>(in + r * cols + c);
+            tile[i][threadIdx.x * 2] = (uint16_t)(v & 0xFFFFu);
+            tile[i][threadIdx.x * 2 + 1] = (uint16_t)(v >> 16);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+        const int64_t c = c0 + i, r = r0 + threadIdx.x * 2;
+        if (c < cols && r < rows) {
+            const uint32_t v = (uint32_t)tile[threadIdx.x * 2][i] | ((uint32_t)tile[threadIdx.x * 2 + 1][i] << 16);
+            *reinterpret_cast<uint32_t *>(out + c * rows + r) = v;
+        }
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Tensor map over a row-major [rows][kc] operand whose rows are `row_bytes` apart, fetched in
+// boxes of (128 bytes of K) x box_rows with the 128-byte swizzle.
+int make_operand_map(CUtensorMap *map, const void *ptr, CUtensorMapDataType dt, int64_t rows, int64_t kc_elems,
+                     int64_t row_bytes, int box_x_elems, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) { snprintf(last_error_buffer(), 256, "cuTensorMapEncodeTiled entry point not found"); return SNIP_ERR_CUDA; }
+    cuuint64_t dims[2] = {(cuuint64_t)kc_elems, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)box_x_elems, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(last_error_buffer(), 256, "cuTensorMapEncodeTiled failed: CUresult %d (rows %lld, k %lld, row bytes %lld, dtype %d)",
+                 (int)r, (long long)rows, (long long)kc_elems, (long long)row_bytes, (int)dt);
+        return SNIP_ERR_CUDA;
+    }
+    return SNIP_OK;
+}
+
+int sm_count()
+{
+    static thread_local int dev_cached = -1, n = 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev != dev_cached) { cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev); dev_cached = dev; }
+    return n;
+}
+
+template <MmaKind KIND, int BN, int SCALE, bool OUT_F32>
+int launch_gemm(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &g, uint32_t idesc, cudaStream_t st)
+{
+    using C = Cfg<KIND, BN>;
+    auto kern = gemm_kernel<KIND, BN, SCALE, OUT_F32>;
+    static thread_local bool attr_set = false;
+    if (!attr_set) {
+        SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+        attr_set = true;
+    }
+    const int num_tiles = (int)(ceil_div(g.Mo, BM) * ceil_div(g.No, BN));
+    const int grid = num_tiles < sm_count() ? num_tiles : sm_count();
+    kern<<<grid, kGemmThreads, C::kSmemBytes, st>>>(tmA, tmB, g, idesc);
+    SNIP_CUDA_TRY(cudaGetLastError());
+    return SNIP_OK;
+}
+
+template <MmaKind KIND, int BN>
+int launch_gemm_scale(int scale, bool out_f32, const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &g, uint32_t idesc,
+                      cudaStream_t st)
+{
+    if (scale == SCALE_BLOCK_B)
+        return out_f32 ? launch_gemm<KIND, BN, SCALE_BLOCK_B, true>(tmA, tmB, g, idesc, st)
+                       : launch_gemm<KIND, BN, SCALE_BLOCK_B, false>(tmA, tmB, g, idesc, st);
+    return out_f32 ? launch_gemm<KIND, BN, SCALE_VEC_B, true>(tmA, tmB, g, idesc, st)
+                   : launch_gemm<KIND, BN, SCALE_VEC_B, false>(tmA, tmB, g, idesc, st);
+}
+
+}  // namespace
+
+size_t gemm_ws_bytes() { return 256; }
+
+int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st)
+{
+    dim3 grid((unsigned)ceil_div(cols, 64), (unsigned)ceil_div(rows, 64)), block(32, 8);
+    transpose_bf16_kernel<<<grid, block, 0, st>>>(static_cast<const uint16_t *>(in), static_cast<uint16_t *>(out), rows, cols);
+    SNIP_CUDA_TRY(cudaGetLastError());
+    return SNIP_OK;
+}
+
+// Core GEMM over stored operands.  a_codes: [Mo][Kc] and b_codes: [No][Kc], contraction-major.
+// scale_mode: SCALE_NONE for BF16, SCALE_BLOCK_B (fwd / dgrad), SCALE_VEC_B (wgrad).
+int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
+              int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
+              int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    if (!a_codes || !b_codes || !out) return SNIP_ERR_ARG;
+    if (!valid_dim(Mo) || !valid_dim(No) || !valid_dim(Kc) || Mo > INT32_MAX || No > INT32_MAX || Kc > INT32_MAX) return SNIP_ERR_SHAPE;
+    if (out_dtype != SNIP_OUT_BF16 && out_dtype != SNIP_OUT_FP32) return SNIP_ERR_ARG;
+    if (accumulate && out_dtype != SNIP_OUT_FP32) return SNIP_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < gemm_ws_bytes()) return SNIP_ERR_WORKSPACE;
+    if (!aligned16(a_codes) || !aligned16(b_codes) || !aligned16(out) || !aligned16(ws)) return SNIP_ERR_ALIGN;
+    const bool a16 = fmt_a == SNIP_FMT_BF16, b16 = fmt_b == SNIP_FMT_BF16;
+    if (a16 != b16) return SNIP_ERR_UNSUPPORTED;
+    if (!a16 && (!sa || !sb)) return SNIP_ERR_ARG;
+    int rc = require_sm100();
+    if (rc != SNIP_OK) return rc;
+
+    GemmArgs g;
+    g.Mo = (int32_t)Mo; g.No = (int32_t)No; g.Kc = (int32_t)Kc;
+    g.sa = sa; g.sa_chunk_stride = sa_chunk_stride;
+    g.sb = sb; g.sb_chunk_stride = sb_chunk_stride; g.sb_blk_stride = sb_blk_stride;
+    g.out = out; g.ldo = No; g.accumulate = accumulate;
+    g.status = static_cast<uint32_t *>(ws);
+    const bool f32 = out_dtype == SNIP_OUT_FP32;
+
+    CUtensorMap tmA, tmB;
+    if (a16) {
+        rc = make_operand_map(&tmA, a_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Mo, Kc, Kc * 2, 64, BM);
+        if (rc) return rc;
+        rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, No, Kc, Kc * 2, 64, 256);
+        if (rc) return rc;
+        const uint32_t idesc = make_idesc(1, 1, BM, 256);
+        return f32 ? launch_gemm<MmaKind::F16, 256, SCALE_NONE, true>(tmA, tmB, g, idesc, st)
+                   : launch_gemm<MmaKind::F16, 256, SCALE_NONE, false>(tmA, tmB, g, idesc, st);
+    }
+    if (fmt_a == SNIP_FMT_FP4_E2M1 && fmt_b == SNIP_FMT_FP4_E2M1) {
+        // packed FP4 on both sides: kind::mxf4 at twice the FP8 rate; the bytes are fetched as plain u8
+        constexpr int BN = 192;
+        rc = make_operand_map(&tmA, a_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, Kc / 2, Kc / 2, 128, BM);
+        if (rc) return rc;
+        rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN);
+        if (rc) return rc;
+        const uint32_t idesc = make_idesc_block_scaled(1, 1, BM, BN);
+        return launch_gemm_scale<MmaKind::MXF4, BN>(scale_mode, f32, tmA, tmB, g, idesc, st);
+    }
+    // FP8 x FP8 and the mixed pairs: kind::f8f6f4; FP4 operands are expanded by the TMA unit to one
+    // 16-byte-aligned group per 16 elements, which is the layout this MMA kind reads
+    constexpr int BN = 256;
+    const bool a4 = fmt_a == SNIP_FMT_FP4_E2M1, b4 = fmt_b == SNIP_FMT_FP4_E2M1;
+    rc = make_operand_map(&tmA, a_codes, a4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, Kc,
+                          a4 ? Kc / 2 : Kc, 128, BM);
+    if (rc) return rc;
+    rc = make_operand_map(&tmB, b_codes, b4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc,
+                          b4 ? Kc / 2 : Kc, 128, BN);
+    if (rc) return rc;
+    const uint32_t idesc = make_idesc(a4 ? 5 : 0, b4 ? 5 : 0, BM, BN);
+    return launch_gemm_scale<MmaKind::F8F6F4, BN>(scale_mode, f32, tmA, tmB, g, idesc, st);
+}
+
+}  // namespace snip
+
+extern "C" int snip_gemm_quantized(int op, const snip_qtensor_t *a, const snip_qtensor_t *b, void *out, int out_dtype,
+                                   int accumulate, void *ws, size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    if (!a || !b || op < SNIP_OP_FWD || op > SNIP_OP_WGRAD) return SNIP_ERR_ARG;
+    if (!valid_fmt(a->fmt) || !valid_fmt(b->fmt)) return SNIP_ERR_ARG;
+    const bool q = a->fmt != SNIP_FMT_BF16;
+    int64_t Mo, No, Kc;
+    const float *sa = a->scales, *sb = b->scales;
+    int64_t sa_cs, sb_cs, sb_bs;
+    int mode;
+    if (op == SNIP_OP_FWD) {
+        // A = X[M,K] ROW tiles, B = W[N,K] blocks
+        if (a->cols != b->cols || a->transposed || b->transposed) return SNIP_ERR_SHAPE;
+        if (q && (a->block != SNIP_BLOCK_ROW_1x128 || b->block != SNIP_BLOCK_BLK_128x128)) return SNIP_ERR_UNSUPPORTED;
+        Mo = a->rows; No = b->rows; Kc = a->cols;
+        sa_cs = Mo; sb_bs = ceil_div(Kc, 128); sb_cs = 1; mode = SCALE_BLOCK_B;
+    } else if (op == SNIP_OP_DGRAD) {
+        // A = dY[M,N] ROW tiles, B = W[N,K] blocks stored transposed ([K,N])
+        if (a->cols != b->rows || a->transposed || !b->transposed) return SNIP_ERR_SHAPE;
+        if (q && (a->block != SNIP_BLOCK_ROW_1x128 || b->block != SNIP_BLOCK_BLK_128x128)) return SNIP_ERR_UNSUPPORTED;
+        Mo = a->rows; No = b->cols; Kc = a->cols;
+        sa_cs = Mo; sb_bs = 1; sb_cs = ceil_div(No, 128); mode = SCALE_BLOCK_B;
+    } else {
+        // A = dY[M,N] COL tiles stored transposed ([N,M]), B = X[M,K] COL tiles stored transposed ([K,M])
+        if (a->rows != b->rows || !a->transposed || !b->transposed) return SNIP_ERR_SHAPE;
+        if (q && (a->block != SNIP_BLOCK_COL_128x1 || b->block != SNIP_BLOCK_COL_128x1)) return SNIP_ERR_UNSUPPORTED;
+        Mo = a->cols; No = b->cols; Kc = a->rows;
+        sa_cs = Mo; sb_cs = No; sb_bs = 0; mode = SCALE_VEC_B;
+    }
+    if (!q) mode = SCALE_NONE;
+    return gemm_impl(a->fmt, b->fmt, a->codes, b->codes, Mo, No, Kc, sa, sa_cs, sb, sb_cs, sb_bs, mode, out, out_dtype, accumulate,
+                     ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int snip_poll_status(const void *ws, int *status_host)
+{
+    using namespace snip;
+    if (!ws || !status_host) return SNIP_ERR_ARG;
+    uint32_t v = 0;
+    SNIP_CUDA_TRY(cudaMemcpy(&v, ws, sizeof(v), cudaMemcpyDeviceToHost));
+    *status_host = (int)v;
+    return SNIP_OK;
+}

@@ -1,0 +1,239 @@
+// The three GEMMs of one linear layer under a precision choice (paper Fig. 5): quantize the two
+// operands with the tile kind their contraction calls for, then run the block-scaled GEMM.
+// Also snip_layer_stats (Sec. 3.1, Step 1).  Host-side composition only; all arithmetic is in
+// the kernels of quantize.cu and gemm.cu.
+#include "common.cuh"
+
+namespace snip {
+
+int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, void *codes,
+                  float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st);
+int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
+              int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
+              int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st);
+int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st);
+size_t gemm_ws_bytes();
+
+namespace {
+
+enum { SCALE_NONE = 0, SCALE_BLOCK_B = 1, SCALE_VEC_B = 2 };
+
+size_t code_bytes(int fmt, int64_t rows, int64_t cols)
+{
+    if (fmt == SNIP_FMT_FP8_E4M3) return (size_t)(rows * cols);
+    if (fmt == SNIP_FMT_FP4_E2M1) return (size_t)(rows * cols / 2);
+    return (size_t)(rows * cols * 2);  // bf16 transposed copy
+}
+size_t scale_bytes(int block, int64_t rows, int64_t cols)
+{
+    const int64_t tr = ceil_div(rows, 128), tc = ceil_div(cols, 128);
+    const int64_t n = block == SNIP_BLOCK_ROW_1x128 ? tc * rows : block == SNIP_BLOCK_COL_128x1 ? tr * cols : tr * tc;
+    return (size_t)n * sizeof(float);
+}
+size_t stats_bytes(int64_t rows, int64_t cols)
+{
+    size_t w = 0;
+    snip_quantize_sizes(rows, cols, SNIP_FMT_FP8_E4M3, SNIP_BLOCK_ROW_1x128, SNIP_Q_STATS, nullptr, nullptr, &w);
+    return w;
+}
+
+// Carves the workspace of a linear call: [status 256][codes A][scales A][codes B][scales B][stats scratch]
+struct Carve {
+    uint8_t *base;
+    size_t off = 0, cap;
+    Carve(void *p, size_t c) : base(static_cast<uint8_t *>(p)), cap(c) {}
+    void *take(size_t bytes)
+    {
+        void *r = base ? base + off : nullptr;
+        off += align_up(bytes, 256);
+        return r;
+    }
+};
+
+struct LinearPlan {
+    // operand A: rows_a x cols_a logical matrix, quantized with block_a, stored transposed or not
+    int64_t rows_a, cols_a, rows_b, cols_b;
+    int block_a, block_b;
+    bool tr_a, tr_b;
+    int64_t Mo, No, Kc;
+    int scale_mode;
+};
+
+LinearPlan plan_for(int op, int64_t M, int64_t N, int64_t K)
+{
+    LinearPlan p{};
+    if (op == SNIP_OP_FWD) {
+        p = {M, K, N, K, SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_BLK_128x128, false, false, M, N, K, SCALE_BLOCK_B};
+    } else if (op == SNIP_OP_DGRAD) {
+        p = {M, N, N, K, SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_BLK_128x128, false, true, M, K, N, SCALE_BLOCK_B};
+    } else {
+        p = {M, N, M, K, SNIP_BLOCK_COL_128x1, SNIP_BLOCK_COL_128x1, true, true, N, K, M, SCALE_VEC_B};
+    }
+    return p;
+}
+
+size_t linear_ws_bytes(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b)
+{
+    const LinearPlan p = plan_for(op, M, N, K);
+    Carve c(nullptr, 0);
+    c.take(gemm_ws_bytes());
+    const bool need_a = fmt_a != SNIP_FMT_BF16 || p.tr_a, need_b = fmt_b != SNIP_FMT_BF16 || p.tr_b;
+    if (need_a) { c.take(code_bytes(fmt_a, p.rows_a, p.cols_a)); c.take(scale_bytes(p.block_a, p.rows_a, p.cols_a)); }
+    if (need_b) { c.take(code_bytes(fmt_b, p.rows_b, p.cols_b)); c.take(scale_bytes(p.block_b, p.rows_b, p.cols_b)); }
+    c.take(stats_bytes(p.rows_a, p.cols_a));
+    c.take(stats_bytes(p.rows_b, p.cols_b));
+    return c.off;
+}
+
+int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b, int out_dtype,
+                int accumulate, snip_stats_t *stats_a, snip_stats_t *stats_b, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    if (!A || !B || !out) return SNIP_ERR_ARG;
+    if (!valid_fmt(fmt_a) || !valid_fmt(fmt_b)) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    if ((fmt_a == SNIP_FMT_BF16) != (fmt_b == SNIP_FMT_BF16)) return SNIP_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < linear_ws_bytes(op, M, N, K, fmt_a, fmt_b)) return SNIP_ERR_WORKSPACE;
+    if (!aligned16(ws)) return SNIP_ERR_ALIGN;
+    const LinearPlan p = plan_for(op, M, N, K);
+    Carve c(ws, ws_bytes);
+    void *gws = c.take(gemm_ws_bytes());
+    const bool q = fmt_a != SNIP_FMT_BF16;
+    const bool need_a = q || p.tr_a, need_b = q || p.tr_b;
+    void *codes_a = nullptr, *codes_b = nullptr;
+    float *scales_a = nullptr, *scales_b = nullptr;
+    if (need_a) { codes_a = c.take(code_bytes(fmt_a, p.rows_a, p.cols_a)); scales_a = static_cast<float *>(c.take(scale_bytes(p.block_a, p.rows_a, p.cols_a))); }
+    if (need_b) { codes_b = c.take(code_bytes(fmt_b, p.rows_b, p.cols_b)); scales_b = static_cast<float *>(c.take(scale_bytes(p.block_b, p.rows_b, p.cols_b))); }
+    const size_t sws_a_bytes = stats_bytes(p.rows_a, p.cols_a), sws_b_bytes = stats_bytes(p.rows_b, p.cols_b);
+    void *sws_a = c.take(sws_a_bytes), *sws_b = c.take(sws_b_bytes);
+
+    int rc;
+    const void *ga = A, *gb = B;
+    if (q) {
+        rc = quantize_impl(A, p.rows_a, p.cols_a, p.cols_a, fmt_a, p.block_a, (p.tr_a ? SNIP_Q_TRANSPOSED : 0u) | (stats_a ? SNIP_Q_STATS : 0u),
+                           codes_a, scales_a, stats_a, nullptr, sws_a, sws_a_bytes, st);
+        if (rc) return rc;
+        rc = quantize_impl(B, p.rows_b, p.cols_b, p.cols_b, fmt_b, p.block_b, (p.tr_b ? SNIP_Q_TRANSPOSED : 0u) | (stats_b ? SNIP_Q_STATS : 0u),
+                           codes_b, scales_b, stats_b, nullptr, sws_b, sws_b_bytes, st);
+        if (rc) return rc;
+        ga = codes_a; gb = codes_b;
+    } else {
+        // BF16 tag: identity quantization; only operands whose contraction index is not contiguous are copied
+        if (p.tr_a) { rc = transpose_bf16(A, codes_a, p.rows_a, p.cols_a, st); if (rc) return rc; ga = codes_a; }
+        if (p.tr_b) { rc = transpose_bf16(B, codes_b, p.rows_b, p.cols_b, st); if (rc) return rc; gb = codes_b; }
+        if (stats_a) { rc = quantize_impl(A, p.rows_a, p.cols_a, p.cols_a, SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, SNIP_Q_STATS, nullptr, nullptr, stats_a, nullptr, sws_a, sws_a_bytes, st); if (rc) return rc; }
+        if (stats_b) { rc = quantize_impl(B, p.rows_b, p.cols_b, p.cols_b, SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, SNIP_Q_STATS, nullptr, nullptr, stats_b, nullptr, sws_b, sws_b_bytes, st); if (rc) return rc; }
+    }
+    int64_t sa_cs = p.Mo, sb_cs, sb_bs;
+    if (op == SNIP_OP_FWD) { sb_bs = ceil_div(K, 128); sb_cs = 1; }
+    else if (op == SNIP_OP_DGRAD) { sb_bs = 1; sb_cs = ceil_div(K, 128); }
+    else { sb_bs = 0; sb_cs = p.No; }
+    return gemm_impl(fmt_a, fmt_b, ga, gb, p.Mo, p.No, p.Kc, scales_a, sa_cs, scales_b, sb_cs, sb_bs, q ? p.scale_mode : SCALE_NONE, out,
+                     out_dtype, accumulate, gws, gemm_ws_bytes(), st);
+}
+
+}  // namespace
+}  // namespace snip
+
+extern "C" int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b, size_t *gemm_bytes, size_t *linear_bytes)
+{
+    using namespace snip;
+    if (op < SNIP_OP_FWD || op > SNIP_OP_WGRAD || !valid_fmt(fmt_a) || !valid_fmt(fmt_b)) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    if (gemm_bytes) *gemm_bytes = gemm_ws_bytes();
+    if (linear_bytes) *linear_bytes = linear_ws_bytes(op, M, N, K, fmt_a, fmt_b);
+    return SNIP_OK;
+}
+
+extern "C" int snip_linear_fwd(const void *X, const void *W, void *Y, int64_t M, int64_t N, int64_t K, int fmt_x, int fmt_w, int out_dtype,
+                               snip_stats_t *stats_x, snip_stats_t *stats_w, void *ws, size_t ws_bytes, void *stream)
+{
+    return snip::linear_impl(SNIP_OP_FWD, X, W, Y, M, N, K, fmt_x, fmt_w, out_dtype, 0, stats_x, stats_w, ws, ws_bytes,
+                             static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int snip_linear_dgrad(const void *dY, const void *W, void *dX, int64_t M, int64_t N, int64_t K, int fmt_dy, int fmt_w,
+                                 int out_dtype, snip_stats_t *stats_dy, snip_stats_t *stats_w, void *ws, size_t ws_bytes, void *stream)
+{
+    return snip::linear_impl(SNIP_OP_DGRAD, dY, W, dX, M, N, K, fmt_dy, fmt_w, out_dtype, 0, stats_dy, stats_w, ws, ws_bytes,
+                             static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int snip_linear_wgrad(const void *dY, const void *X, void *dW, int64_t M, int64_t N, int64_t K, int fmt_dy, int fmt_x,
+                                 int out_dtype, int accumulate, snip_stats_t *stats_dy, snip_stats_t *stats_x, void *ws, size_t ws_bytes,
+                                 void *stream)
+{
+    return snip::linear_impl(SNIP_OP_WGRAD, dY, X, dW, M, N, K, fmt_dy, fmt_x, out_dtype, accumulate, stats_dy, stats_x, ws, ws_bytes,
+                             static_cast<cudaStream_t>(stream));
+}
+
+// ---- layer statistics ---------------------------------------------------------------------
+
+extern "C" int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes)
+{
+    using namespace snip;
+    if (!ws_bytes) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    size_t w = stats_bytes(M, K);
+    size_t t = stats_bytes(N, K); if (t > w) w = t;
+    t = stats_bytes(M, N); if (t > w) w = t;
+    *ws_bytes = align_up(w, 256) + 256;  // + one snip_stats_t slot
+    return SNIP_OK;
+}
+
+namespace snip {
+namespace {
+__global__ void gather_stat_kernel(const snip_stats_t *s, double *dst_x, double *dst_err)
+{
+    if (dst_x) *dst_x = s->sumsq_x;
+    if (dst_err) *dst_err = s->sumsq_err;
+}
+}  // namespace
+}  // namespace snip
+
+extern "C" int snip_layer_stats(const snip_layer_tensors_t *t, uint32_t fmt_mask, snip_layer_stats_t *out, void *ws, size_t ws_bytes,
+                                void *stream)
+{
+    using namespace snip;
+    if (!t || !out || !ws) return SNIP_ERR_ARG;
+    size_t need = 0;
+    int rc = snip_layer_stats_workspace(t->M, t->N, t->K, &need);
+    if (rc) return rc;
+    if (ws_bytes < need) return SNIP_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SNIP_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(snip_layer_stats_t), st));
+    snip_stats_t *slot = reinterpret_cast<snip_stats_t *>(static_cast<uint8_t *>(ws));
+    void *sws = static_cast<uint8_t *>(ws) + 256;
+    const size_t sws_bytes = ws_bytes - 256;
+    const int64_t M = t->M, N = t->N, K = t->K;
+    struct T { const void *p; int64_t r, c; int qidx; } tens[6] = {
+        {t->X, M, K, 0}, {t->W, N, K, 1}, {t->Y, M, N, -1}, {t->dY, M, N, 2}, {t->dX, M, K, -1}, {t->dW, N, K, -1}};
+    for (int i = 0; i < 6; ++i) {
+        if (!tens[i].p) continue;
+        bool have_plain = false;
+        if (tens[i].qidx >= 0) {
+            const int blocks_xdy[2] = {SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_COL_128x1};
+            const int blocks_w[1] = {SNIP_BLOCK_BLK_128x128};
+            const int *blocks = tens[i].qidx == 1 ? blocks_w : blocks_xdy;
+            const int nb = tens[i].qidx == 1 ? 1 : 2;
+            for (int f = 0; f < 2; ++f) {
+                if (!(fmt_mask & (2u << f))) continue;
+                for (int b = 0; b < nb; ++b) {
+                    rc = quantize_impl(tens[i].p, tens[i].r, tens[i].c, tens[i].c, f == 0 ? SNIP_FMT_FP8_E4M3 : SNIP_FMT_FP4_E2M1, blocks[b],
+                                       SNIP_Q_STATS | SNIP_Q_NO_CODES, nullptr, nullptr, slot, nullptr, sws, sws_bytes, st);
+                    if (rc) return rc;
+                    gather_stat_kernel<<<1, 1, 0, st>>>(slot, have_plain ? nullptr : &out->sumsq[i], &out->sumsq_err[tens[i].qidx][f][blocks[b]]);
+                    SNIP_CUDA_TRY(cudaGetLastError());
+                    have_plain = true;
+                }
+            }
+        }
+        if (!have_plain) {
+            rc = quantize_impl(tens[i].p, tens[i].r, tens[i].c, tens[i].c, SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, SNIP_Q_STATS, nullptr,
+                               nullptr, slot, nullptr, sws, sws_bytes, st);
+            if (rc) return rc;
+            gather_stat_kernel<<<1, 1, 0, st>>>(slot, &out->sumsq[i], nullptr);
+            SNIP_CUDA_TRY(cudaGetLastError());
+        }
+    }
+    return SNIP_OK;
+}

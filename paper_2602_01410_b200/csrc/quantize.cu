@@ -1,0 +1,574 @@
+// Per-block-scaled quantizers BF16 -> FP8 E4M3 / FP4 E2M1 with fused error-norm statistics.
+//
+// Computes, per tile (paper Sec. 2.3):  amax = max|x|,  S = FPX_MAX / amax,
+// code = RNE_fmt(x * S);  and per tensor (Sec. 3.1, Step 1)  sum x^2 and sum (x - code/S)^2.
+// Tile kinds: 1x128 along the columns (ROW), 128x1 along the rows (COL), 128x128 (BLK).
+//
+// Memory-bound design: one CTA owns a 128x128 bf16 tile; each of its 256 threads holds an
+// 8x8 sub-block in registers (eight 128-bit loads in flight per thread), so every element is
+// read from HBM exactly once and the three tile kinds differ only in how the block-amax is
+// reduced (16-lane shuffles for ROW, a small shared-memory exchange for COL, both for BLK).
+// Codes are written with 64/128-bit stores; transposed outputs are staged through an
+// XOR-swizzled shared-memory tile so that the global stores stay fully coalesced.
+#include <cuda_bf16.h>
+#include <float.h>
+
+#include "common.cuh"
+
+namespace snip {
+
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kThreads = 256;
+
+struct CtaPartial {  // one per CTA, reduced in fixed order by stats_reduce_kernel
+    double sumsq_x;
+    double sumsq_err;
+    float amax;
+    float pad[3];
+};
+
+struct QuantArgs {
+    const uint16_t *x;
+    int64_t rows, cols, ld;
+    uint8_t *codes;       // may be null (NO_CODES)
+    float *scales;        // may be null (NO_CODES)
+    CtaPartial *partials; // may be null (no stats)
+    float2 *row_partials; // [col tiles][rows] {sum x^2, sum err^2}; may be null
+};
+
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t v)
+{
+    // packed bf16 max of |v| against a non-negative accumulator
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&acc);
+    uint32_t av = v & 0x7FFF7FFFu;
+    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&av);
+    __nv_bfloat162 m = __hmax2(a, b);
+    return *reinterpret_cast<uint32_t *>(&m);
+}
+
+__device__ __forceinline__ uint32_t max2(uint32_t x, uint32_t y)
+{
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&x);
+    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&y);
+    __nv_bfloat162 m = __hmax2(a, b);
+    return *reinterpret_cast<uint32_t *>(&m);
+}
+
+// Scale of a tile from its amax: IEEE binary32 quotient, 1 for an empty tile, clamped.
+template <int FMT>
+__device__ __forceinline__ float tile_scale(float amax)
+{
+    constexpr float kMax = (FMT == SNIP_FMT_FP8_E4M3) ? 448.0f : 6.0f;
+    if (amax == 0.0f) return 1.0f;
+    float s = __fdiv_rn(kMax, amax);
+    return fminf(s, FLT_MAX);  // +inf -> FLT_MAX
+}
+
+// Two binary32 values -> two codes.  `lo` lands in the low byte / nibble.
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; mov.b16 %0, {t, 0}; }"
+        : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// Two codes -> two binary32 values (exact).
+__device__ __forceinline__ float2 dec_e4m3x2(uint32_t c)
+{
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)c));
+    return __half22float2(*reinterpret_cast<__half2 *>(&h2));
+}
+__device__ __forceinline__ float2 dec_e2m1x2(uint32_t c)
+{
+    uint32_t h2;
+    asm("{ .reg .b8 t, u; mov.b16 {t, u}, %1; cvt.rn.f16x2.e2m1x2 %0, t; }"
+        : "=r"(h2) : "h"((uint16_t)c));
+    return __half22float2(*reinterpret_cast<__half2 *>(&h2));
+}
+
+// Quantize 8 consecutive elements (one 128-bit load) that share or do not share a scale.
+// s[i], inv[i]: scale and reciprocal for element i.  Returns the packed codes
+// (FP8: 8 bytes in out[0..1]; FP4: 4 bytes in out[0]) and adds to the statistics.
+template <int FMT, bool STATS>
+__device__ __forceinline__ void quant8(const uint4 &v, const float *s, const float *inv,
+                                       uint32_t out[2], float &sx, float &se)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t c[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float x0 = bf16lo(w[i]), x1 = bf16hi(w[i]);
+        float t0 = __fmul_rn(x0, s[2 * i]), t1 = __fmul_rn(x1, s[2 * i + 1]);
+        if (FMT == SNIP_FMT_FP8_E4M3) c[i] = cvt_e4m3x2(t0, t1);
+        else c[i] = cvt_e2m1x2(t0, t1);
+        if (STATS) {
+            float2 d = (FMT == SNIP_FMT_FP8_E4M3) ? dec_e4m3x2(c[i]) : dec_e2m1x2(c[i]);
+            float e0 = fmaf(-d.x, inv[2 * i], x0), e1 = fmaf(-d.y, inv[2 * i + 1], x1);
+            sx = fmaf(x0, x0, sx);
+            sx = fmaf(x1, x1, sx);
+            se = fmaf(e0, e0, se);
+            se = fmaf(e1, e1, se);
+        }
+    }
+    if (FMT == SNIP_FMT_FP8_E4M3) {
+        out[0] = c[0] | (c[1] << 16);
+        out[1] = c[2] | (c[3] << 16);
+    } else {
+        out[0] = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
+        out[1] = 0;
+    }
+}
+
+// FMT: target format (BF16 = statistics only).  BLOCK: tile kind.  TRANSPOSED: codes stored as
+// the transpose.  CODES: write codes and scales.  STATS: accumulate sums.  ROWSTATS: per-row sums.
+template <int FMT, int BLOCK, bool TRANSPOSED, bool CODES, bool STATS, bool ROWSTATS>
+__global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
+{
+    constexpr bool kQuant = (FMT != SNIP_FMT_BF16);
+    constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;  // bytes per 8 elements
+    constexpr int kRowBytes = kTile * kCodeBytes8 / 8;               // staged bytes per line
+
+    __shared__ __align__(16) uint8_t stage[TRANSPOSED && CODES && kQuant ? kTile * kRowBytes : 16];
+    __shared__ uint32_t col_amax[8][kTile / 2];  // packed bf16 pairs, one row per warp
+    __shared__ float col_scale[kTile];
+    __shared__ float red_f[8][3];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int64_t r0 = (int64_t)blockIdx.y * kTile, c0 = (int64_t)blockIdx.x * kTile;
+    const int64_t rbase = r0 + 8 * ty, cbase = c0 + 8 * tx;
+    const bool col_ok = cbase < a.cols;  // cols is a multiple of 64, so 8-groups never straddle
+
+    // ---- load the 8x8 sub-block: eight independent 128-bit loads ------------------------
+    uint4 v[8];
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        const int64_t r = rbase + p;
+        if (col_ok && r < a.rows)
+            v[p] = __ldg(reinterpret_cast<const uint4 *>(a.x + r * a.ld + cbase));
+        else
+            v[p] = make_uint4(0, 0, 0, 0);
+    }
+
+    // ---- block amax -> scales --------------------------------------------------------
+    float s_row[8], s_col[8];  // scale per row p (ROW) / per column j (COL); BLK uses s_row[0]
+    (void)s_row; (void)s_col;
+    float my_amax = 0.0f;      // this thread's amax, for the tensor-wide statistic
+    if (kQuant || STATS) {
+        uint32_t rmax[8];      // per row: packed max over the 8 columns (as 4 pairs folded)
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            uint32_t m = absmax2(0u, v[p].x);
+            m = absmax2(m, v[p].y);
+            m = absmax2(m, v[p].z);
+            m = absmax2(m, v[p].w);
+            rmax[p] = m;
+        }
+        if (BLOCK == SNIP_BLOCK_ROW_1x128 && kQuant) {
+            // fold pairs, pack two rows per register, reduce across the 16 lanes of the row
+            uint32_t pk[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t m0 = rmax[2 * q], m1 = rmax[2 * q + 1];
+                m0 = max2(m0, m0 >> 16);  // low half = row 2q
+                m1 = max2(m1, m1 << 16);  // high half = row 2q+1
+                pk[q] = (m0 & 0xFFFFu) | (m1 & 0xFFFF0000u);
+            }
+#pragma unroll
+            for (int off = 1; off < 16; off <<= 1)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) pk[q] = max2(pk[q], __shfl_xor_sync(0xFFFFFFFFu, pk[q], off));
+            // lane (tx & 7) derives the scale of row p = tx & 7, then the 8 scales are shared
+            const int myp = tx & 7;
+            uint32_t sel = pk[0];
+#pragma unroll
+            for (int q = 1; q < 4; ++q) sel = ((myp >> 1) == q) ? pk[q] : sel;
+            float am = (myp & 1) ? bf16hi(sel) : bf16lo(sel);
+            float mine = tile_scale<FMT>(am);
+#pragma unroll
+            for (int p = 0; p < 8; ++p) s_row[p] = __shfl_sync(0xFFFFFFFFu, mine, (lane & 16) | p);
+            if (STATS) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) my_amax = fmaxf(my_amax, fmaxf(bf16lo(pk[q]), bf16hi(pk[q])));
+            }
+            if (CODES && tx == 0) {
+                // scales[tile j][row]: eight consecutive rows per thread
+                float *dst = a.scales + (int64_t)blockIdx.x * a.rows + rbase;
+                if (rbase < a.rows) {
+                    *reinterpret_cast<float4 *>(dst) = make_float4(s_row[0], s_row[1], s_row[2], s_row[3]);
+                    *reinterpret_cast<float4 *>(dst + 4) = make_float4(s_row[4], s_row[5], s_row[6], s_row[7]);
+                }
+            }
+        } else {
+            // column maxima over this thread's 8 rows (4 packed registers = 8 columns)
+            uint32_t cm[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                cm[0] = absmax2(cm[0], v[p].x);
+                cm[1] = absmax2(cm[1], v[p].y);
+                cm[2] = absmax2(cm[2], v[p].z);
+                cm[3] = absmax2(cm[3], v[p].w);
+            }
+            if (BLOCK == SNIP_BLOCK_COL_128x1 && kQuant) {
+                // the two row groups of a warp, then the 8 warps through shared memory
+#pragma unroll
+                for (int q = 0; q < 4; ++q) cm[q] = max2(cm[q], __shfl_xor_sync(0xFFFFFFFFu, cm[q], 16));
+                if (lane < 16)
+                    *reinterpret_cast<uint4 *>(&col_amax[warp][4 * tx]) = make_uint4(cm[0], cm[1], cm[2], cm[3]);
+                __syncthreads();
+                if (tid < kTile) {
+                    const uint16_t *h = reinterpret_cast<const uint16_t *>(&col_amax[0][0]);
+                    uint32_t m = 0;
+#pragma unroll
+                    for (int w = 0; w < 8; ++w) m = max(m, (uint32_t)h[w * kTile + tid]);  // non-negative bf16: integer order
+                    float am = __uint_as_float(m << 16);
+                    float s = tile_scale<FMT>(am);
+                    col_scale[tid] = s;
+                    if (CODES && c0 + tid < a.cols) a.scales[(int64_t)blockIdx.y * a.cols + c0 + tid] = s;
+                    if (STATS) my_amax = am;
+                }
+                __syncthreads();
+                const float4 s0 = *reinterpret_cast<const float4 *>(&col_scale[8 * tx]);
+                const float4 s1 = *reinterpret_cast<const float4 *>(&col_scale[8 * tx + 4]);
+                s_col[0] = s0.x; s_col[1] = s0.y; s_col[2] = s0.z; s_col[3] = s0.w;
+                s_col[4] = s1.x; s_col[5] = s1.y; s_col[6] = s1.z; s_col[7] = s1.w;
+            } else {
+                // BLK (or statistics-only): one amax for the whole CTA tile
+                uint32_t m = max2(max2(cm[0], cm[1]), max2(cm[2], cm[3]));
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) m = max2(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
+                float am = fmaxf(bf16lo(m), bf16hi(m));
+                if (lane == 0) red_f[warp][2] = am;
+                __syncthreads();
+                float bm = red_f[0][2];
+#pragma unroll
+                for (int w = 1; w < 8; ++w) bm = fmaxf(bm, red_f[w][2]);
+                my_amax = bm;
+                if (kQuant) {
+                    s_row[0] = tile_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm);
+                    if (CODES && tid == 0) a.scales[(int64_t)blockIdx.y * gridDim.x + blockIdx.x] = s_row[0];
+                }
+                __syncthreads();  // red_f is reused below
+            }
+        }
+    }
+
+    // ---- encode, statistics, store ------------------------------------------------------
+    float sx = 0.0f, se = 0.0f;
+    float rsx[8], rse[8];
+    (void)rsx; (void)rse;
+    if (kQuant) {
+        float sc[8], inv[8];
+        if (BLOCK == SNIP_BLOCK_COL_128x1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { sc[j] = s_col[j]; inv[j] = STATS ? __fdiv_rn(1.0f, s_col[j]) : 0.0f; }
+        } else if (BLOCK == SNIP_BLOCK_BLK_128x128) {
+            const float iv = STATS ? __fdiv_rn(1.0f, s_row[0]) : 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { sc[j] = s_row[0]; inv[j] = iv; }
+        }
+        uint32_t codes[8][2];
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            if (BLOCK == SNIP_BLOCK_ROW_1x128) {
+                const float iv = STATS ? __fdiv_rn(1.0f, s_row[p]) : 0.0f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { sc[j] = s_row[p]; inv[j] = iv; }
+            }
+            float px = 0.0f, pe = 0.0f;
+            quant8<FMT, STATS>(v[p], sc, inv, codes[p], px, pe);
+            if (STATS) { sx += px; se += pe; }
+            if (ROWSTATS) { rsx[p] = px; rse[p] = pe; }
+        }
+        if (CODES) {
+            if (!TRANSPOSED) {
+                const int64_t out_ld = a.cols * kCodeBytes8 / 8;  // bytes per output row
+#pragma unroll
+                for (int p = 0; p < 8; ++p) {
+                    const int64_t r = rbase + p;
+                    if (col_ok && r < a.rows) {
+                        uint8_t *dst = a.codes + r * out_ld + cbase * kCodeBytes8 / 8;
+                        if (FMT == SNIP_FMT_FP8_E4M3)
+                            *reinterpret_cast<uint2 *>(dst) = make_uint2(codes[p][0], codes[p][1]);
+                        else
+                            *reinterpret_cast<uint32_t *>(dst) = codes[p][0];
+                    }
+                }
+            } else {
+                // Transpose the 8x8 sub-block of codes in registers: for column j collect the
+                // codes of rows p = 0..7, then stage line (8*tx + j) of the transposed tile.
+                // Chunk index ty is XOR-ed with tx so that the 16 lanes of a row group hit
+                // distinct banks.
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t lo = 0, hi = 0;
+                    if (FMT == SNIP_FMT_FP8_E4M3) {
+#pragma unroll
+                        for (int p = 0; p < 8; ++p) {
+                            uint32_t b = (codes[p][j >> 2] >> (8 * (j & 3))) & 0xFFu;
+                            if (p < 4) lo |= b << (8 * p); else hi |= b << (8 * (p - 4));
+                        }
+                        uint2 *dst = reinterpret_cast<uint2 *>(stage + (8 * tx + j) * kRowBytes) + (ty ^ tx);
+                        *dst = make_uint2(lo, hi);
+                    } else {
+#pragma unroll
+                        for (int p = 0; p < 8; ++p) {
+                            uint32_t b = (codes[p][0] >> (4 * j)) & 0xFu;
+                            lo |= b << (4 * p);
+                        }
+                        uint32_t *dst = reinterpret_cast<uint32_t *>(stage + (8 * tx + j) * kRowBytes) + (ty ^ tx);
+                        *dst = lo;
+                    }
+                }
+                __syncthreads();
+                // write out: line c of the staged tile holds rows r0..r0+127 of column c0+c
+                const int64_t out_ld = a.rows * kCodeBytes8 / 8;  // bytes per transposed row
+                constexpr int kChunks = kRowBytes / 16;            // 16-byte chunks per line
+                const int valid_rows = (int)min((int64_t)kTile, a.rows - r0);
+                for (int idx = tid; idx < kTile * kChunks; idx += kThreads) {
+                    const int c = idx / kChunks, q = idx % kChunks;
+                    if (c0 + c >= a.cols) continue;
+                    const int key = (c >> 3) & 15;
+                    uint4 o;
+                    if (FMT == SNIP_FMT_FP8_E4M3) {
+                        const uint2 *src = reinterpret_cast<const uint2 *>(stage + c * kRowBytes);
+                        uint2 h0 = src[(2 * q) ^ key], h1 = src[(2 * q + 1) ^ key];
+                        o = make_uint4(h0.x, h0.y, h1.x, h1.y);
+                        if (16 * q >= valid_rows) continue;  // rows is a multiple of 64
+                    } else {
+                        const uint32_t *src = reinterpret_cast<const uint32_t *>(stage + c * kRowBytes);
+                        o = make_uint4(src[(4 * q) ^ key], src[(4 * q + 1) ^ key], src[(4 * q + 2) ^ key],
+                                       src[(4 * q + 3) ^ key]);
+                        if (32 * q >= valid_rows) continue;
+                    }
+                    uint8_t *dst = a.codes + (c0 + c) * out_ld + r0 * kCodeBytes8 / 8 + 16 * q;
+                    *reinterpret_cast<uint4 *>(dst) = o;
+                }
+            }
+        }
+    } else if (STATS) {
+        // BF16: identity, only sum x^2
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            const uint32_t w[4] = {v[p].x, v[p].y, v[p].z, v[p].w};
+            float px = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float x0 = bf16lo(w[i]), x1 = bf16hi(w[i]);
+                px = fmaf(x0, x0, px);
+                px = fmaf(x1, x1, px);
+            }
+            sx += px;
+            if (ROWSTATS) { rsx[p] = px; rse[p] = 0.0f; }
+        }
+    }
+
+    // ---- statistics: warp -> CTA -> one partial per CTA ------------------------------------
+    if (ROWSTATS) {
+        // per row: add the 16 lanes that share the row, lane tx==0 writes {sum x^2, sum err^2}
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+#pragma unroll
+            for (int off = 1; off < 16; off <<= 1) {
+                rsx[p] += __shfl_xor_sync(0xFFFFFFFFu, rsx[p], off);
+                rse[p] += __shfl_xor_sync(0xFFFFFFFFu, rse[p], off);
+            }
+        }
+        if (tx == 0 && rbase < a.rows) {
+            float2 *dst = a.row_partials + (int64_t)blockIdx.x * a.rows + rbase;
+#pragma unroll
+            for (int p = 0; p < 8; ++p) dst[p] = make_float2(rsx[p], rse[p]);
+        }
+    }
+    if (STATS) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            sx += __shfl_xor_sync(0xFFFFFFFFu, sx, off);
+            se += __shfl_xor_sync(0xFFFFFFFFu, se, off);
+            my_amax = fmaxf(my_amax, __shfl_xor_sync(0xFFFFFFFFu, my_amax, off));
+        }
+        if (lane == 0) { red_f[warp][0] = sx; red_f[warp][1] = se; red_f[warp][2] = my_amax; }
+        __syncthreads();
+        if (tid == 0) {
+            double dx = 0.0, de = 0.0;
+            float am = 0.0f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) { dx += (double)red_f[w][0]; de += (double)red_f[w][1]; am = fmaxf(am, red_f[w][2]); }
+            CtaPartial *dst = a.partials + (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+            dst->sumsq_x = dx;
+            dst->sumsq_err = de;
+            dst->amax = am;
+        }
+    }
+}
+
+// Fixed-order reduction of the per-CTA partials into one snip_stats_t (deterministic).
+__global__ void __launch_bounds__(1024) stats_reduce_kernel(const CtaPartial *partials, int64_t n, snip_stats_t *out)
+{
+    __shared__ double sh_x[1024], sh_e[1024];
+    __shared__ float sh_m[1024];
+    double dx = 0.0, de = 0.0;
+    float am = 0.0f;
+    for (int64_t i = threadIdx.x; i < n; i += 1024) {
+        dx += partials[i].sumsq_x;
+        de += partials[i].sumsq_err;
+        am = fmaxf(am, partials[i].amax);
+    }
+    sh_x[threadIdx.x] = dx; sh_e[threadIdx.x] = de; sh_m[threadIdx.x] = am;
+    __syncthreads();
+    for (int s = 512; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) {
+            sh_x[threadIdx.x] += sh_x[threadIdx.x + s];
+            sh_e[threadIdx.x] += sh_e[threadIdx.x + s];
+            sh_m[threadIdx.x] = fmaxf(sh_m[threadIdx.x], sh_m[threadIdx.x + s]);
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        out->sumsq_x = sh_x[0];
+        out->sumsq_err = sh_e[0];
+        out->amax = sh_m[0];
+        out->reserved = 0;
+    }
+}
+
+// Per-row sums: add the column-tile partials of each row in ascending tile order.
+__global__ void row_stats_reduce_kernel(const float2 *row_partials, int64_t rows, int64_t col_tiles, double *row_stats)
+{
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    double dx = 0.0, de = 0.0;
+    for (int64_t j = 0; j < col_tiles; ++j) {
+        float2 p = row_partials[j * rows + r];
+        dx += (double)p.x;
+        de += (double)p.y;
+    }
+    row_stats[2 * r] = dx;
+    row_stats[2 * r + 1] = de;
+}
+
+template <int FMT, int BLOCK, bool TRANSPOSED>
+void launch_variant(const QuantArgs &a, bool codes, bool stats, bool rowstats, dim3 grid, cudaStream_t st)
+{
+    if (codes && stats && rowstats) quantize_kernel<FMT, BLOCK, TRANSPOSED, true, true, true><<<grid, kThreads, 0, st>>>(a);
+    else if (codes && stats) quantize_kernel<FMT, BLOCK, TRANSPOSED, true, true, false><<<grid, kThreads, 0, st>>>(a);
+    else if (codes) quantize_kernel<FMT, BLOCK, TRANSPOSED, true, false, false><<<grid, kThreads, 0, st>>>(a);
+    else if (rowstats) quantize_kernel<FMT, BLOCK, false, false, true, true><<<grid, kThreads, 0, st>>>(a);
+    else quantize_kernel<FMT, BLOCK, false, false, true, false><<<grid, kThreads, 0, st>>>(a);
+}
+
+template <int FMT>
+void launch_fmt(const QuantArgs &a, int block, bool transposed, bool codes, bool stats, bool rowstats, dim3 grid, cudaStream_t st)
+{
+    if (block == SNIP_BLOCK_ROW_1x128) {
+        if (transposed) launch_variant<FMT, SNIP_BLOCK_ROW_1x128, true>(a, codes, stats, rowstats, grid, st);
+        else launch_variant<FMT, SNIP_BLOCK_ROW_1x128, false>(a, codes, stats, rowstats, grid, st);
+    } else if (block == SNIP_BLOCK_COL_128x1) {
+        if (transposed) launch_variant<FMT, SNIP_BLOCK_COL_128x1, true>(a, codes, stats, rowstats, grid, st);
+        else launch_variant<FMT, SNIP_BLOCK_COL_128x1, false>(a, codes, stats, rowstats, grid, st);
+    } else {
+        if (transposed) launch_variant<FMT, SNIP_BLOCK_BLK_128x128, true>(a, codes, stats, rowstats, grid, st);
+        else launch_variant<FMT, SNIP_BLOCK_BLK_128x128, false>(a, codes, stats, rowstats, grid, st);
+    }
+}
+
+size_t stats_ws_bytes(int64_t rows, int64_t cols, bool rowstats)
+{
+    const int64_t tr = ceil_div(rows, kTile), tc = ceil_div(cols, kTile);
+    size_t b = align_up((size_t)(tr * tc) * sizeof(CtaPartial), 256);
+    if (rowstats) b += align_up((size_t)(tc * rows) * sizeof(float2), 256);
+    return b;
+}
+
+}  // namespace
+
+// Internal entry used by snip_quantize and by the linear-layer calls.
+int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags,
+                  void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes,
+                  cudaStream_t st)
+{
+    if (!x || !valid_fmt(fmt) || !valid_block(block)) return SNIP_ERR_ARG;
+    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0) return SNIP_ERR_SHAPE;
+    const bool want_stats = (flags & SNIP_Q_STATS) != 0;
+    const bool want_rows = row_stats != nullptr;
+    const bool want_codes = fmt != SNIP_FMT_BF16 && !(flags & SNIP_Q_NO_CODES);
+    const bool transposed = (flags & SNIP_Q_TRANSPOSED) != 0;
+    if (want_stats && !stats) return SNIP_ERR_ARG;
+    if (want_codes && (!codes || !scales)) return SNIP_ERR_ARG;
+    if (!want_codes && !want_stats && !want_rows) return SNIP_ERR_ARG;  // nothing to do
+    if (!aligned16(x) || (want_codes && (!aligned16(codes) || !aligned16(scales))) || (stats && !aligned16(stats)) ||
+        (row_stats && !aligned16(row_stats)))
+        return SNIP_ERR_ALIGN;
+    const bool any_stats = want_stats || want_rows;
+    const size_t need = any_stats ? stats_ws_bytes(rows, cols, want_rows) : 0;
+    if (need > 0 && (!ws || ws_bytes < need)) return SNIP_ERR_WORKSPACE;
+    if (need > 0 && !aligned16(ws)) return SNIP_ERR_ALIGN;
+    int rc = require_sm100();
+    if (rc != SNIP_OK) return rc;
+
+    const int64_t tr = ceil_div(rows, kTile), tc = ceil_div(cols, kTile);
+    if (tr > 65535) return SNIP_ERR_SHAPE;
+    QuantArgs a;
+    a.x = static_cast<const uint16_t *>(x);
+    a.rows = rows; a.cols = cols; a.ld = ld;
+    a.codes = want_codes ? static_cast<uint8_t *>(codes) : nullptr;
+    a.scales = want_codes ? scales : nullptr;
+    a.partials = any_stats ? static_cast<CtaPartial *>(ws) : nullptr;
+    a.row_partials = want_rows ? reinterpret_cast<float2 *>(static_cast<uint8_t *>(ws) + align_up((size_t)(tr * tc) * sizeof(CtaPartial), 256)) : nullptr;
+    dim3 grid((unsigned)tc, (unsigned)tr);
+    if (fmt == SNIP_FMT_FP8_E4M3) launch_fmt<SNIP_FMT_FP8_E4M3>(a, block, transposed, want_codes, any_stats, want_rows, grid, st);
+    else if (fmt == SNIP_FMT_FP4_E2M1) launch_fmt<SNIP_FMT_FP4_E2M1>(a, block, transposed, want_codes, any_stats, want_rows, grid, st);
+    else launch_variant<SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, false>(a, false, true, want_rows, grid, st);
+    SNIP_CUDA_TRY(cudaGetLastError());
+    if (want_stats) {
+        stats_reduce_kernel<<<1, 1024, 0, st>>>(a.partials, tr * tc, stats);
+        SNIP_CUDA_TRY(cudaGetLastError());
+    }
+    if (want_rows) {
+        row_stats_reduce_kernel<<<(unsigned)ceil_div(rows, 256), 256, 0, st>>>(a.row_partials, rows, tc, row_stats);
+        SNIP_CUDA_TRY(cudaGetLastError());
+    }
+    return SNIP_OK;
+}
+
+}  // namespace snip
+
+extern "C" int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int block, uint32_t flags,
+                                   size_t *codes_bytes, size_t *scales_bytes, size_t *ws_bytes)
+{
+    using namespace snip;
+    if (!valid_fmt(fmt) || !valid_block(block)) return SNIP_ERR_ARG;
+    if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
+    const bool want_codes = fmt != SNIP_FMT_BF16 && !(flags & SNIP_Q_NO_CODES);
+    size_t cb = 0, sb = 0;
+    if (want_codes) {
+        cb = (size_t)(rows * cols) / (fmt == SNIP_FMT_FP4_E2M1 ? 2 : 1);
+        const int64_t tr = ceil_div(rows, 128), tc = ceil_div(cols, 128);
+        int64_t n = block == SNIP_BLOCK_ROW_1x128 ? tc * rows : block == SNIP_BLOCK_COL_128x1 ? tr * cols : tr * tc;
+        sb = (size_t)n * sizeof(float);
+    }
+    if (codes_bytes) *codes_bytes = cb;
+    if (scales_bytes) *scales_bytes = sb;
+    if (ws_bytes) *ws_bytes = stats_ws_bytes(rows, cols, true);
+    return SNIP_OK;
+}
+
+extern "C" int snip_quantize(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,
+                             uint32_t flags, void *codes, float *scales, snip_stats_t *stats, double *row_stats,
+                             void *ws, size_t ws_bytes, void *stream)
+{
+    return snip::quantize_impl(x, rows, cols, ld, fmt, block, flags, codes, scales, stats, row_stats, ws, ws_bytes,
+                               static_cast<cudaStream_t>(stream));
+}
