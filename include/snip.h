@@ -121,7 +121,9 @@ const char *snip_last_cuda_error(void);
 /*
  * Byte sizes of the outputs and of the workspace that snip_quantize needs for a rows x cols
  * input.  Host-only.  Any of the three output pointers may be NULL.
- * codes_bytes: rows*cols (FP8), rows*cols/2 (FP4), 0 (BF16 or NO_CODES).
+ * codes_bytes: rows*cols (FP8), rows*cols/2 (FP4; plus 64 bytes of tail slack when a dimension is
+ * not a multiple of 128: the GEMM may read, and ignores, up to 32 bytes past the last code), 0
+ * (BF16 or NO_CODES).
  * scales_bytes: 4 * number of tiles (0 for BF16 or NO_CODES).
  * ws_bytes: 0 unless SNIP_Q_STATS is set or row_stats will be requested (the value returned
  * covers both).

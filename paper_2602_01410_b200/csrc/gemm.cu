@@ -42,6 +42,7 @@ struct GemmArgs {
     void *out;
     int64_t ldo;
     int32_t accumulate;
+    uint32_t stage_tx_bytes;   // bytes the two TMA loads of one stage report to the barrier
     uint32_t *status;
 };
 
@@ -187,7 +188,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(s), C::kStageBytes);
+                    mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
                     tma_load_2d(smem_a0 + s * C::kABytes, &tmA, full_bar(s), ks * C::kStageElemsX, m_idx * BM);
                     tma_load_2d(smem_b0 + s * C::kBBytes, &tmB, full_bar(s), ks * C::kStageElemsX, n_idx * BN);
                 }
@@ -487,6 +488,7 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     g.sb = sb; g.sb_chunk_stride = sb_chunk_stride; g.sb_blk_stride = sb_blk_stride;
     g.out = out; g.ldo = No; g.accumulate = accumulate;
     g.status = static_cast<uint32_t *>(ws);
+    g.stage_tx_bytes = 0;
     const bool f32 = out_dtype == SNIP_OUT_FP32;
 
     CUtensorMap tmA, tmB;
@@ -496,6 +498,7 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
         rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, No, Kc, Kc * 2, 64, 256);
         if (rc) return rc;
         const uint32_t idesc = make_idesc(1, 1, BM, 256);
+        g.stage_tx_bytes = (BM + 256) * 128;
         return f32 ? launch_gemm<MmaKind::F16, 256, SCALE_NONE, true>(tmA, tmB, g, idesc, st)
                    : launch_gemm<MmaKind::F16, 256, SCALE_NONE, false>(tmA, tmB, g, idesc, st);
     }
@@ -507,19 +510,29 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
         rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN);
         if (rc) return rc;
         const uint32_t idesc = make_idesc_block_scaled(1, 1, BM, BN);
+        g.stage_tx_bytes = (BM + BN) * 128;
         return launch_gemm_scale<MmaKind::MXF4, BN>(scale_mode, f32, tmA, tmB, g, idesc, st);
     }
     // FP8 x FP8 and the mixed pairs: kind::f8f6f4; FP4 operands are expanded by the TMA unit to one
     // 16-byte-aligned group per 16 elements, which is the layout this MMA kind reads
     constexpr int BN = 256;
     const bool a4 = fmt_a == SNIP_FMT_FP4_E2M1, b4 = fmt_b == SNIP_FMT_FP4_E2M1;
-    rc = make_operand_map(&tmA, a_codes, a4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, Kc,
+    // The expanding 4-bit tensor-map type only accepts an inner extent that is a multiple of 128
+    // elements.  A contraction length ending in a 64-wide tile is therefore declared rounded up: the
+    // extra 64 codes of each row are the first codes of the next row (for the last row, 32 bytes of
+    // the slack that snip_quantize_sizes reserves); they meet zero-filled FP8 codes of the other
+    // operand, whose map has the exact extent, so they contribute nothing.
+    const int64_t kpad = ceil_div(Kc, 128) * 128;
+    rc = make_operand_map(&tmA, a_codes, a4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, a4 ? kpad : Kc,
                           a4 ? Kc / 2 : Kc, 128, BM);
     if (rc) return rc;
-    rc = make_operand_map(&tmB, b_codes, b4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc,
+    rc = make_operand_map(&tmB, b_codes, b4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, No, b4 ? kpad : Kc,
                           b4 ? Kc / 2 : Kc, 128, BN);
     if (rc) return rc;
     const uint32_t idesc = make_idesc(a4 ? 5 : 0, b4 ? 5 : 0, BM, BN);
+    // an FP4 operand expanded by the TMA unit occupies 128 B per row in shared memory but reports
+    // only its 64 packed source bytes to the barrier
+    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128);
     return launch_gemm_scale<MmaKind::F8F6F4, BN>(scale_mode, f32, tmA, tmB, g, idesc, st);
 }
 

@@ -21,7 +21,7 @@ enum { SCALE_NONE = 0, SCALE_BLOCK_B = 1, SCALE_VEC_B = 2 };
 size_t code_bytes(int fmt, int64_t rows, int64_t cols)
 {
     if (fmt == SNIP_FMT_FP8_E4M3) return (size_t)(rows * cols);
-    if (fmt == SNIP_FMT_FP4_E2M1) return (size_t)(rows * cols / 2);
+    if (fmt == SNIP_FMT_FP4_E2M1) return (size_t)(rows * cols / 2) + 64;  // + tail slack, see snip_quantize_sizes
     return (size_t)(rows * cols * 2);  // bf16 transposed copy
 }
 size_t scale_bytes(int block, int64_t rows, int64_t cols)

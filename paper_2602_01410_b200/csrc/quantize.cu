@@ -555,6 +555,9 @@ extern "C" int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int bloc
     size_t cb = 0, sb = 0;
     if (want_codes) {
         cb = (size_t)(rows * cols) / (fmt == SNIP_FMT_FP4_E2M1 ? 2 : 1);
+        // 64 bytes of tail slack after FP4 codes: the GEMM's 4-bit tensor map may read (and ignore)
+        // up to 32 bytes past the last row when the contraction length ends in a 64-wide tile
+        if (fmt == SNIP_FMT_FP4_E2M1 && ((rows % 128) || (cols % 128))) cb += 64;
         const int64_t tr = ceil_div(rows, 128), tc = ceil_div(cols, 128);
         int64_t n = block == SNIP_BLOCK_ROW_1x128 ? tc * rows : block == SNIP_BLOCK_COL_128x1 ? tr * cols : tr * tc;
         sb = (size_t)n * sizeof(float);

@@ -51,7 +51,7 @@ def test_quantize_sizes_and_shape_errors(lib):
     assert lib.snip_quantize_sizes(256, 320, 1, 0, 0, cb, sb, wb) == 0
     assert cb.value == 256 * 320 and sb.value == 4 * 3 * 256
     assert lib.snip_quantize_sizes(256, 320, 2, 1, 0, cb, sb, wb) == 0
-    assert cb.value == 256 * 320 // 2 and sb.value == 4 * 2 * 320
+    assert cb.value == 256 * 320 // 2 + 64 and sb.value == 4 * 2 * 320
     assert lib.snip_quantize_sizes(256, 320, 2, 2, 0, cb, sb, wb) == 0
     assert sb.value == 4 * 2 * 3
     assert lib.snip_quantize_sizes(256, 320, 0, 2, 0, cb, sb, wb) == 0 and cb.value == 0 and sb.value == 0

@@ -30,7 +30,7 @@ def check_quantize(api, x_bits, fmt, block, transposed, row_stats=False):
     codes, scales, stats, rstats = api.snip_quantize(to_dev(x_bits), fmt, block, flags, want_row_stats=row_stats)
     torch.cuda.synchronize()
     want_codes = q.packed(transposed)
-    got_codes = codes.cpu().numpy().reshape(want_codes.shape)
+    got_codes = codes.cpu().numpy()[:want_codes.size].reshape(want_codes.shape)
     assert np.array_equal(got_codes, want_codes), f"codes differ at {np.argwhere(got_codes != want_codes)[:5]}"
     got_scales = scales.cpu().numpy().reshape(q.scales.shape)
     assert np.array_equal(got_scales.view(np.uint32), q.scales.view(np.uint32))
@@ -80,7 +80,7 @@ def test_degenerate_tiles(api, fmt, block):
     q = orc.quantize(x, fmt, block)
     codes, scales, _, _ = api.snip_quantize(to_dev(x), fmt, block, 0)
     torch.cuda.synchronize()
-    assert np.array_equal(codes.cpu().numpy().reshape(q.packed().shape), q.packed())
+    assert np.array_equal(codes.cpu().numpy()[:q.packed().size].reshape(q.packed().shape), q.packed())
     assert np.array_equal(scales.cpu().numpy().reshape(q.scales.shape).view(np.uint32), q.scales.view(np.uint32))
 
 
