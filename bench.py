@@ -1,0 +1,515 @@
+#!/usr/bin/env python
+"""Benchmark of the SNIP mixed-precision linear hot path on B200.
+
+A step = one transformer block of the Llama-7B-shaped workload (tokens 16384; fused QKV, O,
+gate, up, down): for every linear the forward, input-gradient and weight-gradient GEMMs, each
+preceded by the quantization of its two operands with fused error-norm statistics, run once with
+every GEMM in FP4 E2M1 and once with every GEMM in FP8 E4M3.
+
+Prints ONE JSON line (rank 0).  `value` is GEMM TFLOP/s (2*M*N*K per GEMM) over the whole step,
+quantizers and statistics included, with inputs resident in HBM.  `roofline` describes the
+dominant kernel family (the GEMM kernels of the slower format), timed with CUDA events around
+each launch inside the timed region.  `e2e` repeats the step through the snip_linear_* calls with
+the inputs starting in pinned host memory.  `cpu_baseline` times the CPU oracle on a bounded
+sample on this machine's host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 7b|1b|small]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FMT_BF16, FMT_FP8, FMT_FP4 = 0, 1, 2
+FMT_NAME = {0: "bf16", 1: "fp8_e4m3", 2: "fp4_e2m1"}
+NOMINAL_RATIO = {0: 1.0, 1: 2.0, 2: 4.0}   # dense tensor peak relative to bf16
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        for ln in self.lines:
+            f = [v.strip() for v in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [c for c, p in zip(sm, power) if p > 300] or sm
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+
+WORKLOADS = {
+    # name: (config index in paper_2602_01410_b200.workloads.CONFIGS, tokens override)
+    "7b": (3, None),
+    "1b": (1, None),
+    "small": (0, None),
+}
+
+
+def make_device_inputs(cfg, torch, device, seed):
+    """bf16 tensors of one block, drawn on the device with the recipe of workloads.py (normal X
+    with outlier channels, N(0,0.02) W, row-scaled dY).  The bench needs the distribution, not
+    the exact bytes; parity tests use the host generators."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    M = cfg.M
+    lin = []
+    for li, L in enumerate(cfg.linears):
+        x = torch.randn(M, L.K, generator=g, device=device, dtype=torch.float32)
+        n_out = max(1, int(-(-cfg.outlier_frac * L.K // 1)))
+        cols = torch.randperm(L.K, generator=g, device=device)[:n_out]
+        x[:, cols] *= cfg.outlier_scale
+        w = torch.randn(L.N, L.K, generator=g, device=device, dtype=torch.float32) * 0.02
+        dy = torch.randn(M, L.N, generator=g, device=device, dtype=torch.float32) * 1e-3
+        dy *= torch.exp(torch.randn(M, 1, generator=g, device=device, dtype=torch.float32))
+        lin.append((x.to(torch.bfloat16), w.to(torch.bfloat16), dy.to(torch.bfloat16)))
+        del x, w, dy
+    return lin
+
+
+class Step:
+    """Device buffers and the call sequence of one step."""
+
+    def __init__(self, api, torch, cfg, device, formats):
+        self.api, self.torch, self.cfg, self.formats = api, torch, cfg, formats
+        self.inputs = make_device_inputs(cfg, torch, device, 260201410)
+        M = cfg.M
+        self.out = []
+        ws_bytes = 0
+        for L in cfg.linears:
+            self.out.append((torch.empty(M, L.N, dtype=torch.bfloat16, device=device),
+                             torch.empty(M, L.K, dtype=torch.bfloat16, device=device),
+                             torch.empty(L.N, L.K, dtype=torch.bfloat16, device=device)))
+            for op in (api.OP_FWD, api.OP_DGRAD, api.OP_WGRAD):
+                for f in formats:
+                    ws_bytes = max(ws_bytes, api.snip_workspace_size(op, M, L.N, L.K, f, f)[1])
+        self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
+        n_gemm = len(cfg.linears) * 3 * len(formats)
+        self.stats = torch.zeros(n_gemm * 2, 32, dtype=torch.uint8, device=device)  # one 16-byte-aligned snip_stats_t per row
+        self.flops = sum(2.0 * M * L.N * L.K * 3 for L in cfg.linears) * len(formats)
+        self.launches_per_step = n_gemm * 5  # 2 quantizers + 2 statistics reductions + 1 GEMM
+
+    # -- the step through the snip_linear_* entry points (what a user calls) -------------
+    def run_linear_calls(self):
+        api = self.api
+        i = 0
+        for f in self.formats:
+            for (x, w, dy), (y, dx, dw) in zip(self.inputs, self.out):
+                M, K = x.shape
+                N = w.shape[0]
+                lib, p, st = api._lib, api._p, api._stream()
+                sa, sb = self.stats[2 * i], self.stats[2 * i + 1]
+                api._check("snip_linear_fwd", lib.snip_linear_fwd(p(x), p(w), p(y), M, N, K, f, f, api.OUT_BF16, p(sa), p(sb), p(self.ws), self.ws.numel(), st)); i += 1
+                sa, sb = self.stats[2 * i], self.stats[2 * i + 1]
+                api._check("snip_linear_dgrad", lib.snip_linear_dgrad(p(dy), p(w), p(dx), M, N, K, f, f, api.OUT_BF16, p(sa), p(sb), p(self.ws), self.ws.numel(), st)); i += 1
+                sa, sb = self.stats[2 * i], self.stats[2 * i + 1]
+                api._check("snip_linear_wgrad", lib.snip_linear_wgrad(p(dy), p(x), p(dw), M, N, K, f, f, api.OUT_BF16, 0, p(sa), p(sb), p(self.ws), self.ws.numel(), st)); i += 1
+
+    # -- the same device work as separate quantize / GEMM calls, so that CUDA events can bracket
+    #    every GEMM launch inside the timed region ------------------------------------------------
+    def _alloc_decomposed(self):
+        api, torch = self.api, self.torch
+        cb = sb = wb = 0
+        M = self.cfg.M
+        for L in self.cfg.linears:
+            for (r, c) in ((M, L.K), (L.N, L.K), (M, L.N)):
+                for blk in (api.BLOCK_ROW, api.BLOCK_COL, api.BLOCK_BLK):
+                    a, b, w = api.snip_quantize_sizes(r, c, FMT_FP8, blk, api.Q_STATS)
+                    cb, sb, wb = max(cb, a), max(sb, b), max(wb, w)
+        dev = self.ws.device
+        self.codes = [torch.empty(cb, dtype=torch.uint8, device=dev) for _ in range(2)]
+        self.scales = [torch.empty(sb // 4, dtype=torch.float32, device=dev) for _ in range(2)]
+        self.qws = torch.empty(wb, dtype=torch.uint8, device=dev)
+        self.gws = torch.zeros(1024, dtype=torch.uint8, device=dev)
+
+    def run_decomposed(self, events=None):
+        api, torch = self.api, self.torch
+        if not hasattr(self, "codes"):
+            self._alloc_decomposed()
+        lib, p, st = api._lib, api._p, api._stream()
+        T = api.Q_TRANSPOSED
+        i = 0
+
+        def quant(x, fmt, block, flags, slot, stats):
+            r, c = x.shape
+            api._check("snip_quantize", lib.snip_quantize(p(x), r, c, c, fmt, block, flags | api.Q_STATS, p(self.codes[slot]), p(self.scales[slot]),
+                                                          p(stats), None, p(self.qws), self.qws.numel(), st))
+
+        def gemm(op, fmt, ra, ca, blka, ta, rb, cb_, blkb, tb, out, flops):
+            a = api.make_qtensor(self.codes[0], self.scales[0], ra, ca, fmt, blka, ta)
+            b = api.make_qtensor(self.codes[1], self.scales[1], rb, cb_, fmt, blkb, tb)
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            api._check("snip_gemm_quantized", lib.snip_gemm_quantized(op, a, b, p(out), api.OUT_BF16, 0, p(self.gws), self.gws.numel(), st))
+            if events is not None:
+                e1.record()
+                events.append((fmt, op, flops, e0, e1))
+
+        for f in self.formats:
+            for (x, w, dy), (y, dx, dw) in zip(self.inputs, self.out):
+                M, K = x.shape
+                N = w.shape[0]
+                fl = 2.0 * M * N * K
+                quant(x, f, api.BLOCK_ROW, 0, 0, self.stats[2 * i]); quant(w, f, api.BLOCK_BLK, 0, 1, self.stats[2 * i + 1]); i += 1
+                gemm(api.OP_FWD, f, M, K, api.BLOCK_ROW, 0, N, K, api.BLOCK_BLK, 0, y, fl)
+                quant(dy, f, api.BLOCK_ROW, 0, 0, self.stats[2 * i]); quant(w, f, api.BLOCK_BLK, T, 1, self.stats[2 * i + 1]); i += 1
+                gemm(api.OP_DGRAD, f, M, N, api.BLOCK_ROW, 0, N, K, api.BLOCK_BLK, 1, dx, fl)
+                quant(dy, f, api.BLOCK_COL, T, 0, self.stats[2 * i]); quant(x, f, api.BLOCK_COL, T, 1, self.stats[2 * i + 1]); i += 1
+                gemm(api.OP_WGRAD, f, M, N, api.BLOCK_COL, 1, M, K, api.BLOCK_COL, 1, dw, fl)
+
+
+class KernelTimer:
+    """Times one kernel family alone (pre-quantized operands), CUDA events around each launch,
+    rotating over operand sets so that L2 cannot serve the inputs."""
+
+    def __init__(self, api, torch, cfg, device):
+        self.api, self.torch, self.cfg, self.device = api, torch, cfg, device
+
+    def gemm(self, fmt, op, lin_index, iters=20, warmup=3):
+        api, torch = self.api, self.torch
+        L = self.cfg.linears[lin_index]
+        M, N, K = self.cfg.M, L.N, L.K
+        g = torch.Generator(device=self.device); g.manual_seed(1)
+        def rnd(r, c, s=1.0):
+            return (torch.randn(r, c, generator=g, device=self.device, dtype=torch.float32) * s).to(torch.bfloat16)
+        if op == api.OP_FWD:
+            A, B, out_shape = rnd(M, K), rnd(N, K, 0.02), (M, N)
+            qa = api.snip_quantize(A, fmt, api.BLOCK_ROW); qb = api.snip_quantize(B, fmt, api.BLOCK_BLK)
+            a = api.make_qtensor(qa[0], qa[1], M, K, fmt, api.BLOCK_ROW); b = api.make_qtensor(qb[0], qb[1], N, K, fmt, api.BLOCK_BLK)
+        elif op == api.OP_DGRAD:
+            A, B, out_shape = rnd(M, N, 1e-3), rnd(N, K, 0.02), (M, K)
+            qa = api.snip_quantize(A, fmt, api.BLOCK_ROW); qb = api.snip_quantize(B, fmt, api.BLOCK_BLK, api.Q_TRANSPOSED)
+            a = api.make_qtensor(qa[0], qa[1], M, N, fmt, api.BLOCK_ROW); b = api.make_qtensor(qb[0], qb[1], N, K, fmt, api.BLOCK_BLK, True)
+        else:
+            A, B, out_shape = rnd(M, N, 1e-3), rnd(M, K), (N, K)
+            qa = api.snip_quantize(A, fmt, api.BLOCK_COL, api.Q_TRANSPOSED); qb = api.snip_quantize(B, fmt, api.BLOCK_COL, api.Q_TRANSPOSED)
+            a = api.make_qtensor(qa[0], qa[1], M, N, fmt, api.BLOCK_COL, True); b = api.make_qtensor(qb[0], qb[1], M, K, fmt, api.BLOCK_COL, True)
+        out = torch.empty(out_shape, dtype=torch.bfloat16, device=self.device)
+        ws = torch.zeros(1024, dtype=torch.uint8, device=self.device)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.device)
+        times = []
+        for i in range(warmup + iters):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            api.snip_gemm_quantized(op, a, b, out_shape, api.OUT_BF16, out=out, ws=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= warmup:
+                times.append(e0.elapsed_time(e1))
+        assert api.snip_poll_status(ws) == 0
+        return 2.0 * M * N * K, times
+
+    def quantizer(self, fmt, block, transposed, rows, cols, iters=20, warmup=3):
+        api, torch = self.api, self.torch
+        g = torch.Generator(device=self.device); g.manual_seed(2)
+        xs = [torch.randn(rows, cols, generator=g, device=self.device, dtype=torch.float32).to(torch.bfloat16) for _ in range(3)]
+        flags = api.Q_STATS | (api.Q_TRANSPOSED if transposed else 0)
+        codes, scales, stats, _ = api.snip_quantize(xs[0], fmt, block, flags)
+        _, _, wb = api.snip_quantize_sizes(rows, cols, fmt, block, flags)
+        ws = torch.empty(wb, dtype=torch.uint8, device=self.device)
+        times = []
+        for i in range(warmup + iters):
+            x = xs[i % 3]
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            api.snip_quantize(x, fmt, block, flags, codes=codes, scales=scales, stats=stats, ws=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= warmup:
+                times.append(e0.elapsed_time(e1))
+        bytes_per_elt = 2.0 + (1.0 if fmt == FMT_FP8 else 0.5) + 4.0 / 128.0
+        return bytes_per_elt * rows * cols, times
+
+
+def cpu_baseline_sample(cfg, tokens=4096):
+    """The CPU oracle, as it stands, on a bounded sample: `tokens` rows of the O projection
+    (K -> K) through quantize + fwd + dgrad + wgrad in FP8.  Returns (TFLOP/s, cores, text)."""
+    from oracle import snip_oracle as orc
+    from paper_2602_01410_b200 import workloads as wl
+    li = 1 if len(cfg.linears) > 1 else 0
+    L = cfg.linears[li]
+    x, w, dy = wl.linear_inputs(cfg, 0, li, M=tokens)
+    t0 = time.perf_counter()
+    orc.linear_fwd(x, w, FMT_FP8, FMT_FP8)
+    orc.linear_dgrad(dy, w, FMT_FP8, FMT_FP8)
+    orc.linear_wgrad(dy, x, FMT_FP8, FMT_FP8)
+    dt = time.perf_counter() - t0
+    flops = 3 * 2.0 * tokens * L.N * L.K
+    return flops / dt / 1e12, orc.num_threads(), (f"{tokens} tokens of linear '{L.name}' ({L.K}->{L.N}), FP8: 3 quantize pairs + "
+                                                   f"fwd/dgrad/wgrad float64 GEMMs, {dt:.2f} s")
+
+
+def run_profile_case(name):
+    """A few launches of one kernel on a small case (inputs above L2 size, well under a GB)."""
+    import torch
+    from paper_2602_01410_b200 import api, workloads as wl
+    from dataclasses import replace
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    parts = name.split("_")
+    fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4}[parts[1]]
+    if parts[0] == "quantize":
+        kind = "_".join(parts[2:])
+        block, tr = {"row": (api.BLOCK_ROW, False), "col_t": (api.BLOCK_COL, True), "blk_t": (api.BLOCK_BLK, True),
+                     "blk": (api.BLOCK_BLK, False), "col": (api.BLOCK_COL, False)}[kind]
+        kt = KernelTimer(api, torch, wl.CONFIGS[3], device)
+        by, times = kt.quantizer(fmt, block, tr, 16384, 4096, iters=3, warmup=1)
+        print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
+    else:
+        op = {"fwd": api.OP_FWD, "dgrad": api.OP_DGRAD, "wgrad": api.OP_WGRAD}[parts[2]]
+        M, N, K = (int(v) for v in parts[3].split("x")) if len(parts) > 3 else (4096, 4096, 4096)
+        cfg = replace(wl.CONFIGS[3], M=M, linears=(wl.Linear("case", K, N),))
+        kt = KernelTimer(api, torch, cfg, device)
+        if fmt == FMT_BF16:
+            raise SystemExit("bf16 GEMM cases run through snip_linear_*; use fp8/fp4 here")
+        fl, times = kt.gemm(fmt, op, 0, iters=3, warmup=1)
+        print(f"{name}: {fl / (min(times) * 1e-3) / 1e12:.0f} TFLOP/s best of {len(times)}")
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on a bounded sample per step (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2602_01410_b200 import workloads as wl
+    cfg = wl.CONFIGS[WORKLOADS[args.workload][0]]
+    tokens = 512
+    vals = []
+    for i in range(args.warmup + args.steps):
+        v, cores, sample = cpu_baseline_sample(cfg, tokens)
+        if i >= args.warmup:
+            vals.append(v)
+    v = sum(vals) / len(vals)
+    L = cfg.linears[1 if len(cfg.linears) > 1 else 0]
+    ms = 3 * 2.0 * tokens * L.N * L.K / (v * 1e12) * 1e3
+    line = {"impl": "reference", "metric": "mixed-precision linear fwd+dgrad+wgrad TFLOP/s", "value": v, "unit": "TFLOP/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: sample of {sample}"},
+            "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="snip")
+    ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-legs", action="store_true")
+    ap.add_argument("--profile-case", default=None,
+                    help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t> "
+                         "or gemm_<bf16|fp8|fp4>_<fwd|dgrad|wgrad>[_MxNxK]")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.profile_case:
+        return run_profile_case(args.profile_case)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2602_01410_b200 import api, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    cfg = wl.CONFIGS[WORKLOADS[args.workload][0]]
+    formats = (FMT_FP4, FMT_FP8)
+    step = Step(api, torch, cfg, device, formats)
+    peaks = load_peaks()
+
+    # ---- timed region: K steps, inputs resident in HBM ------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step.run_decomposed()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    events = []
+    e0.record()
+    for _ in range(args.steps):
+        step.run_decomposed(events)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    assert api.snip_poll_status(step.gws) == 0, "device-side timeout reported"
+    # GEMM launches inside the timed region, per format: total flops / total event time
+    in_region = {}
+    for fmt, op, fl, a, b in events:
+        d = in_region.setdefault(fmt, {"flops": 0.0, "ms": 0.0, "launches": 0})
+        d["flops"] += fl; d["ms"] += a.elapsed_time(b); d["launches"] += 1
+    ms_per_step = ms_total / args.steps
+    value = step.flops * world / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: inputs start in pinned host memory, statistics come back -------------------
+    e2e = None
+    if rank == 0 or world > 1:
+        host = [tuple(t.cpu().pin_memory() for t in trip) for trip in step.inputs]
+        h2d = sum(t.numel() * 2 for trip in host for t in trip)
+        stats_host = torch.empty_like(step.stats, device="cpu").pin_memory()
+        def e2e_step():
+            for trip_d, trip_h in zip(step.inputs, host):
+                for d, h in zip(trip_d, trip_h):
+                    d.copy_(h, non_blocking=True)
+            step.run_linear_calls()
+            stats_host.copy_(step.stats, non_blocking=True)
+        e2e_step(); barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        s1.record()
+        barrier()
+        ms_e2e = s0.elapsed_time(s1) / n_e2e
+        if world > 1:
+            t = torch.tensor([ms_e2e], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": step.flops * world / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": stats_host.numel()}
+        del host
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- kernel legs: the GEMM and quantizer kernels alone, events around each launch ---------------
+    roofline, kernels = None, {}
+    if not args.no_kernel_legs:
+        del step.inputs, step.out, step.codes, step.scales
+        torch.cuda.empty_cache()
+        kt = KernelTimer(api, torch, cfg, device)
+        qkv = 0
+        fam = {}
+        for f in formats:
+            per_op = {}
+            tot_fl, tot_ms = 0.0, 0.0
+            for op, name in ((api.OP_FWD, "fwd"), (api.OP_DGRAD, "dgrad"), (api.OP_WGRAD, "wgrad")):
+                fl, times = kt.gemm(f, op, qkv)
+                avg = sum(times) / len(times)
+                per_op[name] = {"tflops": fl / (avg * 1e-3) / 1e12, "ms": avg}
+                tot_fl += fl; tot_ms += avg
+            peak = peaks["bf16_tflops"] * NOMINAL_RATIO[f]
+            fam[f] = {"achieved": tot_fl / (tot_ms * 1e-3) / 1e12, "peak": peak, "per_op": per_op, "ms": tot_ms}
+            kernels[f"gemm_{FMT_NAME[f]}"] = {"tflops": fam[f]["achieved"], "frac_of_peak": fam[f]["achieved"] / peak,
+                                              "peak_tflops": peak, "per_op": per_op}
+    dom = max(in_region, key=lambda f: in_region[f]["ms"])
+    d = in_region[dom]
+    dom_peak = peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[dom]
+    roofline = {"kernel": f"gemm_kernel, {FMT_NAME[dom]} operands (all {d['launches']} launches of the timed region)", "bound": "tensor",
+                "achieved": d["flops"] / (d["ms"] * 1e-3) / 1e12, "peak": dom_peak, "unit": "TFLOP/s",
+                "frac": d["flops"] / (d["ms"] * 1e-3) / 1e12 / dom_peak, "traffic": None,
+                "share_of_step": d["ms"] / ms_total,
+                "peak_source": f"{peaks['source']} cuBLAS bf16 sustained x{NOMINAL_RATIO[dom]:.0f} (nominal {FMT_NAME[dom]}/bf16 ratio)"}
+    for f, d in in_region.items():
+        kernels[f"gemm_{FMT_NAME[f]}_in_step"] = {"tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12, "ms_per_step": d["ms"] / args.steps,
+                                                   "frac_of_sustained_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f])}
+    if not args.no_kernel_legs:
+        for f in formats:
+            for block, tr, name in ((api.BLOCK_ROW, False, "row"), (api.BLOCK_COL, True, "col_t"), (api.BLOCK_BLK, True, "blk_t")):
+                by, times = kt.quantizer(f, block, tr, cfg.M, 4096)
+                avg = sum(times) / len(times)
+                kernels[f"quantize_{FMT_NAME[f]}_{name}"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, cores, sample = cpu_baseline_sample(cfg)
+        cpu = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+
+    line = {"metric": "mixed-precision linear fwd+dgrad+wgrad TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp4_e2m1+fp8_e4m3 (fp32 accumulate)", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: one block (qkv,o,gate,up,down) x (fwd,dgrad,wgrad) all-FP4 then all-FP8, tokens {cfg.M}, quantize+stats every GEMM",
+                       "l2": "inputs larger than L2", "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": step.launches_per_step * args.steps,
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
