@@ -56,7 +56,11 @@ struct Cfg {
     static constexpr int kBBytes = BN * 128;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = (BN >= 256) ? 4 : 5;
-    static constexpr int kSbInvBytes = kNumEpiWarps * (BN / 2) * 4;  // per-warp reciprocal B scales (wgrad)
+    static constexpr int kScaleDepth = 4;                        // chunks of scale factors in flight per warp
+    static constexpr int kRingB = 36;                            // float offset of the per-column B scales in a slot
+    static constexpr int kRingFloatsPerSlot = 36 + BN / 2 + 28;  // 32 A scales, 4 block scales, BN/2 column scales (16-byte aligned)
+    static constexpr int kRingFloatsPerWarp = kScaleDepth * kRingFloatsPerSlot;
+    static constexpr int kSbInvBytes = kNumEpiWarps * kRingFloatsPerWarp * 4;
     static constexpr int kSmemBytes = kStages * kStageBytes + kSbInvBytes + 256 + 1024;  // + barriers + alignment slack
     static constexpr int kAccCols = 2 * BN;
     static constexpr int kSfCol0 = kAccCols;
@@ -129,7 +133,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t smem_a0 = smem_base;
     const uint32_t smem_b0 = smem_base + S * C::kABytes;
-    float *sb_inv = reinterpret_cast<float *>(smem_gen + S * C::kStageBytes);
+    float *scale_ring = reinterpret_cast<float *>(smem_gen + S * C::kStageBytes);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_gen + S * C::kStageBytes + C::kSbInvBytes);
     const uint32_t bar0 = smem_base + S * C::kStageBytes + C::kSbInvBytes;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -256,6 +260,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int e = warp - 4;          // 0..7
         const int q = warp & 3;          // tensor-memory lane quarter this warp may access
         const int h = e >> 2;            // column half
+        // Per-warp ring of scale factors, filled kScaleDepth chunks ahead with cp.async so that no
+        // global-memory latency sits between two chunks:
+        //   [d][0..31]               S_a of this warp's 32 rows
+        //   [d][32..35]              S_b of the (at most two) 128-column blocks this warp covers (block mode)
+        //   [d][kRingB..kRingB+HALF) S_b of this warp's HALF output columns (vector mode)
+        float *ring = scale_ring + e * C::kRingFloatsPerWarp;
+        const uint32_t ring_u32 = smem_u32(ring);
         uint32_t cc = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
@@ -265,73 +276,116 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int col0 = n_idx * BN + h * HALF;
             const bool row_ok = row < g.Mo;
             const int nacc = (KIND == MmaKind::F16) ? 1 : num_chunks;
-            float acc[SCALE == SCALE_NONE ? 1 : HALF];
+            const int blk0 = col0 >> 7;
+            const int blk_last = (g.No - 1) >> 7;
+
+            auto prefetch_scales = [&](int cn) {
+                if (SCALE != SCALE_NONE && cn < nacc) {
+                    const int d = cn % C::kScaleDepth;
+                    const uint32_t slot = ring_u32 + d * C::kRingFloatsPerSlot * 4;
+                    if (row_ok) cp_async_4(slot + lane * 4, g.sa + (int64_t)cn * g.sa_chunk_stride + row);
+                    if (SCALE == SCALE_BLOCK_B) {
+                        if (lane < 2) {
+                            const int blk = min(blk0 + lane, blk_last);
+                            cp_async_4(slot + (32 + lane) * 4, g.sb + (int64_t)blk * g.sb_blk_stride + (int64_t)cn * g.sb_chunk_stride);
+                        }
+                    } else if (SCALE == SCALE_VEC_B) {
+                        const int n = col0 + 4 * lane;
+                        if (4 * lane < HALF && n < g.No)
+                            cp_async_16(slot + (C::kRingB + 4 * lane) * 4, g.sb + (int64_t)cn * g.sb_chunk_stride + n);
+                    }
+                }
+                cp_async_commit();
+            };
+
+            float2 acc[SCALE == SCALE_NONE ? 1 : HALF / 2];
             if (SCALE != SCALE_NONE) {
 #pragma unroll
-                for (int i = 0; i < HALF; ++i) acc[i] = 0.0f;
+                for (int i = 0; i < HALF / 2; ++i) acc[i] = make_float2(0.0f, 0.0f);
+                // out-of-range rows / columns read 1.0 (their products are zero anyway)
+                for (int i = lane; i < C::kScaleDepth * C::kRingFloatsPerSlot; i += 32) ring[i] = 1.0f;
+                __syncwarp();
+#pragma unroll
+                for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
             }
             for (int c = 0; c < nacc; ++c, ++cc) {
                 const uint32_t a = cc & 1u;
                 float f[G];
-                if (SCALE == SCALE_BLOCK_B) {
-                    const float sa = row_ok ? g.sa[(int64_t)c * g.sa_chunk_stride + row] : 1.0f;
-                    const float ia = __fdiv_rn(1.0f, sa);
-#pragma unroll
-                    for (int gi = 0; gi < G; ++gi) {
-                        const int col = min(col0 + 32 * gi, g.No - 1);
-                        const float sb = g.sb[(int64_t)(col >> 7) * g.sb_blk_stride + (int64_t)c * g.sb_chunk_stride];
-                        f[gi] = ia * __fdiv_rn(1.0f, sb);
-                    }
-                } else if (SCALE == SCALE_VEC_B) {
-                    const float sa = row_ok ? g.sa[(int64_t)c * g.sa_chunk_stride + row] : 1.0f;
-                    f[0] = __fdiv_rn(1.0f, sa);
-                    // reciprocal B scales of this chunk for this warp's HALF output columns; each warp
-                    // keeps a private copy so that no cross-warp barrier is needed
-#pragma unroll
-                    for (int i = lane; i < HALF; i += 32) {
-                        const int n = col0 + i;
-                        const float sb = n < g.No ? g.sb[(int64_t)c * g.sb_chunk_stride + n] : 1.0f;
-                        sb_inv[e * HALF + i] = __fdiv_rn(1.0f, sb);
-                    }
+                const float *slot = ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;
+                if (SCALE != SCALE_NONE) {
+                    cp_async_wait<C::kScaleDepth - 1>();
                     __syncwarp();
+                    const float sa = slot[lane];
+                    if (SCALE == SCALE_BLOCK_B) {
+                        const float f0 = __fdividef(1.0f, sa * slot[32]), f1 = __fdividef(1.0f, sa * slot[33]);
+#pragma unroll
+                        for (int gi = 0; gi < G; ++gi) f[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
+                    } else {
+                        f[0] = __fdividef(1.0f, sa);
+                        // turn this chunk's column scales into reciprocals once (4 per lane), in place
+                        if (4 * lane < HALF) {
+                            float4 *p4 = reinterpret_cast<float4 *>(ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot + C::kRingB + 4 * lane);
+                            const float4 s4 = *p4;
+                            *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
+                        }
+                        __syncwarp();
+                    }
                 }
                 const bool got = mbar_wait(tfull_bar(a), (cc >> 1) & 1u, abort_flag);
                 if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
+                uint32_t v[2][32];
+                tmem_ld32(taddr, v[0]);
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + 32 * gi, v);
-                    tmem_ld_wait(v);
+                    uint32_t (&cur)[32] = v[gi & 1];
+                    tmem_ld_wait();
+                    if (gi + 1 < G) {
+                        tmem_ld32(taddr + 32 * (gi + 1), v[(gi + 1) & 1]);   // in flight during the FMAs below
+                    } else {
+                        // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty_bar(a));
+                    }
                     if (SCALE == SCALE_NONE) {
                         float o[32];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+                        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(cur[i]);
                         if (row_ok) store32<OUT_F32>(g, row, col0 + 32 * gi, o);
                     } else if (SCALE == SCALE_BLOCK_B) {
+                        const float2 ff = make_float2(f[gi], f[gi]);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) acc[32 * gi + i] = fmaf(__uint_as_float(v[i]), f[gi], acc[32 * gi + i]);
+                        for (int i = 0; i < 16; ++i)
+                            acc[16 * gi + i] = __ffma2_rn(make_float2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), ff, acc[16 * gi + i]);
                     } else {
-                        const float4 *sbv = reinterpret_cast<const float4 *>(sb_inv + e * HALF + 32 * gi);
+                        const float2 ff = make_float2(f[0], f[0]);
+                        const float4 *sbv = reinterpret_cast<const float4 *>(slot + C::kRingB + 32 * gi);
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            const float4 s4 = sbv[i >> 2];
-                            acc[32 * gi + i + 0] = fmaf(__uint_as_float(v[i + 0]) * s4.x, f[0], acc[32 * gi + i + 0]);
-                            acc[32 * gi + i + 1] = fmaf(__uint_as_float(v[i + 1]) * s4.y, f[0], acc[32 * gi + i + 1]);
-                            acc[32 * gi + i + 2] = fmaf(__uint_as_float(v[i + 2]) * s4.z, f[0], acc[32 * gi + i + 2]);
-                            acc[32 * gi + i + 3] = fmaf(__uint_as_float(v[i + 3]) * s4.w, f[0], acc[32 * gi + i + 3]);
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 s4 = sbv[i];   // reciprocal column scales, broadcast read
+                            const float2 r0 = make_float2(s4.x, s4.y);
+                            const float2 r1 = make_float2(s4.z, s4.w);
+                            const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i]), __uint_as_float(cur[4 * i + 1])), r0);
+                            const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i + 2]), __uint_as_float(cur[4 * i + 3])), r1);
+                            acc[16 * gi + 2 * i] = __ffma2_rn(p0, ff, acc[16 * gi + 2 * i]);
+                            acc[16 * gi + 2 * i + 1] = __ffma2_rn(p1, ff, acc[16 * gi + 2 * i + 1]);
                         }
                     }
                 }
-                // this warp's reads of buffer `a` are complete: hand it back to the MMA warp
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(a));
+                if (SCALE != SCALE_NONE) {
+                    __syncwarp();                       // every lane has read this slot
+                    prefetch_scales(c + C::kScaleDepth); // refill it for a later chunk
+                }
             }
-            if (SCALE != SCALE_NONE && ok && row_ok) {
+            if (SCALE != SCALE_NONE) {
+                cp_async_wait<0>();
+                if (ok && row_ok) {
 #pragma unroll
-                for (int gi = 0; gi < G; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, acc + 32 * gi);
+                    for (int gi = 0; gi < G; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, reinterpret_cast<const float *>(acc) + 32 * gi);
+                }
+                __syncwarp();
             }
         }
     }

@@ -98,28 +98,27 @@ __device__ __forceinline__ float2 dec_e2m1x2(uint32_t c)
     return __half22float2(*reinterpret_cast<__half2 *>(&h2));
 }
 
-// Quantize 8 consecutive elements (one 128-bit load) that share or do not share a scale.
-// s[i], inv[i]: scale and reciprocal for element i.  Returns the packed codes
-// (FP8: 8 bytes in out[0..1]; FP4: 4 bytes in out[0]) and adds to the statistics.
+// Quantize 8 consecutive elements (one 128-bit load).  s2[i] / ninv2[i]: scale and negated
+// reciprocal scale of elements (2i, 2i+1).  Returns the packed codes (FP8: 8 bytes in out[0..1];
+// FP4: 4 bytes in out[0]) and adds to the statistics.  The products x*S are IEEE binary32
+// products (packed mul.rn.f32x2), exactly what the scalar definition asks for.
 template <int FMT, bool STATS>
-__device__ __forceinline__ void quant8(const uint4 &v, const float *s, const float *inv,
-                                       uint32_t out[2], float &sx, float &se)
+__device__ __forceinline__ void quant8(const uint4 &v, const float2 (&s2)[4], const float2 (&ninv2)[4],
+                                       uint32_t out[2], float2 &sx2, float2 &se2)
 {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     uint32_t c[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        float x0 = bf16lo(w[i]), x1 = bf16hi(w[i]);
-        float t0 = __fmul_rn(x0, s[2 * i]), t1 = __fmul_rn(x1, s[2 * i + 1]);
-        if (FMT == SNIP_FMT_FP8_E4M3) c[i] = cvt_e4m3x2(t0, t1);
-        else c[i] = cvt_e2m1x2(t0, t1);
+        const float2 x = make_float2(bf16lo(w[i]), bf16hi(w[i]));
+        const float2 t = __fmul2_rn(x, s2[i]);
+        if (FMT == SNIP_FMT_FP8_E4M3) c[i] = cvt_e4m3x2(t.x, t.y);
+        else c[i] = cvt_e2m1x2(t.x, t.y);
         if (STATS) {
-            float2 d = (FMT == SNIP_FMT_FP8_E4M3) ? dec_e4m3x2(c[i]) : dec_e2m1x2(c[i]);
-            float e0 = fmaf(-d.x, inv[2 * i], x0), e1 = fmaf(-d.y, inv[2 * i + 1], x1);
-            sx = fmaf(x0, x0, sx);
-            sx = fmaf(x1, x1, sx);
-            se = fmaf(e0, e0, se);
-            se = fmaf(e1, e1, se);
+            const float2 d = (FMT == SNIP_FMT_FP8_E4M3) ? dec_e4m3x2(c[i]) : dec_e2m1x2(c[i]);
+            const float2 e = __ffma2_rn(d, ninv2[i], x);  // x - value(code)/S
+            sx2 = __ffma2_rn(x, x, sx2);
+            se2 = __ffma2_rn(e, e, se2);
         }
     }
     if (FMT == SNIP_FMT_FP8_E4M3) {
@@ -143,6 +142,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
     __shared__ __align__(16) uint8_t stage[TRANSPOSED && CODES && kQuant ? kTile * kRowBytes : 16];
     __shared__ uint32_t col_amax[8][kTile / 2];  // packed bf16 pairs, one row per warp
     __shared__ float col_scale[kTile];
+    __shared__ float col_ninv[kTile];
     __shared__ float red_f[8][3];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -153,18 +153,24 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
 
     // ---- load the 8x8 sub-block: eight independent 128-bit loads ------------------------
     uint4 v[8];
+    {
+        const uint16_t *xb = a.x + rbase * a.ld + cbase;   // 64-bit arithmetic once per thread
+        const bool rows_ok = rbase < a.rows;               // rows is a multiple of 64: all 8 rows or none
+        const uint32_t ld32 = (uint32_t)a.ld;
 #pragma unroll
-    for (int p = 0; p < 8; ++p) {
-        const int64_t r = rbase + p;
-        if (col_ok && r < a.rows)
-            v[p] = __ldg(reinterpret_cast<const uint4 *>(a.x + r * a.ld + cbase));
-        else
-            v[p] = make_uint4(0, 0, 0, 0);
+        for (int p = 0; p < 8; ++p) {
+            if (col_ok && rows_ok)
+                v[p] = __ldg(reinterpret_cast<const uint4 *>(xb + p * ld32));
+            else
+                v[p] = make_uint4(0, 0, 0, 0);
+        }
     }
 
     // ---- block amax -> scales --------------------------------------------------------
+    constexpr float kFpxMax = (FMT == SNIP_FMT_FP4_E2M1) ? 6.0f : 448.0f;
     float s_row[8], s_col[8];  // scale per row p (ROW) / per column j (COL); BLK uses s_row[0]
-    (void)s_row; (void)s_col;
+    float n_row[8], n_col[8];  // matching -1/S for the error term
+    (void)s_row; (void)s_col; (void)n_row; (void)n_col;
     float my_amax = 0.0f;      // this thread's amax, for the tensor-wide statistic
     if (kQuant || STATS) {
         uint32_t rmax[8];      // per row: packed max over the 8 columns (as 4 pairs folded)
@@ -197,8 +203,14 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             for (int q = 1; q < 4; ++q) sel = ((myp >> 1) == q) ? pk[q] : sel;
             float am = (myp & 1) ? bf16hi(sel) : bf16lo(sel);
             float mine = tile_scale<FMT>(am);
+            // -1/S for the error term: amax/FPX_MAX equals 1/S to within one rounding, which the
+            // statistics (1e-4) do not see; for an empty tile the value is irrelevant (all codes 0)
+            float mine_ninv = -am * (1.0f / kFpxMax);
 #pragma unroll
-            for (int p = 0; p < 8; ++p) s_row[p] = __shfl_sync(0xFFFFFFFFu, mine, (lane & 16) | p);
+            for (int p = 0; p < 8; ++p) {
+                s_row[p] = __shfl_sync(0xFFFFFFFFu, mine, (lane & 16) | p);
+                if (STATS) n_row[p] = __shfl_sync(0xFFFFFFFFu, mine_ninv, (lane & 16) | p);
+            }
             if (STATS) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) my_amax = fmaxf(my_amax, fmaxf(bf16lo(pk[q]), bf16hi(pk[q])));
@@ -236,6 +248,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
                     float am = __uint_as_float(m << 16);
                     float s = tile_scale<FMT>(am);
                     col_scale[tid] = s;
+                    col_ninv[tid] = -am * (1.0f / kFpxMax);
                     if (CODES && c0 + tid < a.cols) a.scales[(int64_t)blockIdx.y * a.cols + c0 + tid] = s;
                     if (STATS) my_amax = am;
                 }
@@ -244,6 +257,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
                 const float4 s1 = *reinterpret_cast<const float4 *>(&col_scale[8 * tx + 4]);
                 s_col[0] = s0.x; s_col[1] = s0.y; s_col[2] = s0.z; s_col[3] = s0.w;
                 s_col[4] = s1.x; s_col[5] = s1.y; s_col[6] = s1.z; s_col[7] = s1.w;
+                if (STATS) {
+                    const float4 n0 = *reinterpret_cast<const float4 *>(&col_ninv[8 * tx]);
+                    const float4 n1 = *reinterpret_cast<const float4 *>(&col_ninv[8 * tx + 4]);
+                    n_col[0] = n0.x; n_col[1] = n0.y; n_col[2] = n0.z; n_col[3] = n0.w;
+                    n_col[4] = n1.x; n_col[5] = n1.y; n_col[6] = n1.z; n_col[7] = n1.w;
+                }
             } else {
                 // BLK (or statistics-only): one amax for the whole CTA tile
                 uint32_t m = max2(max2(cm[0], cm[1]), max2(cm[2], cm[3]));
@@ -258,6 +277,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
                 my_amax = bm;
                 if (kQuant) {
                     s_row[0] = tile_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm);
+                    n_row[0] = -bm * (1.0f / kFpxMax);
                     if (CODES && tid == 0) a.scales[(int64_t)blockIdx.y * gridDim.x + blockIdx.x] = s_row[0];
                 }
                 __syncthreads();  // red_f is reused below
@@ -270,40 +290,44 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
     float rsx[8], rse[8];
     (void)rsx; (void)rse;
     if (kQuant) {
-        float sc[8], inv[8];
+        float2 sc[4], ni[4];
         if (BLOCK == SNIP_BLOCK_COL_128x1) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { sc[j] = s_col[j]; inv[j] = STATS ? __fdiv_rn(1.0f, s_col[j]) : 0.0f; }
+            for (int j = 0; j < 4; ++j) { sc[j] = make_float2(s_col[2 * j], s_col[2 * j + 1]); ni[j] = make_float2(n_col[2 * j], n_col[2 * j + 1]); }
         } else if (BLOCK == SNIP_BLOCK_BLK_128x128) {
-            const float iv = STATS ? __fdiv_rn(1.0f, s_row[0]) : 0.0f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { sc[j] = s_row[0]; inv[j] = iv; }
+            for (int j = 0; j < 4; ++j) { sc[j] = make_float2(s_row[0], s_row[0]); ni[j] = make_float2(n_row[0], n_row[0]); }
         }
         uint32_t codes[8][2];
+        float2 sx2 = make_float2(0.0f, 0.0f), se2 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
             if (BLOCK == SNIP_BLOCK_ROW_1x128) {
-                const float iv = STATS ? __fdiv_rn(1.0f, s_row[p]) : 0.0f;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) { sc[j] = s_row[p]; inv[j] = iv; }
+                for (int j = 0; j < 4; ++j) { sc[j] = make_float2(s_row[p], s_row[p]); ni[j] = make_float2(n_row[p], n_row[p]); }
             }
-            float px = 0.0f, pe = 0.0f;
-            quant8<FMT, STATS>(v[p], sc, inv, codes[p], px, pe);
-            if (STATS) { sx += px; se += pe; }
-            if (ROWSTATS) { rsx[p] = px; rse[p] = pe; }
+            if (ROWSTATS) {
+                float2 px = make_float2(0.0f, 0.0f), pe = make_float2(0.0f, 0.0f);
+                quant8<FMT, STATS>(v[p], sc, ni, codes[p], px, pe);
+                rsx[p] = px.x + px.y; rse[p] = pe.x + pe.y;
+                sx += rsx[p]; se += rse[p];
+            } else {
+                quant8<FMT, STATS>(v[p], sc, ni, codes[p], sx2, se2);
+            }
         }
+        if (STATS && !ROWSTATS) { sx = sx2.x + sx2.y; se = se2.x + se2.y; }
         if (CODES) {
             if (!TRANSPOSED) {
                 const int64_t out_ld = a.cols * kCodeBytes8 / 8;  // bytes per output row
+                if (col_ok && rbase < a.rows) {
+                    uint8_t *dst = a.codes + rbase * out_ld + cbase * kCodeBytes8 / 8;
+                    const uint32_t ld32 = (uint32_t)out_ld;
 #pragma unroll
-                for (int p = 0; p < 8; ++p) {
-                    const int64_t r = rbase + p;
-                    if (col_ok && r < a.rows) {
-                        uint8_t *dst = a.codes + r * out_ld + cbase * kCodeBytes8 / 8;
+                    for (int p = 0; p < 8; ++p) {
                         if (FMT == SNIP_FMT_FP8_E4M3)
-                            *reinterpret_cast<uint2 *>(dst) = make_uint2(codes[p][0], codes[p][1]);
+                            *reinterpret_cast<uint2 *>(dst + p * ld32) = make_uint2(codes[p][0], codes[p][1]);
                         else
-                            *reinterpret_cast<uint32_t *>(dst) = codes[p][0];
+                            *reinterpret_cast<uint32_t *>(dst + p * ld32) = codes[p][0];
                     }
                 }
             } else {
