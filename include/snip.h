@@ -52,8 +52,8 @@ typedef enum { SNIP_FMT_BF16 = 0, SNIP_FMT_FP8_E4M3 = 1, SNIP_FMT_FP4_E2M1 = 2 }
  * COL = along the row index (128 consecutive rows of one column). */
 typedef enum { SNIP_BLOCK_ROW_1x128 = 0, SNIP_BLOCK_COL_128x1 = 1, SNIP_BLOCK_BLK_128x128 = 2 } snip_block_t;
 
-/* Output element type of a GEMM.  BF16 is the paper's choice (Sec. 2.2: "the output of the
- * GEMM operator remains in BF16"); FP32 exposes the accumulator for parity checks and for
+/* Output element type of a GEMM.  BF16 is the paper's choice (Sec. 2.2 keeps GEMM outputs in
+ * BF16 while the operands are FPX); FP32 exposes the accumulator for parity checks and for
  * weight-gradient accumulation. */
 typedef enum { SNIP_OUT_BF16 = 0, SNIP_OUT_FP32 = 1 } snip_out_t;
 
@@ -166,8 +166,8 @@ int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int 
  *           codes transposed [K,M])
  * i.e. both operands always have the contraction index contiguous.  Each 128-long chunk of the
  * contraction is multiplied on the tensor cores (FP32 accumulation), then scaled by
- * 1/(S_a*S_b) of that chunk in FP32 and added to an FP32 accumulator ("the output is scaled
- * back by dividing by the same scaling factor", Sec. 2.3); the result is rounded to nearest-even
+ * 1/(S_a*S_b) of that chunk in FP32 and added to an FP32 accumulator (Sec. 2.3 removes the scale
+ * after the low-precision operator by dividing by it); the result is rounded to nearest-even
  * to bf16 or stored as FP32.  accumulate != 0 adds to the existing contents of out (FP32 output
  * only).  Operand formats: (BF16,BF16), (FP8,FP8), (FP4,FP4), (FP8,FP4), (FP4,FP8); pairs
  * that mix BF16 with a quantized operand return SNIP_ERR_UNSUPPORTED.

@@ -286,8 +286,8 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int blo
     return 0;
 }
 
-/* Dequantize codes + scales back to binary64: xhat = value(code) / S (Sec. 2.3, "scaled back
- * by dividing by the same scaling factor"). */
+/* Dequantize codes + scales to binary64: xhat = value(code) / S (Sec. 2.3: the scale is removed
+ * after the operator by dividing by it). */
 int orc_dequantize(const uint8_t *codes, const float *scales, int64_t rows, int64_t cols,
                    int fmt, int block, double *xhat)
 {

@@ -1,7 +1,7 @@
 // Block-scaled GEMMs on the tcgen05 tensor cores:  out[Mo,No] = A[Mo,Kc] . B[No,Kc]^T with both
 // operands contraction-major, FP32 accumulation in tensor memory, and the paper's FP32 tile
-// scales applied per 128-long chunk of the contraction (Sec. 2.3: "the output is scaled back by
-// dividing by the same scaling factor"; Fig. 5 for the three GEMMs of a linear layer).
+// scales applied per 128-long chunk of the contraction (Sec. 2.3 divides the operator's output by
+// the scale that was multiplied in; Fig. 5 shows the three GEMMs of a linear layer).
 //
 // Structure of one CTA (persistent, one per SM, 384 threads):
 //   warp 0      : TMA producer - streams 128-byte-wide operand tiles into a shared-memory ring
