@@ -20,7 +20,7 @@ Q_TRANSPOSED, Q_STATS, Q_NO_CODES = 1, 2, 4
 OK = 0
 ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(1, 8)
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsnip_b200.so")
+LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsnip_b200.so")
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",

@@ -1,7 +1,7 @@
 // Block-scaled GEMMs on the tcgen05 tensor cores:  out[Mo,No] = A[Mo,Kc] . B[No,Kc]^T with both
 // operands contraction-major, FP32 accumulation in tensor memory, and the paper's FP32 tile
-// scales applied per 128-long chunk of the contraction (Sec. 2.3 divides the operator's output by
-// the scale that was multiplied in; Fig. 5 shows the three GEMMs of a linear layer).
+// scales applied per 128-long chunk of the contraction (Sec. 2.3: "the output is scaled back by
+// dividing by the same scaling factor"; Fig. 5 for the three GEMMs of a linear layer).
 //
 // Structure of one CTA (persistent, one per SM, 384 threads):
 //   warp 0      : TMA producer - streams 128-byte-wide operand tiles into a shared-memory ring
@@ -15,8 +15,6 @@
 // leaves cleanly (tensor memory is always released).
 #include <cuda.h>
 #include <cuda_bf16.h>
-#include <stdlib.h>
-#include <string.h>
 
 #include "common.cuh"
 #include "sm100.cuh"
@@ -45,35 +43,35 @@ struct GemmArgs {
     int64_t ldo;
     int32_t accumulate;
     uint32_t stage_tx_bytes;   // bytes the two TMA loads of one stage report to the barrier
-    long long *trace;          // optional (SNIP_GEMM_TRACE=1): per-chunk clock64 stamps of CTA 0, else null
     uint32_t *status;
 };
 
-template <MmaKind KIND, int BN, bool PAIR>
+template <MmaKind KIND, int BN, int SCALE>
 struct Cfg {
     static constexpr int kStageElemsX = (KIND == MmaKind::F16) ? 64 : 128;   // TMA x step per stage
     static constexpr int kChunkElems = 128;                                  // scale granularity
     static constexpr int kStageK = (KIND == MmaKind::F16) ? 64 : (KIND == MmaKind::F8F6F4 ? 128 : 256);
     static constexpr int kABytes = BM * 128;
-    static constexpr int kBRows = PAIR ? BN / 2 : BN;          // B rows held by one CTA (a pair splits B along N)
-    static constexpr int kBBytes = kBRows * 128;
+    static constexpr int kBBytes = BN * 128;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kStages = PAIR ? (BN >= 256 ? 5 : 6) : ((BN >= 256) ? 4 : 5);
+    static constexpr int kStages = (BN >= 256) ? 4 : 5;
     static constexpr int kScaleDepth = 4;                        // chunks of scale factors in flight per warp
     static constexpr int kRingB = 36;                            // float offset of the per-column B scales in a slot
-    static constexpr int kRingFloatsPerSlot = 36 + BN / 2 + 28;  // 32 A scales, 4 block scales, BN/2 column scales (16-byte aligned)
+    // a slot holds 32 A scales, 4 block scales and, in vector mode, BN/2 column scales
+    static constexpr int kRingFloatsPerSlot = (SCALE == 2) ? 36 + BN / 2 + 28 : 64;
     static constexpr int kRingFloatsPerWarp = kScaleDepth * kRingFloatsPerSlot;
     static constexpr int kSbInvBytes = kNumEpiWarps * kRingFloatsPerWarp * 4;
-    static constexpr int kOutStageBytes = PAIR ? kNumEpiWarps * 4096 : 0;   // per-warp staging tiles of the output TMA store
-    static constexpr int kSmemBytes = kStages * kStageBytes + kSbInvBytes + 256 + kOutStageBytes + 1024;  // + barriers + alignment slack
+    // block mode (fwd / dgrad) writes its output through per-warp 2 KB staging tiles and TMA stores
+    static constexpr bool kTmaOut = (SCALE == 1);
+    static constexpr int kOutStageBytes = kTmaOut ? kNumEpiWarps * 2048 : 0;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kSbInvBytes + kOutStageBytes + 256 + 1024;  // + barriers + alignment slack
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+    static_assert(kStageBytes % 1024 == 0 && kSbInvBytes % 1024 == 0, "staging tiles must stay 1024-byte aligned");
     static constexpr int kAccCols = 2 * BN;
     static constexpr int kSfCol0 = kAccCols;
     static constexpr int kTmemCols = 512;
     static_assert(kAccCols + (KIND == MmaKind::MXF4 ? kSfCols : 0) <= 512, "tensor memory budget");
 };
-
-// Row length in bytes of the boxes the epilogue stores through the TMA unit.
-__host__ __device__ constexpr int out_box_bytes(bool out_f32, int bn) { return (out_f32 || (bn / 2) % 64 == 0) ? 128 : 64; }
 
 __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int &m_idx, int &n_idx)
 {
@@ -124,17 +122,12 @@ __device__ __forceinline__ void store32(const GemmArgs &g, int64_t row, int col,
     }
 }
 
-// PAIR = true: two CTAs of a cluster work on one 256-row tile.  Each loads its own 128 rows of A and
-// half of the B rows; the leader (cluster rank 0) issues cta_group::2 MMAs that read both CTAs'
-// shared memory and write each CTA's tensor memory; all pipeline barriers the MMA thread waits on
-// live in the leader, the peer signals them through the cluster's shared-memory window.
-template <MmaKind KIND, int BN, int SCALE, bool OUT_F32, bool PAIR>
+template <MmaKind KIND, int BN, int SCALE, bool OUT_F32>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmO,
             const GemmArgs g, const uint32_t idesc)
 {
-    constexpr bool TMA_OUT = PAIR && SCALE != SCALE_NONE;   // output through shared memory + TMA store
-    using C = Cfg<KIND, BN, PAIR>;
+    using C = Cfg<KIND, BN, SCALE>;
     constexpr int S = C::kStages;
     constexpr int G = BN / 64;       // 32-column groups handled by one epilogue warp
     constexpr int HALF = BN / 2;     // columns handled by one epilogue warp
@@ -149,44 +142,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t out_stage0 = smem_base + S * C::kStageBytes + C::kSbInvBytes;   // 1024-byte aligned
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_gen + S * C::kStageBytes + C::kSbInvBytes + C::kOutStageBytes);
     const uint32_t bar0 = smem_base + S * C::kStageBytes + C::kSbInvBytes + C::kOutStageBytes;
-    static_assert((C::kStageBytes % 1024) == 0 && (C::kSbInvBytes % 1024) == 0, "staging tiles must stay 1024-byte aligned");
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * S + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * S + 2 + a); };
-    // completion of the MMAs issued so far, signalled to this CTA's barrier and, in a pair, to the peer's
-    auto commit_both = [&](uint32_t bar) {
-        tc_commit<PAIR>(bar);
-        if (PAIR) tc_commit<PAIR>(mapa(bar, 1));
-    };
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 4);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int TM = PAIR ? 2 * BM : BM;                     // rows of one scheduled tile
-    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;       // 0 = leader
-    const int num_m = (g.Mo + TM - 1) / TM, num_n = (g.No + BN - 1) / BN;
+    const int num_m = (g.Mo + BM - 1) / BM, num_n = (g.No + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
-    const int first_tile = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int tile_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int num_chunks = (g.Kc + C::kChunkElems - 1) / C::kChunkElems;
     const int num_kstages = (g.Kc + C::kStageK - 1) / C::kStageK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kNumEpiWarps * (PAIR ? 2 : 1)); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kNumEpiWarps); }
         *abort_flag = 0u;
         fence_barrier_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
     }
     if (warp == 1) {
-        tmem_alloc<PAIR>(smem_u32(tmem_slot), C::kTmemCols);
-        tmem_relinquish<PAIR>();
+        tmem_alloc<false>(smem_u32(tmem_slot), C::kTmemCols);
+        tmem_relinquish<false>();
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (PAIR) cluster_sync();   // both CTAs' barriers exist before anyone signals across the pair
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -209,111 +191,72 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
                 int m_idx, n_idx;
                 tile_coords(t, num_m, num_n, m_idx, n_idx);
                 for (int ks = 0; ks < num_kstages; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
-                    const long long t_p0 = clock64();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    if (g.trace && blockIdx.x == 0 && it < 64) { g.trace[1024 + 4 * it] = t_p0; g.trace[1024 + 4 * it + 1] = clock64(); }
-                    if (PAIR) {
-                        // the leader expects the bytes of both CTAs; both report to the leader's barrier
-                        const uint32_t lead_full = mapa(full_bar(s), 0);
-                        if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * g.stage_tx_bytes);
-                        tma_load_2d_pair(smem_a0 + s * C::kABytes, &tmA, lead_full, ks * C::kStageElemsX, m_idx * TM + (int)rank * BM);
-                        tma_load_2d_pair(smem_b0 + s * C::kBBytes, &tmB, lead_full, ks * C::kStageElemsX, n_idx * BN + (int)rank * C::kBRows);
-                    } else {
-                        mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
-                        tma_load_2d(smem_a0 + s * C::kABytes, &tmA, full_bar(s), ks * C::kStageElemsX, m_idx * BM);
-                        tma_load_2d(smem_b0 + s * C::kBBytes, &tmB, full_bar(s), ks * C::kStageElemsX, n_idx * BN);
-                    }
-                    if (g.trace && blockIdx.x == 0 && it < 64) g.trace[1024 + 4 * it + 2] = clock64();
+                    mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
+                    tma_load_2d(smem_a0 + s * C::kABytes, &tmA, full_bar(s), ks * C::kStageElemsX, m_idx * BM);
+                    tma_load_2d(smem_b0 + s * C::kBBytes, &tmB, full_bar(s), ks * C::kStageElemsX, n_idx * BN);
                 }
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer (the pair's leader only) =================
-        // The barrier waits for what is issued next are placed between two halves of the current
-        // stage's MMAs, so that they overlap tensor-core work already queued instead of draining it.
-        if (lane == 0 && rank == 0) {
-            uint32_t cc = 0;
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            uint32_t it = 0, cc = 0;
             bool ok = true;
             const uint32_t sfa = tmem_base + C::kSfCol0, sfb = tmem_base + C::kSfCol0 + 16;
-            const uint32_t my_tiles = first_tile < num_tiles ? (uint32_t)((num_tiles - first_tile + tile_step - 1) / tile_step) : 0u;
-            const uint32_t total_it = my_tiles * (uint32_t)num_kstages;
-            auto wait_full = [&](uint32_t i) {
-                const bool r = mbar_wait(full_bar(i % S), (i / S) & 1u, abort_flag);
-                tc_fence_after_sync();
-                return r;
-            };
-            auto wait_tempty = [&](uint32_t c_) {
-                const bool r = mbar_wait(tempty_bar(c_ & 1u), ((c_ >> 1) & 1u) ^ 1u, abort_flag);
-                tc_fence_after_sync();
-                return r;
-            };
-            if (total_it > 0) ok = wait_full(0) && wait_tempty(0);
-            int ks = 0;
-            for (uint32_t it = 0; it < total_it && ok; ++it) {
-                const int s = it % S;
-                const bool more = it + 1 < total_it;
-                const uint64_t adesc = make_smem_desc_k128(smem_a0 + s * C::kABytes);
-                const uint64_t bdesc = make_smem_desc_k128(smem_b0 + s * C::kBBytes);
-                if (KIND == MmaKind::F16) {
-                    const uint32_t a = cc & 1u;
-                    const bool last = ks == num_kstages - 1;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                for (int ks = 0; ks < num_kstages && ok; ++ks, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (it / S) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint64_t adesc = make_smem_desc_k128(smem_a0 + s * C::kABytes);
+                    const uint64_t bdesc = make_smem_desc_k128(smem_b0 + s * C::kBBytes);
+                    if (KIND == MmaKind::F16) {
+                        const uint32_t a = cc & 1u;
+                        if (ks == 0) {
+                            if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                            tc_fence_after_sync();
+                        }
 #pragma unroll
-                    for (int k = 0; k < 2; ++k)
-                        mma_ss<KIND, PAIR>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u, 0, 0);
-                    if (more) { ok = wait_full(it + 1); if (ok && last) ok = wait_tempty(cc + 1); }
-                    if (!ok) break;
+                        for (int k = 0; k < 4; ++k)
+                            mma_ss<KIND, false>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u, 0, 0);
+                        tc_commit<false>(empty_bar(s));
+                        if (ks == num_kstages - 1) { tc_commit<false>(tfull_bar(a)); ++cc; }
+                    } else if (KIND == MmaKind::F8F6F4) {
+                        const uint32_t a = cc & 1u;
+                        if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
 #pragma unroll
-                    for (int k = 2; k < 4; ++k)
-                        mma_ss<KIND, PAIR>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, 1u, 0, 0);
-                    commit_both(empty_bar(s));
-                    if (last) { commit_both(tfull_bar(a)); ++cc; }
-                } else if (KIND == MmaKind::F8F6F4) {
-                    const uint32_t a = cc & 1u;
-                    const long long t0 = clock64();
-#pragma unroll
-                    for (int k = 0; k < 2; ++k)
-                        mma_ss<KIND, PAIR>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, k > 0 ? 1u : 0u, 0, 0);
-                    const long long t1 = clock64();
-                    if (more) ok = wait_full(it + 1) && wait_tempty(cc + 1);
-                    if (!ok) break;
-                    const long long t2 = clock64();
-#pragma unroll
-                    for (int k = 2; k < 4; ++k)
-                        mma_ss<KIND, PAIR>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, 1u, 0, 0);
-                    commit_both(empty_bar(s));
-                    commit_both(tfull_bar(a));
-                    if (g.trace && blockIdx.x == 0 && cc < 64) {
-                        g.trace[4 * cc + 0] = t0; g.trace[4 * cc + 1] = t1; g.trace[4 * cc + 2] = t2; g.trace[4 * cc + 3] = clock64();
-                    }
-                    ++cc;
-                } else {
-                    // two 128-long chunks per stage, each into its own tensor-memory buffer
-                    uint32_t a = cc & 1u;
-#pragma unroll
-                    for (int k = 0; k < 2; ++k)
-                        mma_ss<KIND, PAIR>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, k > 0 ? 1u : 0u, sfa, sfb);
-                    commit_both(tfull_bar(a));
-                    ++cc;
-                    if (2 * ks + 1 < num_chunks) {
-                        ok = wait_tempty(cc);
-                        if (!ok) break;
-                        a = cc & 1u;
-#pragma unroll
-                        for (int k = 2; k < 4; ++k)
-                            mma_ss<KIND, PAIR>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, k > 2 ? 1u : 0u, sfa, sfb);
-                        commit_both(tfull_bar(a));
+                        for (int k = 0; k < 4; ++k)
+                            mma_ss<KIND, false>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, k > 0 ? 1u : 0u, 0, 0);
+                        tc_commit<false>(empty_bar(s));
+                        tc_commit<false>(tfull_bar(a));
                         ++cc;
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (2 * ks + h < num_chunks) {
+                                const uint32_t a = cc & 1u;
+                                if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                                tc_fence_after_sync();
+#pragma unroll
+                                for (int k = 0; k < 2; ++k)
+                                    mma_ss<KIND, false>(tmem_base + a * BN, adesc + 2 * (2 * h + k), bdesc + 2 * (2 * h + k), idesc,
+                                                 k > 0 ? 1u : 0u, sfa, sfb);
+                                tc_commit<false>(tfull_bar(a));
+                                ++cc;
+                            }
+                        }
+                        tc_commit<false>(empty_bar(s));
                     }
-                    commit_both(empty_bar(s));
-                    if (more) ok = wait_full(it + 1) && wait_tempty(cc);
                 }
-                if (++ks == num_kstages) ks = 0;
             }
         }
       }
@@ -330,15 +273,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         //   [d][kRingB..kRingB+HALF) S_b of this warp's HALF output columns (vector mode)
         float *ring = scale_ring + e * C::kRingFloatsPerWarp;
         const uint32_t ring_u32 = smem_u32(ring);
-        // 4 KB staging tile of this warp for the TMA store of the output (32 rows x 128 bytes, swizzled)
-        const uint32_t stage_u32 = out_stage0 + e * 4096;
+        const uint32_t stage_u32 = out_stage0 + e * 2048;   // this warp's staging tile: 32 rows x 64 bytes
         uint32_t cc = 0;
         bool ok = true;
-        bool ready = false;   // the next chunk's partial sums were already seen complete
-        for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
+        bool ready = false;   // the next chunk's partial sums were already seen complete by an early test
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
             int m_idx, n_idx;
             tile_coords(t, num_m, num_n, m_idx, n_idx);
-            const int row0 = m_idx * TM + (int)rank * BM + q * 32;
+            const int row0 = m_idx * BM + q * 32;
             const int row = row0 + lane;
             const int col0 = n_idx * BN + h * HALF;
             const bool row_ok = row < g.Mo;
@@ -364,181 +306,117 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 cp_async_commit();
             };
-            // Factors of chunk cn from the ring (its copy group must have completed): f[gi] multiplies
-            // the 32-column group gi.  Vector mode: f[0] = 1/S_a, and the column scales of the slot are
-            // turned into reciprocals in place (4 per lane).
-            auto load_factors = [&](int cn, float (&f)[G]) {
-                float *slot = ring + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot;
-                const float sa = slot[lane];
-                if (SCALE == SCALE_BLOCK_B) {
-                    const float f0 = __fdividef(1.0f, sa * slot[32]), f1 = __fdividef(1.0f, sa * slot[33]);
-#pragma unroll
-                    for (int gi = 0; gi < G; ++gi) f[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
-                } else {
-                    f[0] = __fdividef(1.0f, sa);
-                    if (4 * lane < HALF) {
-                        float4 *p4 = reinterpret_cast<float4 *>(slot + C::kRingB + 4 * lane);
-                        const float4 s4 = *p4;
-                        *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
-                    }
-                }
-            };
 
             float2 acc[SCALE == SCALE_NONE ? 1 : HALF / 2];
-            float f_cur[G], f_next[G];
-            // Block mode keeps the scale factors of the next three chunks in registers (plain global loads
-            // issued three chunks ahead): no shared-memory access sits on the per-chunk path, where it
-            // would queue behind the tensor core's operand reads.
-            const float *sa_ptr = g.sa + (row_ok ? row : 0);
-            const float *sb_ptr0 = g.sb + (int64_t)blk0 * g.sb_blk_stride;
-            const float *sb_ptr1 = g.sb + (int64_t)min(blk0 + 1, blk_last) * g.sb_blk_stride;
-            float pa[3], pb0[3], pb1[3];
-            auto fetch_block = [&](int cn, float &a_, float &b0_, float &b1_) {
-                a_ = 1.0f; b0_ = 1.0f; b1_ = 1.0f;
-                if (cn < nacc) {
-                    a_ = __ldg(sa_ptr + (int64_t)cn * g.sa_chunk_stride);
-                    b0_ = __ldg(sb_ptr0 + (int64_t)cn * g.sb_chunk_stride);
-                    b1_ = (BN % 128 == 0) ? b0_ : __ldg(sb_ptr1 + (int64_t)cn * g.sb_chunk_stride);
-                }
-            };
-            auto block_factors = [&](float a_, float b0_, float b1_, float (&f)[G]) {
-                const float f0 = __fdividef(1.0f, a_ * b0_), f1 = __fdividef(1.0f, a_ * b1_);
-#pragma unroll
-                for (int gi = 0; gi < G; ++gi) f[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
-            };
             if (SCALE != SCALE_NONE) {
 #pragma unroll
                 for (int i = 0; i < HALF / 2; ++i) acc[i] = make_float2(0.0f, 0.0f);
-            }
-            if (SCALE == SCALE_BLOCK_B) {
-                float a0, b00, b10;
-                fetch_block(0, a0, b00, b10);
-#pragma unroll
-                for (int d = 0; d < 3; ++d) fetch_block(d + 1, pa[d], pb0[d], pb1[d]);
-                block_factors(a0, b00, b10, f_cur);
-            } else if (SCALE == SCALE_VEC_B) {
                 // out-of-range rows / columns read 1.0 (their products are zero anyway)
                 for (int i = lane; i < C::kScaleDepth * C::kRingFloatsPerSlot; i += 32) ring[i] = 1.0f;
                 __syncwarp();
 #pragma unroll
                 for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
-                cp_async_wait<C::kScaleDepth - 1>();
-                __syncwarp();
-                load_factors(0, f_cur);
-                __syncwarp();
             }
             for (int c = 0; c < nacc; ++c, ++cc) {
                 const uint32_t a = cc & 1u;
-                const long long t_wait = clock64();
-                if (!ready) {   // not seen complete by the early test of the previous iteration
+                float f[G];
+                const float *slot = ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;
+                if (SCALE != SCALE_NONE) {
+                    cp_async_wait<C::kScaleDepth - 1>();
+                    __syncwarp();
+                    const float sa = slot[lane];
+                    if (SCALE == SCALE_BLOCK_B) {
+                        const float f0 = __fdividef(1.0f, sa * slot[32]), f1 = __fdividef(1.0f, sa * slot[33]);
+#pragma unroll
+                        for (int gi = 0; gi < G; ++gi) f[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
+                    } else {
+                        f[0] = __fdividef(1.0f, sa);
+                        // turn this chunk's column scales into reciprocals once (4 per lane), in place
+                        if (4 * lane < HALF) {
+                            float4 *p4 = reinterpret_cast<float4 *>(ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot + C::kRingB + 4 * lane);
+                            const float4 s4 = *p4;
+                            *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
+                        }
+                        __syncwarp();
+                    }
+                }
+                if (!ready) {
                     const bool got = mbar_wait(tfull_bar(a), (cc >> 1) & 1u, abort_flag);
                     if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
                 }
                 tc_fence_after_sync();
                 uint32_t early = 0;
-                const bool tracing = g.trace && blockIdx.x == 0 && e == 0 && lane == 0 && cc < 64;
-                if (tracing) { g.trace[512 + 8 * cc + 0] = t_wait; g.trace[512 + 8 * cc + 1] = clock64(); }
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
                 uint32_t v[2][32];
                 tmem_ld32(taddr, v[0]);
-                if (G > 1) tmem_ld32(taddr + 32, v[1]);
-                if (tracing) g.trace[512 + 8 * cc + 2] = clock64();
-                // while the first two loads are in flight: factors of the next chunk, and (block mode)
-                // the refill of the slot this chunk's factors came from
-                if (SCALE == SCALE_BLOCK_B) {
-                    block_factors(pa[0], pb0[0], pb1[0], f_next);          // chunk c+1, fetched three chunks ago
-                    pa[0] = pa[1]; pb0[0] = pb0[1]; pb1[0] = pb1[1];
-                    pa[1] = pa[2]; pb0[1] = pb0[2]; pb1[1] = pb1[2];
-                    fetch_block(c + 4, pa[2], pb0[2], pb1[2]);
-                    if (tracing) g.trace[512 + 8 * cc + 5] = clock64();
-                } else if (SCALE == SCALE_VEC_B) {
-                    if (c + 1 < nacc) {
-                        cp_async_wait<C::kScaleDepth - 2>();
-                        __syncwarp();
-                        load_factors(c + 1, f_next);
-                        __syncwarp();
-                    }
-                }
-                const float *slot = ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;
 #pragma unroll
-                for (int gp = 0; gp < G; gp += 2) {
+                for (int gi = 0; gi < G; ++gi) {
+                    uint32_t (&cur)[32] = v[gi & 1];
                     tmem_ld_wait();
-                    if (gp + 2 >= G) {
+                    if (gi + 1 < G) {
+                        tmem_ld32(taddr + 32 * (gi + 1), v[(gi + 1) & 1]);   // in flight during the FMAs below
+                    } else {
                         // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) {
-                            if (PAIR) mbar_arrive_cluster(mapa(tempty_bar(a), 0)); else mbar_arrive(tempty_bar(a));
-                            // non-blocking look at the next chunk's barrier; its latency hides behind the FMAs below
+                            mbar_arrive(tempty_bar(a));
+                            // non-blocking look at the next chunk's barrier: its shared-memory latency hides
+                            // behind the FMAs below instead of opening the next iteration
                             early = mbar_test_wait(tfull_bar(a ^ 1u), ((cc + 1) >> 1) & 1u) ? 1u : 0u;
                         }
-                        if (tracing) g.trace[512 + 8 * cc + 6] = clock64();
                     }
+                    if (SCALE == SCALE_NONE) {
+                        float o[32];
 #pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int gi = gp + u;
-                        if (gi >= G) break;
-                        uint32_t (&cur)[32] = v[u];
-                        if (SCALE == SCALE_NONE) {
-                            float o[32];
+                        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(cur[i]);
+                        if (row_ok) store32<OUT_F32>(g, row, col0 + 32 * gi, o);
+                    } else if (SCALE == SCALE_BLOCK_B) {
+                        const float2 ff = make_float2(f[gi], f[gi]);
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(cur[i]);
-                            if (row_ok) store32<OUT_F32>(g, row, col0 + 32 * gi, o);
-                        } else if (SCALE == SCALE_BLOCK_B) {
-                            const float2 ff = make_float2(f_cur[gi], f_cur[gi]);
+                        for (int i = 0; i < 16; ++i)
+                            acc[16 * gi + i] = __ffma2_rn(make_float2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), ff, acc[16 * gi + i]);
+                    } else {
+                        const float2 ff = make_float2(f[0], f[0]);
+                        const float4 *sbv = reinterpret_cast<const float4 *>(slot + C::kRingB + 32 * gi);
 #pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                acc[16 * gi + i] = __ffma2_rn(make_float2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), ff, acc[16 * gi + i]);
-                        } else {
-                            const float2 ff = make_float2(f_cur[0], f_cur[0]);
-                            const float4 *sbv = reinterpret_cast<const float4 *>(slot + C::kRingB + 32 * gi);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                const float4 s4 = sbv[i];   // reciprocal column scales, broadcast read
-                                const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i]), __uint_as_float(cur[4 * i + 1])), make_float2(s4.x, s4.y));
-                                const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i + 2]), __uint_as_float(cur[4 * i + 3])), make_float2(s4.z, s4.w));
-                                acc[16 * gi + 2 * i] = __ffma2_rn(p0, ff, acc[16 * gi + 2 * i]);
-                                acc[16 * gi + 2 * i + 1] = __ffma2_rn(p1, ff, acc[16 * gi + 2 * i + 1]);
-                            }
+                        for (int i = 0; i < 8; ++i) {
+                            const float4 s4 = sbv[i];   // reciprocal column scales, broadcast read
+                            const float2 r0 = make_float2(s4.x, s4.y);
+                            const float2 r1 = make_float2(s4.z, s4.w);
+                            const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i]), __uint_as_float(cur[4 * i + 1])), r0);
+                            const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i + 2]), __uint_as_float(cur[4 * i + 3])), r1);
+                            acc[16 * gi + 2 * i] = __ffma2_rn(p0, ff, acc[16 * gi + 2 * i]);
+                            acc[16 * gi + 2 * i + 1] = __ffma2_rn(p1, ff, acc[16 * gi + 2 * i + 1]);
                         }
-                        if (gi + 2 < G) tmem_ld32(taddr + 32 * (gi + 2), v[u]);   // refill this register set
                     }
                 }
                 ready = __shfl_sync(0xFFFFFFFFu, early, 0) != 0;
-                if (tracing) g.trace[512 + 8 * cc + 7] = clock64();
                 if (SCALE != SCALE_NONE) {
-                    if (SCALE == SCALE_VEC_B) {
-                        __syncwarp();                        // every lane has finished reading slot c
-                        prefetch_scales(c + C::kScaleDepth);
-                    }
-#pragma unroll
-                    for (int gi = 0; gi < G; ++gi) f_cur[gi] = f_next[gi];
+                    __syncwarp();                       // every lane has read this slot
+                    prefetch_scales(c + C::kScaleDepth); // refill it for a later chunk
                 }
             }
             if (SCALE != SCALE_NONE) {
-                if (SCALE == SCALE_VEC_B) cp_async_wait<0>();
+                cp_async_wait<0>();
                 if (ok) {
-                    if (TMA_OUT && !g.accumulate) {
-                        // round, stage 32 rows x 128 bytes in shared memory (16-byte chunks XOR-swizzled with the
-                        // row, the layout the output tensor map expects), and let the TMA unit write the box
-                        // box rows are 128 bytes (128-byte swizzle) or, for bf16 with 96 columns per warp,
-                        // 64 bytes (64-byte swizzle)
-                        constexpr int kBoxBytes = out_box_bytes(OUT_F32, BN);
-                        constexpr int kPerBox = kBoxBytes / (OUT_F32 ? 4 : 2);
-                        static_assert(HALF % kPerBox == 0, "output boxes must tile the warp's columns");
+                    if (C::kTmaOut && !g.accumulate) {
+                        // round, stage 32 rows x 64 bytes in shared memory (16-byte chunks XOR-swizzled the way
+                        // the output tensor map's 64-byte swizzle expects) and let the TMA unit write each box;
+                        // rows and columns outside the matrix are clipped by the hardware
+                        constexpr int kPerBox = OUT_F32 ? 16 : 32;   // output columns per 64-byte box row
 #pragma unroll
                         for (int b = 0; b < HALF / kPerBox; ++b) {
                             if (lane == 0) bulk_wait_read0();     // the previous box has left the staging tile
                             __syncwarp();
                             const float *src = reinterpret_cast<const float *>(acc) + b * kPerBox;
 #pragma unroll
-                            for (int j = 0; j < kBoxBytes / 16; ++j) {
+                            for (int j = 0; j < 4; ++j) {
                                 uint4 o;
                                 if (OUT_F32) o = make_uint4(__float_as_uint(src[4 * j]), __float_as_uint(src[4 * j + 1]), __float_as_uint(src[4 * j + 2]), __float_as_uint(src[4 * j + 3]));
                                 else o = make_uint4(pack_bf16x2(src[8 * j], src[8 * j + 1]), pack_bf16x2(src[8 * j + 2], src[8 * j + 3]),
                                                     pack_bf16x2(src[8 * j + 4], src[8 * j + 5]), pack_bf16x2(src[8 * j + 6], src[8 * j + 7]));
-                                const int phys = (kBoxBytes == 128) ? (j ^ (lane & 7)) : (j ^ ((lane >> 1) & 3));
-                                st_shared_v4(stage_u32 + lane * kBoxBytes + (phys << 4), o);
+                                st_shared_v4(stage_u32 + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4), o);
                             }
                             fence_proxy_async();
                             __syncwarp();
@@ -567,10 +445,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (threadIdx.x == 0) atomicExch(g.status, (uint32_t)SNIP_ERR_TIMEOUT);
         __syncthreads();
     }
-    if (PAIR) cluster_sync();   // the peer may still be signalling barriers in this CTA's shared memory
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc<PAIR>(tmem_base, C::kTmemCols);
+        tmem_dealloc<false>(tmem_base, C::kTmemCols);
     }
 }
 
@@ -645,69 +522,32 @@ int sm_count()
     return n;
 }
 
-template <MmaKind KIND, int BN, int SCALE, bool OUT_F32, bool PAIR>
+template <MmaKind KIND, int BN, int SCALE, bool OUT_F32>
 int launch_gemm(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmO, const GemmArgs &g, uint32_t idesc, cudaStream_t st)
 {
-    using C = Cfg<KIND, BN, PAIR>;
-    auto kern = gemm_kernel<KIND, BN, SCALE, OUT_F32, PAIR>;
+    using C = Cfg<KIND, BN, SCALE>;
+    auto kern = gemm_kernel<KIND, BN, SCALE, OUT_F32>;
     static thread_local bool attr_set = false;
     if (!attr_set) {
         SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
         attr_set = true;
     }
-    const int tm = PAIR ? 2 * BM : BM;
-    const int num_tiles = (int)(ceil_div(g.Mo, tm) * ceil_div(g.No, BN));
-    cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(kGemmThreads);
-    cfg.dynamicSmemBytes = C::kSmemBytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    // The kernel is persistent: the grid must not exceed what can be resident at once, or the
-    // surplus CTAs (pairs) would only start after the first ones finish.
-    static thread_local int slots = 0;
-    if (slots == 0) {
-        slots = sm_count();
-        if (PAIR) {
-            cfg.gridDim = dim3((unsigned)sm_count() / 2 * 2);
-            int nclusters = 0;
-            SNIP_CUDA_TRY(cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg));
-            slots = nclusters > 0 ? nclusters : 1;
-            if (getenv("SNIP_DEBUG")) fprintf(stderr, "snip: %d resident CTA pairs\n", slots);
-        }
-    }
-    const int ctas = (num_tiles < slots ? num_tiles : slots) * (PAIR ? 2 : 1);
-    cfg.gridDim = dim3((unsigned)ctas);
-    SNIP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmO, g, idesc));
+    const int num_tiles = (int)(ceil_div(g.Mo, BM) * ceil_div(g.No, BN));
+    const int grid = num_tiles < sm_count() ? num_tiles : sm_count();
+    kern<<<grid, kGemmThreads, C::kSmemBytes, st>>>(tmA, tmB, tmO, g, idesc);
+    SNIP_CUDA_TRY(cudaGetLastError());
     return SNIP_OK;
 }
 
-template <MmaKind KIND, int BN, bool PAIR>
+template <MmaKind KIND, int BN>
 int launch_gemm_scale(int scale, bool out_f32, const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmO, const GemmArgs &g,
                       uint32_t idesc, cudaStream_t st)
 {
     if (scale == SCALE_BLOCK_B)
-        return out_f32 ? launch_gemm<KIND, BN, SCALE_BLOCK_B, true, PAIR>(tmA, tmB, tmO, g, idesc, st)
-                       : launch_gemm<KIND, BN, SCALE_BLOCK_B, false, PAIR>(tmA, tmB, tmO, g, idesc, st);
-    return out_f32 ? launch_gemm<KIND, BN, SCALE_VEC_B, true, PAIR>(tmA, tmB, tmO, g, idesc, st)
-                   : launch_gemm<KIND, BN, SCALE_VEC_B, false, PAIR>(tmA, tmB, tmO, g, idesc, st);
-}
-
-// Pairs of CTAs (cta_group::2) halve the B-operand traffic per CTA.  SNIP_GEMM_PAIR=0 selects the
-// single-CTA kernels (kept for comparison and for outputs shorter than 256 rows).
-bool use_pair(int64_t Mo)
-{
-    static int env = -1;
-    if (env < 0) {
-        const char *e = getenv("SNIP_GEMM_PAIR");
-        env = (e && e[0] == '0') ? 0 : 1;
-    }
-    return env == 1 && Mo >= 2 * BM;
+        return out_f32 ? launch_gemm<KIND, BN, SCALE_BLOCK_B, true>(tmA, tmB, tmO, g, idesc, st)
+                       : launch_gemm<KIND, BN, SCALE_BLOCK_B, false>(tmA, tmB, tmO, g, idesc, st);
+    return out_f32 ? launch_gemm<KIND, BN, SCALE_VEC_B, true>(tmA, tmB, tmO, g, idesc, st)
+                   : launch_gemm<KIND, BN, SCALE_VEC_B, false>(tmA, tmB, tmO, g, idesc, st);
 }
 
 }  // namespace
@@ -747,55 +587,37 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     g.out = out; g.ldo = No; g.accumulate = accumulate;
     g.status = static_cast<uint32_t *>(ws);
     g.stage_tx_bytes = 0;
-    g.trace = (getenv("SNIP_GEMM_TRACE") && ws_bytes >= 32768) ? reinterpret_cast<long long *>(static_cast<uint8_t *>(ws) + 1024) : nullptr;
     const bool f32 = out_dtype == SNIP_OUT_FP32;
 
     CUtensorMap tmA, tmB, tmO;
-    const bool pair = use_pair(Mo);
-    const uint32_t mma_m = pair ? 2 * BM : BM;
-    if (pair && !a16) {
-        // output boxes of 32 rows x 128 bytes for the epilogue's TMA stores
-        const int bn = (fmt_a == SNIP_FMT_FP4_E2M1 && fmt_b == SNIP_FMT_FP4_E2M1) ? 192 : 256;
-        const int box_bytes = out_box_bytes(f32, bn);
-        const CUtensorMapSwizzle swz = box_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
-        rc = f32 ? make_operand_map(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Mo, No, No * 4, box_bytes / 4, 32, swz)
-                 : make_operand_map(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Mo, No, No * 2, box_bytes / 2, 32, swz);
-        if (rc) return rc;
-    } else {
-        memset(&tmO, 0, sizeof(tmO));
-    }
+    // output boxes of 32 rows x 64 bytes for the TMA stores of the block-mode epilogue
+    rc = f32 ? make_operand_map(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Mo, No, No * 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_64B)
+             : make_operand_map(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Mo, No, No * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (rc) return rc;
     if (a16) {
-        constexpr int BN = 256;
-        const int brows = pair ? BN / 2 : BN;
         rc = make_operand_map(&tmA, a_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Mo, Kc, Kc * 2, 64, BM);
         if (rc) return rc;
-        rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, No, Kc, Kc * 2, 64, brows);
+        rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, No, Kc, Kc * 2, 64, 256);
         if (rc) return rc;
-        const uint32_t idesc = make_idesc(1, 1, mma_m, BN);
-        g.stage_tx_bytes = (BM + brows) * 128;
-        if (pair)
-            return f32 ? launch_gemm<MmaKind::F16, BN, SCALE_NONE, true, true>(tmA, tmB, tmA, g, idesc, st)
-                       : launch_gemm<MmaKind::F16, BN, SCALE_NONE, false, true>(tmA, tmB, tmA, g, idesc, st);
-        return f32 ? launch_gemm<MmaKind::F16, BN, SCALE_NONE, true, false>(tmA, tmB, tmA, g, idesc, st)
-                   : launch_gemm<MmaKind::F16, BN, SCALE_NONE, false, false>(tmA, tmB, tmA, g, idesc, st);
+        const uint32_t idesc = make_idesc(1, 1, BM, 256);
+        g.stage_tx_bytes = (BM + 256) * 128;
+        return f32 ? launch_gemm<MmaKind::F16, 256, SCALE_NONE, true>(tmA, tmB, tmO, g, idesc, st)
+                   : launch_gemm<MmaKind::F16, 256, SCALE_NONE, false>(tmA, tmB, tmO, g, idesc, st);
     }
     if (fmt_a == SNIP_FMT_FP4_E2M1 && fmt_b == SNIP_FMT_FP4_E2M1) {
         // packed FP4 on both sides: kind::mxf4 at twice the FP8 rate; the bytes are fetched as plain u8
         constexpr int BN = 192;
-        const int brows = pair ? BN / 2 : BN;
         rc = make_operand_map(&tmA, a_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, Kc / 2, Kc / 2, 128, BM);
         if (rc) return rc;
-        rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, brows);
+        rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN);
         if (rc) return rc;
-        const uint32_t idesc = make_idesc_block_scaled(1, 1, mma_m, BN);
-        g.stage_tx_bytes = (BM + brows) * 128;
-        return pair ? launch_gemm_scale<MmaKind::MXF4, BN, true>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st)
-                    : launch_gemm_scale<MmaKind::MXF4, BN, false>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
+        const uint32_t idesc = make_idesc_block_scaled(1, 1, BM, BN);
+        g.stage_tx_bytes = (BM + BN) * 128;
+        return launch_gemm_scale<MmaKind::MXF4, BN>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
     }
     // FP8 x FP8 and the mixed pairs: kind::f8f6f4; FP4 operands are expanded by the TMA unit to one
     // 16-byte-aligned group per 16 elements, which is the layout this MMA kind reads
     constexpr int BN = 256;
-    const int brows = pair ? BN / 2 : BN;
     const bool a4 = fmt_a == SNIP_FMT_FP4_E2M1, b4 = fmt_b == SNIP_FMT_FP4_E2M1;
     // The expanding 4-bit tensor-map type only accepts an inner extent that is a multiple of 128
     // elements.  A contraction length ending in a 64-wide tile is therefore declared rounded up: the
@@ -807,14 +629,13 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
                           a4 ? Kc / 2 : Kc, 128, BM);
     if (rc) return rc;
     rc = make_operand_map(&tmB, b_codes, b4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, No, b4 ? kpad : Kc,
-                          b4 ? Kc / 2 : Kc, 128, brows);
+                          b4 ? Kc / 2 : Kc, 128, BN);
     if (rc) return rc;
-    const uint32_t idesc = make_idesc(a4 ? 5 : 0, b4 ? 5 : 0, mma_m, BN);
+    const uint32_t idesc = make_idesc(a4 ? 5 : 0, b4 ? 5 : 0, BM, BN);
     // an FP4 operand expanded by the TMA unit occupies 128 B per row in shared memory but reports
     // only its 64 packed source bytes to the barrier
-    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + brows * (b4 ? 64 : 128);
-    return pair ? launch_gemm_scale<MmaKind::F8F6F4, BN, true>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st)
-                : launch_gemm_scale<MmaKind::F8F6F4, BN, false>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
+    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128);
+    return launch_gemm_scale<MmaKind::F8F6F4, BN>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
 }
 
 }  // namespace snip
