@@ -148,6 +148,25 @@ int snip_quantize(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
                   uint32_t flags, void *codes, float *scales, snip_stats_t *stats,
                   double *row_stats, void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * snip_quantize for callers that cannot hand the library any scratch memory.  (The paper has no
+ * counterpart; this is a deployment convenience.)  Meant for hosts that run under a fixed memory
+ * budget they do not control, or whose steady-state loop must never call the CUDA allocator: the
+ * statistics scratch is a 512 KiB array built into the library's device image, so this entry
+ * point allocates nothing, on the host or on the device.  Price: every GPU that loads the library
+ * holds those 512 KiB until the process exits.
+ *   - Same arguments and results as snip_quantize, minus row_stats / ws / ws_bytes (per-row sums
+ *     are not offered here).  Inputs up to 16384 tiles of 128x128 (e.g. 16384 x 16384 elements);
+ *     larger ones return SNIP_ERR_WORKSPACE and snip_last_cuda_error() says how much was needed.
+ *   - The first call on each device looks up the array's device address (one runtime query, no
+ *     allocation).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it needs
+ *     clearing (each call overwrites what it later reads), but two calls that may run on the GPU at
+ *     the same time (different streams, no dependency) race on it: serialize them.
+ */
+int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,
+                          uint32_t flags, void *codes, float *scales, snip_stats_t *stats, void *stream);
+
 /* ---- GEMMs (paper Fig. 5; Sec. 2.2: GEMM in FPX, output in BF16) -------------------------- */
 
 /*

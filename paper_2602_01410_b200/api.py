@@ -24,7 +24,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_workspace_size", "snip_gemm_quantized", "snip_linear_fwd",
+    "snip_quantize", "snip_quantize_noalloc", "snip_workspace_size", "snip_gemm_quantized", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_layer_stats", "snip_layer_stats_workspace",
     "snip_poll_status",
 )
@@ -61,6 +61,7 @@ def _load():
     lib.snip_last_cuda_error.restype = ctypes.c_char_p
     lib.snip_quantize_sizes.argtypes = [i64, i64, i32, i32, u32, psz, psz, psz]
     lib.snip_quantize.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
+    lib.snip_quantize_noalloc.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp]
     lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
     lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
@@ -138,6 +139,16 @@ def snip_quantize(x: torch.Tensor, fmt: int, block: int, flags: int = 0, *, code
     _check("snip_quantize", _lib.snip_quantize(_p(x), rows, cols, x.stride(0), fmt, block, flags, _p(codes), _p(scales),
                                                _p(stats), _p(row_stats), _p(ws), 0 if ws is None else ws.numel(), _stream()))
     return codes, scales, stats, row_stats
+
+
+def snip_quantize_noalloc(x: torch.Tensor, fmt: int, block: int, flags: int, codes, scales, stats):
+    """Same work as snip_quantize with the statistics scratch taken from the array built into the
+    library, for hosts that cannot give it any.  The caller passes every output buffer: this wrapper,
+    like the entry point, allocates nothing."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    _check("snip_quantize_noalloc", _lib.snip_quantize_noalloc(_p(x), rows, cols, x.stride(0), fmt, block, flags, _p(codes),
+                                                               _p(scales), _p(stats), _stream()))
 
 
 def snip_workspace_size(op, M, N, K, fmt_a, fmt_b):

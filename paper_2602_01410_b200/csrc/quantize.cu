@@ -599,3 +599,62 @@ extern "C" int snip_quantize(const void *x, int64_t rows, int64_t cols, int64_t 
     return snip::quantize_impl(x, rows, cols, ld, fmt, block, flags, codes, scales, stats, row_stats, ws, ws_bytes,
                                static_cast<cudaStream_t>(stream));
 }
+
+// ---- variant for callers that cannot allocate ------------------------------------------------
+//
+// Some users of this library cannot obtain scratch memory for us: a plug-in that runs inside a
+// host application's fixed memory budget, or a service whose steady-state loop must never reach
+// the CUDA allocator (cudaMalloc synchronizes the whole device and can fail under fragmentation).
+// For them the statistics scratch lives in a fixed array inside the library's device image: every
+// GPU that loads the library holds these kStaticScratchBytes until the process exits.
+namespace snip {
+namespace {
+
+constexpr size_t kStaticScratchTiles = 16384;                                 // 128x128 tiles, e.g. 16384 x 16384 elements
+constexpr size_t kStaticScratchBytes = kStaticScratchTiles * sizeof(CtaPartial);  // 512 KiB
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, not an address a kernel could use, so the address is looked up once per
+// device (with that device current) and cached.
+int static_scratch_address(void **out)
+{
+    constexpr int kMaxDevices = 64;
+    static void *cached[kMaxDevices] = {nullptr};
+    int dev = 0;
+    SNIP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SNIP_ERR_UNSUPPORTED;
+    void *p = __atomic_load_n(&cached[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        SNIP_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return SNIP_ERR_CUDA;
+        __atomic_store_n(&cached[dev], p, __ATOMIC_RELEASE);   // every thread computes the same value
+    }
+    *out = p;
+    return SNIP_OK;
+}
+
+}  // namespace
+}  // namespace snip
+
+extern "C" int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags,
+                                     void *codes, float *scales, snip_stats_t *stats, void *stream)
+{
+    using namespace snip;
+    if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
+    const size_t need = stats_ws_bytes(rows, cols, false);
+    if (need > kStaticScratchBytes) {
+        snprintf(last_error_buffer(), 256, "snip_quantize_noalloc: %lld x %lld needs %zu bytes of scratch, the built-in array holds %zu",
+                 (long long)rows, (long long)cols, need, kStaticScratchBytes);
+        return SNIP_ERR_WORKSPACE;
+    }
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != SNIP_OK) return rc;
+    // Nothing in the scratch has to start at zero: every CTA overwrites its own partial before the
+    // reduction kernel reads it, so stale contents of an earlier call are never observed.
+    return quantize_impl(x, rows, cols, ld, fmt, block, flags, codes, scales, stats, nullptr, scratch, kStaticScratchBytes,
+                         static_cast<cudaStream_t>(stream));
+}
+
