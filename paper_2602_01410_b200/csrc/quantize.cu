@@ -145,6 +145,9 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
     __shared__ float col_ninv[kTile];
     __shared__ float red_f[8][3];
 
+    // the statistics reduction that follows on the stream may be scheduled now; it waits for this
+    // grid to finish before it reads anything (programmatic dependent launch)
+    if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tx = tid & 15, ty = tid >> 4;
     const int64_t r0 = (int64_t)blockIdx.y * kTile, c0 = (int64_t)blockIdx.x * kTile;
@@ -438,32 +441,39 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
     }
 }
 
-// Fixed-order reduction of the per-CTA partials into one snip_stats_t (deterministic).
+// Fixed-order reduction of the per-CTA partials into one snip_stats_t (deterministic: every thread
+// owns a fixed strided subset, warps combine with shuffles, warp results are added in warp order).
+// Launched with programmatic stream serialization: it may start while the quantizer still runs and
+// blocks in griddepcontrol.wait until that grid has completed and its writes are visible.
 __global__ void __launch_bounds__(1024) stats_reduce_kernel(const CtaPartial *partials, int64_t n, snip_stats_t *out)
 {
-    __shared__ double sh_x[1024], sh_e[1024];
-    __shared__ float sh_m[1024];
+    __shared__ double sh_x[32], sh_e[32];
+    __shared__ float sh_m[32];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     double dx = 0.0, de = 0.0;
     float am = 0.0f;
     for (int64_t i = threadIdx.x; i < n; i += 1024) {
-        dx += partials[i].sumsq_x;
-        de += partials[i].sumsq_err;
+        const double2 p = *reinterpret_cast<const double2 *>(&partials[i]);
+        dx += p.x;
+        de += p.y;
         am = fmaxf(am, partials[i].amax);
     }
-    sh_x[threadIdx.x] = dx; sh_e[threadIdx.x] = de; sh_m[threadIdx.x] = am;
-    __syncthreads();
-    for (int s = 512; s > 0; s >>= 1) {
-        if ((int)threadIdx.x < s) {
-            sh_x[threadIdx.x] += sh_x[threadIdx.x + s];
-            sh_e[threadIdx.x] += sh_e[threadIdx.x + s];
-            sh_m[threadIdx.x] = fmaxf(sh_m[threadIdx.x], sh_m[threadIdx.x + s]);
-        }
-        __syncthreads();
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        dx += __shfl_xor_sync(0xFFFFFFFFu, dx, off);
+        de += __shfl_xor_sync(0xFFFFFFFFu, de, off);
+        am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, off));
     }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { sh_x[warp] = dx; sh_e[warp] = de; sh_m[warp] = am; }
+    __syncthreads();
     if (threadIdx.x == 0) {
-        out->sumsq_x = sh_x[0];
-        out->sumsq_err = sh_e[0];
-        out->amax = sh_m[0];
+        double tx = 0.0, te = 0.0;
+        float tm = 0.0f;
+        for (int w = 0; w < 32; ++w) { tx += sh_x[w]; te += sh_e[w]; tm = fmaxf(tm, sh_m[w]); }
+        out->sumsq_x = tx;
+        out->sumsq_err = te;
+        out->amax = tm;
         out->reserved = 0;
     }
 }
@@ -557,8 +567,18 @@ int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
     else launch_variant<SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, false>(a, false, true, want_rows, grid, st);
     SNIP_CUDA_TRY(cudaGetLastError());
     if (want_stats) {
-        stats_reduce_kernel<<<1, 1024, 0, st>>>(a.partials, tr * tc, stats);
-        SNIP_CUDA_TRY(cudaGetLastError());
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1);
+        cfg.blockDim = dim3(1024);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const CtaPartial *parts = a.partials;
+        const int64_t nparts = tr * tc;
+        SNIP_CUDA_TRY(cudaLaunchKernelEx(&cfg, stats_reduce_kernel, parts, nparts, stats));
     }
     if (want_rows) {
         row_stats_reduce_kernel<<<(unsigned)ceil_div(rows, 256), 256, 0, st>>>(a.row_partials, rows, tc, row_stats);
