@@ -416,10 +416,8 @@ def main():
     barrier()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    from paper_2602_01410_b200.replicas import combine_replicas
+    ms_total, flops_job = combine_replicas(ms_total, step.flops, dist if world > 1 else None, device)
     assert api.snip_poll_status(step.gws) == 0, "device-side timeout reported"
     # GEMM launches inside the timed region, per format: total flops / total event time
     in_region = {}
@@ -427,7 +425,7 @@ def main():
         d = in_region.setdefault(fmt, {"flops": 0.0, "ms": 0.0, "launches": 0})
         d["flops"] += fl; d["ms"] += a.elapsed_time(b); d["launches"] += 1
     ms_per_step = ms_total / args.steps
-    value = step.flops * world / (ms_per_step * 1e-3) / 1e12
+    value = flops_job / (ms_per_step * 1e-3) / 1e12
 
     # ---- end to end: inputs start in pinned host memory, statistics come back -------------------
     e2e = None
@@ -450,11 +448,8 @@ def main():
         s1.record()
         barrier()
         ms_e2e = s0.elapsed_time(s1) / n_e2e
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": step.flops * world / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+        ms_e2e, flops_e2e = combine_replicas(ms_e2e, step.flops, dist if world > 1 else None, device)
+        e2e = {"value": flops_e2e / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": stats_host.numel()}
         del host
 
