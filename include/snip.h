@@ -167,6 +167,24 @@ int snip_quantize(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
 int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,
                           uint32_t flags, void *codes, float *scales, snip_stats_t *stats, void *stream);
 
+/*
+ * Power-of-two scale option (an added quantization option in the sense of paper Sec. 3.2, which lets
+ * new quantization methods join the per-layer choices; power-of-two block scales are those of the MX
+ * formats cited in Sec. 2.3).  Identical to snip_quantize except for the scale rule:
+ * S = 2^e with the largest e such that amax * 2^e <= FPX_MAX (e clamped to [-126, 127], S = 1 for an
+ * all-zero tile), so x*S is exact and 1/S is an 8-bit exponent the tensor core can apply itself.
+ * `scales` receives S as FP32 in the usual layout (so the results also feed snip_gemm_quantized).
+ * `sf` (may be NULL) receives the UE8M0 bytes of 1/S (byte = 127 - e) as 512-byte atoms, one per
+ * 128x128 tile, atom index [operand row tile][contraction chunk] for the orientation the GEMM
+ * consumes (ROW: as stored; COL: transposed storage required; BLK: follows SNIP_Q_TRANSPOSED);
+ * inside an atom the byte of tile line r is stored four times at (r % 32) * 16 + (r / 32) * 4.
+ * snip_quantize_mx_sizes gives the byte size of sf.  Per-row statistics are not offered here.
+ */
+int snip_quantize_mx_sizes(int64_t rows, int64_t cols, size_t *sf_bytes_host);
+int snip_quantize_mx(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,
+                     uint32_t flags, void *codes, float *scales, void *sf, snip_stats_t *stats,
+                     void *ws, size_t ws_bytes, void *stream);
+
 /* ---- GEMMs (paper Fig. 5; Sec. 2.2: GEMM in FPX, output in BF16) -------------------------- */
 
 /*

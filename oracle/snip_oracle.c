@@ -178,6 +178,24 @@ float orc_tile_scale(int fmt, float amax)
     return r;
 }
 
+/* Power-of-two variant of the scale ("new quantization methods can be added as further options",
+ * Sec. 3.2; block scales that are powers of two are what the MX formats cited in Sec. 2.3 use):
+ * the largest S = 2^e with amax * S <= FPX_MAX, so that the hardware can apply 1/S as an 8-bit
+ * exponent.  e is clamped to [-126, 127]; S = 1 for an all-zero tile.  Worked out on the exponents
+ * and significands, no division: amax = m_a 2^ea, FPX_MAX = m_f 2^ef with m in [1,2), then
+ * e = ef - ea if m_a <= m_f, else ef - ea - 1. */
+float orc_tile_scale_pow2(int fmt, float amax)
+{
+    if (amax == 0.0f) return 1.0f;
+    int xa, xf;
+    double ma = 2.0 * frexp((double)amax, &xa);            /* amax = ma * 2^(xa-1) */
+    double mf = 2.0 * frexp(orc_fpx_max(fmt), &xf);
+    int e = (xf - 1) - (xa - 1) - (ma > mf ? 1 : 0);
+    if (e > 127) e = 127;
+    if (e < -126) e = -126;
+    return (float)ldexp(1.0, e);
+}
+
 /* ---------------------------------------------------------------------------------------- */
 /* Quantizer                                                                                 */
 /* ---------------------------------------------------------------------------------------- */
@@ -214,9 +232,20 @@ static int64_t orc_scale_index(int64_t rows, int64_t cols, int block, int64_t r,
  * fmt = BF16 is the identity: no scales, xhat = x, zero error.
  * Returns 0, or -1 on a bad argument.
  */
+int orc_quantize_rule(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block, int pow2_scale,
+                      uint8_t *codes, float *scales, double *xhat, double *sumsq, double *row_sumsq);
+
 int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block,
                  uint8_t *codes, float *scales, double *xhat, double *sumsq,
                  double *row_sumsq)
+{
+    return orc_quantize_rule(x, rows, cols, fmt, block, 0, codes, scales, xhat, sumsq, row_sumsq);
+}
+
+/* Same with the scale rule selectable: pow2_scale = 0 is the paper's quotient FPX_MAX / amax,
+ * pow2_scale = 1 the power-of-two option above.  Everything else is identical. */
+int orc_quantize_rule(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block, int pow2_scale,
+                      uint8_t *codes, float *scales, double *xhat, double *sumsq, double *row_sumsq)
 {
     if (!x || rows < 0 || cols < 0) return -1;
     if (fmt != ORC_FMT_BF16 && !orc_format(fmt)) return -1;
@@ -245,7 +274,7 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int blo
                     if (a > S[si]) S[si] = a;
                 }
         }
-        for (int64_t i = 0; i < nscales; ++i) S[i] = orc_tile_scale(fmt, S[i]);
+        for (int64_t i = 0; i < nscales; ++i) S[i] = pow2_scale ? orc_tile_scale_pow2(fmt, S[i]) : orc_tile_scale(fmt, S[i]);
         if (scales) memcpy(scales, S, sizeof(float) * (size_t)nscales);
     }
 

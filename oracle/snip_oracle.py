@@ -59,6 +59,10 @@ def lib() -> ctypes.CDLL:
         L.orc_scale_shape.argtypes = [i64, i64, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.orc_quantize.restype = i32
         L.orc_quantize.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp]
+        L.orc_quantize_rule.restype = i32
+        L.orc_quantize_rule.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.orc_tile_scale_pow2.restype = ctypes.c_float
+        L.orc_tile_scale_pow2.argtypes = [i32, ctypes.c_float]
         L.orc_dequantize.restype = i32
         L.orc_dequantize.argtypes = [vp, vp, i64, i64, i32, i32, vp]
         L.orc_pack_codes.restype = i32
@@ -106,6 +110,10 @@ def tile_scale(fmt: int, amax: float) -> np.float32:
     return np.float32(lib().orc_tile_scale(fmt, np.float32(amax)))
 
 
+def tile_scale_pow2(fmt: int, amax: float) -> np.float32:
+    return np.float32(lib().orc_tile_scale_pow2(fmt, np.float32(amax)))
+
+
 def bf16_to_float(bits: np.ndarray) -> np.ndarray:
     """Exact widening of bf16 bit patterns to float64."""
     b = np.ascontiguousarray(bits, dtype=np.uint16)
@@ -146,7 +154,7 @@ class Quantized:
         return pack_codes(self.codes, self.fmt, transposed)
 
 
-def quantize(x_bits: np.ndarray, fmt: int, block: int) -> Quantized:
+def quantize(x_bits: np.ndarray, fmt: int, block: int, pow2_scale: bool = False) -> Quantized:
     x = np.ascontiguousarray(x_bits, dtype=np.uint16)
     assert x.ndim == 2
     rows, cols = x.shape
@@ -156,8 +164,8 @@ def quantize(x_bits: np.ndarray, fmt: int, block: int) -> Quantized:
     xhat = np.empty((rows, cols), dtype=np.float64)
     sumsq = np.zeros(2, dtype=np.float64)
     row_sumsq = np.zeros((rows, 2), dtype=np.float64)
-    rc = lib().orc_quantize(_ptr(x), rows, cols, fmt, block, _ptr(codes), _ptr(scales),
-                            _ptr(xhat), _ptr(sumsq), _ptr(row_sumsq))
+    rc = lib().orc_quantize_rule(_ptr(x), rows, cols, fmt, block, int(pow2_scale), _ptr(codes), _ptr(scales),
+                                 _ptr(xhat), _ptr(sumsq), _ptr(row_sumsq))
     if rc != 0:
         raise ValueError("orc_quantize: bad argument")
     return Quantized(fmt, block, rows, cols, codes, scales, xhat, float(sumsq[0]),
@@ -221,24 +229,24 @@ def gemm_wgrad(dyhat: np.ndarray, xhat: np.ndarray) -> np.ndarray:
 
 # ---- the three GEMMs of one linear layer under a precision choice (Fig. 5) -------------------
 
-def linear_fwd(x_bits, w_bits, fmt_x, fmt_w):
+def linear_fwd(x_bits, w_bits, fmt_x, fmt_w, pow2_scale=False):
     """Quantize X with 1x128 tiles along K and W with 128x128 blocks, then Y = Xhat What^T."""
-    qx = quantize(x_bits, fmt_x, BLOCK_ROW)
-    qw = quantize(w_bits, fmt_w, BLOCK_BLK)
+    qx = quantize(x_bits, fmt_x, BLOCK_ROW, pow2_scale)
+    qw = quantize(w_bits, fmt_w, BLOCK_BLK, pow2_scale)
     return gemm_fwd(qx.xhat, qw.xhat), qx, qw
 
 
-def linear_dgrad(dy_bits, w_bits, fmt_dy, fmt_w):
+def linear_dgrad(dy_bits, w_bits, fmt_dy, fmt_w, pow2_scale=False):
     """Quantize dY with 1x128 tiles along N and W with 128x128 blocks, then dX = dYhat What."""
-    qdy = quantize(dy_bits, fmt_dy, BLOCK_ROW)
-    qw = quantize(w_bits, fmt_w, BLOCK_BLK)
+    qdy = quantize(dy_bits, fmt_dy, BLOCK_ROW, pow2_scale)
+    qw = quantize(w_bits, fmt_w, BLOCK_BLK, pow2_scale)
     return gemm_dgrad(qdy.xhat, qw.xhat), qdy, qw
 
 
-def linear_wgrad(dy_bits, x_bits, fmt_dy, fmt_x):
+def linear_wgrad(dy_bits, x_bits, fmt_dy, fmt_x, pow2_scale=False):
     """Quantize dY and X with 128x1 tiles along M (the contraction), then dW = dYhat^T Xhat."""
-    qdy = quantize(dy_bits, fmt_dy, BLOCK_COL)
-    qx = quantize(x_bits, fmt_x, BLOCK_COL)
+    qdy = quantize(dy_bits, fmt_dy, BLOCK_COL, pow2_scale)
+    qx = quantize(x_bits, fmt_x, BLOCK_COL, pow2_scale)
     return gemm_wgrad(qdy.xhat, qx.xhat), qdy, qx
 
 
@@ -265,3 +273,27 @@ def layer_stats(x_bits, w_bits, y_bits, dy_bits, dx_bits, dw_bits):
             for block in blocks:
                 out["sumsq_err"][(name, fmt, block)] = quantize(t, fmt, block).sumsq_err
     return out
+
+
+def sf_atoms(q: Quantized, transposed: bool) -> np.ndarray:
+    """UE8M0 scale-factor atoms of a power-of-two-scaled Quantized, in the library's layout: one
+    512-byte atom per 128x128 tile, indexed [operand row tile][contraction chunk] for the orientation
+    the GEMM consumes; inside an atom the byte 127 - e of tile line r (S = 2^e) sits four times at
+    (r % 32) * 16 + (r // 32) * 4.  Lines beyond the matrix hold 127."""
+    tr, tc = -(-q.rows // TILE), -(-q.cols // TILE)
+    exps = np.frexp(q.scales.astype(np.float64))[1] - 1            # S = 2^e exactly
+    byte = (127 - exps).astype(np.uint8)
+    out = np.full((tc, tr, 128, 4) if transposed else (tr, tc, 128, 4), 127, dtype=np.uint8)
+    for i in range(tr):
+        for j in range(tc):
+            if q.block == BLOCK_ROW:       # line = row inside the tile; scales[j][row]
+                lines = byte[j, i * TILE:min((i + 1) * TILE, q.rows)]
+            elif q.block == BLOCK_COL:     # line = column inside the tile; scales[i][col]
+                lines = byte[i, j * TILE:min((j + 1) * TILE, q.cols)]
+            else:
+                lines = np.full(TILE, byte[i, j], dtype=np.uint8)
+            atom = out[j, i] if transposed else out[i, j]
+            for r, b in enumerate(lines):
+                atom[(r % 32) * 4 + r // 32, :] = b
+    return out.reshape(-1)
+

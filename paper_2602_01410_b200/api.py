@@ -24,7 +24,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_quantize_noalloc", "snip_workspace_size", "snip_gemm_quantized", "snip_linear_fwd",
+    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_workspace_size", "snip_gemm_quantized", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_layer_stats", "snip_layer_stats_workspace",
     "snip_poll_status",
 )
@@ -62,6 +62,8 @@ def _load():
     lib.snip_quantize_sizes.argtypes = [i64, i64, i32, i32, u32, psz, psz, psz]
     lib.snip_quantize.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
     lib.snip_quantize_noalloc.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp]
+    lib.snip_quantize_mx_sizes.argtypes = [i64, i64, psz]
+    lib.snip_quantize_mx.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
     lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
     lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
@@ -149,6 +151,27 @@ def snip_quantize_noalloc(x: torch.Tensor, fmt: int, block: int, flags: int, cod
     rows, cols = x.shape
     _check("snip_quantize_noalloc", _lib.snip_quantize_noalloc(_p(x), rows, cols, x.stride(0), fmt, block, flags, _p(codes),
                                                                _p(scales), _p(stats), _stream()))
+
+
+def snip_quantize_mx(x: torch.Tensor, fmt: int, block: int, flags: int = 0, *, want_sf=True):
+    """Power-of-two scale option.  Returns (codes, scales, sf, stats): uint8, float32, uint8 (UE8M0
+    atoms, None unless want_sf) and a 32-byte stats buffer (None unless Q_STATS)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    cb, sb, wb = snip_quantize_sizes(rows, cols, fmt, block, flags)
+    dev = x.device
+    codes = torch.empty(cb, dtype=torch.uint8, device=dev)
+    scales = torch.empty(sb // 4, dtype=torch.float32, device=dev)
+    sf = None
+    if want_sf:
+        n = ctypes.c_size_t()
+        _check("snip_quantize_mx_sizes", _lib.snip_quantize_mx_sizes(rows, cols, ctypes.byref(n)))
+        sf = torch.empty(n.value, dtype=torch.uint8, device=dev)
+    stats = torch.empty(32, dtype=torch.uint8, device=dev) if (flags & Q_STATS) else None
+    ws = torch.empty(wb, dtype=torch.uint8, device=dev) if (flags & Q_STATS) else None
+    _check("snip_quantize_mx", _lib.snip_quantize_mx(_p(x), rows, cols, x.stride(0), fmt, block, flags, _p(codes), _p(scales), _p(sf),
+                                                     _p(stats), _p(ws), 0 if ws is None else ws.numel(), _stream()))
+    return codes, scales, sf, stats
 
 
 def snip_workspace_size(op, M, N, K, fmt_a, fmt_b):

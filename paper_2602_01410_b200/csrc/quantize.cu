@@ -36,6 +36,8 @@ struct QuantArgs {
     float *scales;        // may be null (NO_CODES)
     CtaPartial *partials; // may be null (no stats)
     float2 *row_partials; // [col tiles][rows] {sum x^2, sum err^2}; may be null
+    int pow2;             // 1: power-of-two scale rule (largest 2^e with amax * 2^e <= FPX_MAX)
+    uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
 };
 
 __device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
@@ -59,15 +61,37 @@ __device__ __forceinline__ uint32_t max2(uint32_t x, uint32_t y)
     return *reinterpret_cast<uint32_t *>(&m);
 }
 
-// Scale of a tile from its amax: IEEE binary32 quotient, 1 for an empty tile, clamped.
+// Scale of a tile from its amax.  Paper's rule: IEEE binary32 quotient FPX_MAX / amax, 1 for an empty
+// tile, clamped to FLT_MAX.  Power-of-two option: the largest 2^e with amax * 2^e <= FPX_MAX, worked out
+// on the exponent and significand bits (no division), e clamped to [-126, 127].
 template <int FMT>
-__device__ __forceinline__ float tile_scale(float amax)
+__device__ __forceinline__ float tile_scale(float amax, int pow2)
 {
     constexpr float kMax = (FMT == SNIP_FMT_FP8_E4M3) ? 448.0f : 6.0f;
     if (amax == 0.0f) return 1.0f;
+    if (pow2) {
+        constexpr int kMaxExp = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 2;                       // FPX_MAX = m_f * 2^kMaxExp
+        constexpr uint32_t kMaxMant = (FMT == SNIP_FMT_FP8_E4M3) ? 0x600000u : 0x400000u;  // m_f = 1.75 / 1.5
+        const uint32_t b = __float_as_uint(amax);
+        const int ef = (int)(b >> 23);                 // biased exponent; 0 for a (bf16) subnormal amax
+        if (ef == 0) return __uint_as_float(254u << 23);   // amax < 2^-126: the clamp e = 127 applies
+        int e = kMaxExp - (ef - 127) - (((b & 0x7FFFFFu) > kMaxMant) ? 1 : 0);
+        e = max(-126, min(127, e));
+        return __uint_as_float((uint32_t)(e + 127) << 23);
+    }
     float s = __fdiv_rn(kMax, amax);
     return fminf(s, FLT_MAX);  // +inf -> FLT_MAX
 }
+// -1/S for the error term.  Paper's rule: amax/FPX_MAX equals 1/S to within one rounding, which the
+// statistics (1e-4) do not see; power-of-two rule: exact.  For an empty tile the value is irrelevant.
+template <int FMT>
+__device__ __forceinline__ float neg_inv_scale(float amax, float s, int pow2)
+{
+    constexpr float kMax = (FMT == SNIP_FMT_FP8_E4M3) ? 448.0f : 6.0f;
+    return pow2 ? -__fdiv_rn(1.0f, s) : -amax * (1.0f / kMax);
+}
+// UE8M0 byte of 1/S for a power-of-two S, replicated into the four bytes of a word
+__device__ __forceinline__ uint32_t sf_word(float s) { return (254u - (__float_as_uint(s) >> 23)) * 0x01010101u; }
 
 // Two binary32 values -> two codes.  `lo` lands in the low byte / nibble.
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
@@ -170,7 +194,6 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
     }
 
     // ---- block amax -> scales --------------------------------------------------------
-    constexpr float kFpxMax = (FMT == SNIP_FMT_FP4_E2M1) ? 6.0f : 448.0f;
     float s_row[8], s_col[8];  // scale per row p (ROW) / per column j (COL); BLK uses s_row[0]
     float n_row[8], n_col[8];  // matching -1/S for the error term
     (void)s_row; (void)s_col; (void)n_row; (void)n_col;
@@ -205,10 +228,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
 #pragma unroll
             for (int q = 1; q < 4; ++q) sel = ((myp >> 1) == q) ? pk[q] : sel;
             float am = (myp & 1) ? bf16hi(sel) : bf16lo(sel);
-            float mine = tile_scale<FMT>(am);
-            // -1/S for the error term: amax/FPX_MAX equals 1/S to within one rounding, which the
-            // statistics (1e-4) do not see; for an empty tile the value is irrelevant (all codes 0)
-            float mine_ninv = -am * (1.0f / kFpxMax);
+            float mine = tile_scale<FMT>(am, a.pow2);
+            float mine_ninv = neg_inv_scale<FMT>(am, mine, a.pow2);
 #pragma unroll
             for (int p = 0; p < 8; ++p) {
                 s_row[p] = __shfl_sync(0xFFFFFFFFu, mine, (lane & 16) | p);
@@ -217,6 +238,15 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             if (STATS) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) my_amax = fmaxf(my_amax, fmaxf(bf16lo(pk[q]), bf16hi(pk[q])));
+            }
+            if (CODES && tx == 0 && a.sf) {
+                // atom [row tile][column tile]: word (r % 32) * 4 + r / 32 holds row r's byte four times
+                uint32_t *atom = a.sf + ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * 128;
+#pragma unroll
+                for (int p = 0; p < 8; ++p) {
+                    const int r = 8 * ty + p;
+                    atom[(r & 31) * 4 + (r >> 5)] = (rbase + p < a.rows) ? sf_word(s_row[p]) : 0x7F7F7F7Fu;
+                }
             }
             if (CODES && tx == 0) {
                 // scales[tile j][row]: eight consecutive rows per thread
@@ -249,9 +279,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
 #pragma unroll
                     for (int w = 0; w < 8; ++w) m = max(m, (uint32_t)h[w * kTile + tid]);  // non-negative bf16: integer order
                     float am = __uint_as_float(m << 16);
-                    float s = tile_scale<FMT>(am);
+                    float s = tile_scale<FMT>(am, a.pow2);
                     col_scale[tid] = s;
-                    col_ninv[tid] = -am * (1.0f / kFpxMax);
+                    col_ninv[tid] = neg_inv_scale<FMT>(am, s, a.pow2);
+                    // atom [column tile][row tile] (the operand is consumed transposed): one word per column
+                    if (CODES && a.sf) a.sf[((int64_t)blockIdx.x * gridDim.y + blockIdx.y) * 128 + (tid & 31) * 4 + (tid >> 5)] = (c0 + tid < a.cols) ? sf_word(s) : 0x7F7F7F7Fu;
                     if (CODES && c0 + tid < a.cols) a.scales[(int64_t)blockIdx.y * a.cols + c0 + tid] = s;
                     if (STATS) my_amax = am;
                 }
@@ -279,8 +311,12 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
                 for (int w = 1; w < 8; ++w) bm = fmaxf(bm, red_f[w][2]);
                 my_amax = bm;
                 if (kQuant) {
-                    s_row[0] = tile_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm);
-                    n_row[0] = -bm * (1.0f / kFpxMax);
+                    s_row[0] = tile_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm, a.pow2);
+                    n_row[0] = neg_inv_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm, s_row[0], a.pow2);
+                    if (CODES && a.sf && tid < kTile) {
+                        const int64_t atom = TRANSPOSED ? (int64_t)blockIdx.x * gridDim.y + blockIdx.y : (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+                        a.sf[atom * 128 + tid] = sf_word(s_row[0]);
+                    }
                     if (CODES && tid == 0) a.scales[(int64_t)blockIdx.y * gridDim.x + blockIdx.x] = s_row[0];
                 }
                 __syncthreads();  // red_f is reused below
@@ -529,10 +565,25 @@ size_t stats_ws_bytes(int64_t rows, int64_t cols, bool rowstats)
 }  // namespace
 
 // Internal entry used by snip_quantize and by the linear-layer calls.
+int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf,
+                     void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st);
+
 int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags,
                   void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes,
                   cudaStream_t st)
 {
+    return quantize_impl_ex(x, rows, cols, ld, fmt, block, flags, 0, nullptr, codes, scales, stats, row_stats, ws, ws_bytes, st);
+}
+
+// pow2 = 1 selects the power-of-two scale rule; sf (optional, needs pow2) receives the UE8M0 atoms.
+int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf,
+                     void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    if (sf) {
+        const bool tr = (flags & SNIP_Q_TRANSPOSED) != 0;
+        // atoms follow the orientation the GEMM consumes: row tiles as stored, column tiles transposed
+        if (!pow2 || !aligned16(sf) || (block == SNIP_BLOCK_ROW_1x128 && tr) || (block == SNIP_BLOCK_COL_128x1 && !tr)) return SNIP_ERR_UNSUPPORTED;
+    }
     if (!x || !valid_fmt(fmt) || !valid_block(block)) return SNIP_ERR_ARG;
     if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0) return SNIP_ERR_SHAPE;
     const bool want_stats = (flags & SNIP_Q_STATS) != 0;
@@ -557,6 +608,7 @@ int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
     QuantArgs a;
     a.x = static_cast<const uint16_t *>(x);
     a.rows = rows; a.cols = cols; a.ld = ld;
+    a.pow2 = pow2; a.sf = static_cast<uint32_t *>(sf);
     a.codes = want_codes ? static_cast<uint8_t *>(codes) : nullptr;
     a.scales = want_codes ? scales : nullptr;
     a.partials = any_stats ? static_cast<CtaPartial *>(ws) : nullptr;
@@ -676,5 +728,25 @@ extern "C" int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, 
     // reduction kernel reads it, so stale contents of an earlier call are never observed.
     return quantize_impl(x, rows, cols, ld, fmt, block, flags, codes, scales, stats, nullptr, scratch, kStaticScratchBytes,
                          static_cast<cudaStream_t>(stream));
+}
+
+// ---- power-of-two ("MX-style") option -------------------------------------------------------
+
+extern "C" int snip_quantize_mx_sizes(int64_t rows, int64_t cols, size_t *sf_bytes)
+{
+    using namespace snip;
+    if (!sf_bytes) return SNIP_ERR_ARG;
+    if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
+    *sf_bytes = (size_t)(ceil_div(rows, 128) * ceil_div(cols, 128)) * 512;
+    return SNIP_OK;
+}
+
+extern "C" int snip_quantize_mx(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags,
+                                void *codes, float *scales, void *sf, snip_stats_t *stats, void *ws, size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    if (fmt == SNIP_FMT_BF16) return SNIP_ERR_UNSUPPORTED;
+    return quantize_impl_ex(x, rows, cols, ld, fmt, block, flags, 1, sf, codes, scales, stats, nullptr, ws, ws_bytes,
+                            static_cast<cudaStream_t>(stream));
 }
 

@@ -123,3 +123,35 @@ def test_ragged_3b_ffn_width(api):
         check_quantize(api, x, fmt, ROW, False)
         check_quantize(api, x, fmt, COL, True)
         check_quantize(api, x, fmt, BLK, True)
+
+
+@pytest.mark.parametrize("fmt", [FP8, FP4])
+@pytest.mark.parametrize("block,transposed", [(ROW, False), (COL, True), (BLK, False), (BLK, True)])
+@pytest.mark.parametrize("shape", [(256, 384), (192, 320)])
+def test_power_of_two_scale_option(api, fmt, block, transposed, shape):
+    rng = np.random.default_rng(77)
+    x = wl.to_bf16_bits(rng.standard_normal(shape).astype(np.float32) * np.exp(rng.standard_normal((shape[0], 1))).astype(np.float32))
+    q = orc.quantize(x, fmt, block, pow2_scale=True)
+    flags = api.Q_STATS | (api.Q_TRANSPOSED if transposed else 0)
+    codes, scales, sf, stats = api.snip_quantize_mx(to_dev(x), fmt, block, flags)
+    torch.cuda.synchronize()
+    want = q.packed(transposed)
+    assert np.array_equal(codes.cpu().numpy()[:want.size].reshape(want.shape), want)
+    assert np.array_equal(scales.cpu().numpy().reshape(q.scales.shape).view(np.uint32), q.scales.view(np.uint32))
+    assert np.array_equal(sf.cpu().numpy(), orc.sf_atoms(q, transposed))
+    st = api.stats_to_host(stats)
+    assert st["sumsq_err"] == pytest.approx(q.sumsq_err, rel=STATS_RTOL)
+    assert st["sumsq_x"] == pytest.approx(q.sumsq_x, rel=STATS_RTOL)
+
+
+def test_power_of_two_scales_on_degenerate_tiles(api):
+    x = np.zeros((128, 256), dtype=np.uint16)
+    x[:, 128:] = 0x0001                                   # bf16 subnormals: exponent clamp
+    x[5, 7] = wl.to_bf16_bits(np.array([3.0e38], dtype=np.float32))[0]
+    for fmt in (FP8, FP4):
+        q = orc.quantize(x, fmt, ROW, pow2_scale=True)
+        codes, scales, sf, _ = api.snip_quantize_mx(to_dev(x), fmt, ROW, 0)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes.cpu().numpy()[:q.packed().size].reshape(q.packed().shape), q.packed())
+        assert np.array_equal(scales.cpu().numpy().reshape(q.scales.shape).view(np.uint32), q.scales.view(np.uint32))
+        assert np.array_equal(sf.cpu().numpy(), orc.sf_atoms(q, False))
