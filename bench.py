@@ -227,24 +227,25 @@ class KernelTimer:
     def __init__(self, api, torch, cfg, device):
         self.api, self.torch, self.cfg, self.device = api, torch, cfg, device
 
-    def gemm(self, fmt, op, lin_index, iters=20, warmup=3):
+    def gemm(self, fmt, op, lin_index, iters=20, warmup=3, mx=False):
         api, torch = self.api, self.torch
         L = self.cfg.linears[lin_index]
         M, N, K = self.cfg.M, L.N, L.K
         g = torch.Generator(device=self.device); g.manual_seed(1)
         def rnd(r, c, s=1.0):
             return (torch.randn(r, c, generator=g, device=self.device, dtype=torch.float32) * s).to(torch.bfloat16)
+        quant = (lambda t, f, blk, fl=0: api.snip_quantize_mx(t, f, blk, fl)) if mx else (lambda t, f, blk, fl=0: api.snip_quantize(t, f, blk, fl))
         if op == api.OP_FWD:
             A, B, out_shape = rnd(M, K), rnd(N, K, 0.02), (M, N)
-            qa = api.snip_quantize(A, fmt, api.BLOCK_ROW); qb = api.snip_quantize(B, fmt, api.BLOCK_BLK)
+            qa = quant(A, fmt, api.BLOCK_ROW); qb = quant(B, fmt, api.BLOCK_BLK)
             a = api.make_qtensor(qa[0], qa[1], M, K, fmt, api.BLOCK_ROW); b = api.make_qtensor(qb[0], qb[1], N, K, fmt, api.BLOCK_BLK)
         elif op == api.OP_DGRAD:
             A, B, out_shape = rnd(M, N, 1e-3), rnd(N, K, 0.02), (M, K)
-            qa = api.snip_quantize(A, fmt, api.BLOCK_ROW); qb = api.snip_quantize(B, fmt, api.BLOCK_BLK, api.Q_TRANSPOSED)
+            qa = quant(A, fmt, api.BLOCK_ROW); qb = quant(B, fmt, api.BLOCK_BLK, api.Q_TRANSPOSED)
             a = api.make_qtensor(qa[0], qa[1], M, N, fmt, api.BLOCK_ROW); b = api.make_qtensor(qb[0], qb[1], N, K, fmt, api.BLOCK_BLK, True)
         else:
             A, B, out_shape = rnd(M, N, 1e-3), rnd(M, K), (N, K)
-            qa = api.snip_quantize(A, fmt, api.BLOCK_COL, api.Q_TRANSPOSED); qb = api.snip_quantize(B, fmt, api.BLOCK_COL, api.Q_TRANSPOSED)
+            qa = quant(A, fmt, api.BLOCK_COL, api.Q_TRANSPOSED); qb = quant(B, fmt, api.BLOCK_COL, api.Q_TRANSPOSED)
             a = api.make_qtensor(qa[0], qa[1], M, N, fmt, api.BLOCK_COL, True); b = api.make_qtensor(qb[0], qb[1], M, K, fmt, api.BLOCK_COL, True)
         out = torch.empty(out_shape, dtype=torch.bfloat16, device=self.device)
         ws = torch.zeros(1024, dtype=torch.uint8, device=self.device)
@@ -254,7 +255,10 @@ class KernelTimer:
             flush.zero_()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            api.snip_gemm_quantized(op, a, b, out_shape, api.OUT_BF16, out=out, ws=ws)
+            if mx:
+                api.snip_gemm_mx(op, a, qa[2], b, qb[2], out_shape, api.OUT_BF16, out=out, ws=ws)
+            else:
+                api.snip_gemm_quantized(op, a, b, out_shape, api.OUT_BF16, out=out, ws=ws)
             e1.record()
             torch.cuda.synchronize()
             if i >= warmup:
@@ -313,7 +317,8 @@ def run_profile_case(name):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     parts = name.split("_")
-    fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4}[parts[1]]
+    mx = parts[1].startswith("mx")
+    fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4, "mxfp8": FMT_FP8, "mxfp4": FMT_FP4}[parts[1]]
     if parts[0] == "quantize":
         kind = "_".join(parts[2:])
         block, tr = {"row": (api.BLOCK_ROW, False), "col_t": (api.BLOCK_COL, True), "blk_t": (api.BLOCK_BLK, True),
@@ -328,7 +333,7 @@ def run_profile_case(name):
         kt = KernelTimer(api, torch, cfg, device)
         if fmt == FMT_BF16:
             raise SystemExit("bf16 GEMM cases run through snip_linear_*; use fp8/fp4 here")
-        fl, times = kt.gemm(fmt, op, 0, iters=3, warmup=1)
+        fl, times = kt.gemm(fmt, op, 0, iters=3, warmup=1, mx=mx)
         print(f"{name}: {fl / (min(times) * 1e-3) / 1e12:.0f} TFLOP/s best of {len(times)}")
 
 

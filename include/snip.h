@@ -216,6 +216,17 @@ int snip_gemm_quantized(int op, const snip_qtensor_t *a_host, const snip_qtensor
                         void *stream);
 
 /*
+ * GEMM for the power-of-two scale option: same three products and operand layouts as
+ * snip_gemm_quantized, over operands produced by snip_quantize_mx; sf_a / sf_b are their UE8M0
+ * atoms.  The tensor core applies 2^-e per 128-long chunk itself (block-scaled MMA), so the whole
+ * contraction accumulates in FP32 tensor memory with no per-chunk promotion.  Operand formats: FP8
+ * and FP4 in any combination (no BF16).  ws: at least 256 bytes, first word = device status word.
+ * (An added option: the paper's rule stays snip_gemm_quantized.)
+ */
+int snip_gemm_mx(int op, const snip_qtensor_t *a_host, const void *sf_a, const snip_qtensor_t *b_host,
+                 const void *sf_b, void *out, int out_dtype, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * One linear layer's forward GEMM under a precision choice: quantize X (1x128 tiles along K)
  * and W (128x128 blocks) into the workspace, then Y = Xq.Wq^T.  stats_x / stats_w may be NULL;
  * if given they receive the statistics of the two quantizations.  (Fig. 5, forward pass.)

@@ -24,7 +24,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_workspace_size", "snip_gemm_quantized", "snip_linear_fwd",
+    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_layer_stats", "snip_layer_stats_workspace",
     "snip_poll_status",
 )
@@ -66,6 +66,7 @@ def _load():
     lib.snip_quantize_mx.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
     lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
+    lib.snip_gemm_mx.argtypes = [i32, ctypes.POINTER(QTensor), vp, ctypes.POINTER(QTensor), vp, vp, i32, vp, sz, vp]
     lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_fwd.argtypes = lin
     lib.snip_linear_dgrad.argtypes = lin
@@ -200,6 +201,15 @@ def snip_gemm_quantized(op, a: QTensor, b: QTensor, out_shape, out_dtype=OUT_BF1
         ws = torch.zeros(g, dtype=torch.uint8, device=out.device)
     _check("snip_gemm_quantized", _lib.snip_gemm_quantized(op, ctypes.byref(a), ctypes.byref(b), _p(out), out_dtype,
                                                            int(accumulate), _p(ws), ws.numel(), _stream()))
+    return out
+
+
+def snip_gemm_mx(op, a: QTensor, sf_a, b: QTensor, sf_b, out_shape, out_dtype=OUT_BF16, *, out=None, ws=None, device="cuda"):
+    out = _out(out_shape, out_dtype, device, out)
+    if ws is None:
+        ws = torch.zeros(256, dtype=torch.uint8, device=out.device)
+    _check("snip_gemm_mx", _lib.snip_gemm_mx(op, ctypes.byref(a), _p(sf_a), ctypes.byref(b), _p(sf_b), _p(out), out_dtype, _p(ws),
+                                             ws.numel(), _stream()))
     return out
 
 

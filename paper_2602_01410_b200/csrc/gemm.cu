@@ -554,6 +554,15 @@ int launch_gemm_scale(int scale, bool out_f32, const CUtensorMap &tmA, const CUt
 
 size_t gemm_ws_bytes() { return 256; }
 
+// Shared with the power-of-two-scale GEMMs: 2-D tiled tensor map over a row-major matrix.
+int make_tiled_map_2d(CUtensorMap *map, const void *ptr, int dtype, int64_t rows, int64_t inner_elems, int64_t row_bytes, int box_x_elems,
+                      int box_rows, int swizzle)
+{
+    return make_operand_map(map, ptr, static_cast<CUtensorMapDataType>(dtype), rows, inner_elems, row_bytes, box_x_elems, box_rows,
+                            static_cast<CUtensorMapSwizzle>(swizzle));
+}
+int gemm_sm_count() { return sm_count(); }
+
 int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st)
 {
     dim3 grid((unsigned)ceil_div(cols, 64), (unsigned)ceil_div(rows, 64)), block(32, 8);

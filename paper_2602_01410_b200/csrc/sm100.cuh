@@ -180,6 +180,13 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// 1-D bulk copy global -> shared (16-byte aligned, size a multiple of 16), counted on `bar`.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 // ---- tensor memory ---------------------------------------------------------------------
 // Allocate `ncols` (power of two >= 32) columns; the base address is written to shared memory.
 // Must be executed by one full warp.
@@ -269,6 +276,20 @@ __device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t v)
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Copy a 512-byte scale-factor atom (32 rows x 16 bytes, rows contiguous) from shared memory into
+// four tensor-memory columns, replicated into the four 32-lane quarters.  Runs in the tensor core's
+// queue, in issue order with the MMAs of the same thread.
+__device__ __forceinline__ void tmem_cp_sf_atom(uint32_t taddr, uint32_t smem_addr)
+{
+    // shared-memory matrix descriptor without swizzle: 8-row groups 128 bytes apart, one 16-byte column
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)(16 >> 4) << 16;     // leading byte offset (a single 16-byte column: unused)
+    d |= (uint64_t)(128 >> 4) << 32;    // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;             // descriptor version for sm_100
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+}
+
 // ---- descriptors -----------------------------------------------------------------------
 // Shared-memory matrix descriptor for a K-major operand tile whose rows are 128 bytes long and
 // stored with the 128-byte swizzle (what a TMA box of 128 bytes x rows produces): rows 128 B
@@ -298,7 +319,7 @@ __host__ __device__ constexpr uint32_t make_idesc_block_scaled(uint32_t a_fmt, u
     return (a_fmt << 7) | (b_fmt << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24);
 }
 
-enum class MmaKind { F16, F8F6F4, MXF4 };
+enum class MmaKind { F16, F8F6F4, MXF4, MXF8 };   // MXF8 = kind::mxf8f6f4 with hardware block scales
 
 template <MmaKind KIND, bool PAIR>
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
@@ -313,6 +334,11 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                                                       \
                      "tcgen05.mma.cta_group::" GROUP ".kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),                   \
                      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");                                        \
+    } else if constexpr (KIND == MmaKind::MXF8) {                                                                              \
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                                                       \
+                     "tcgen05.mma.cta_group::" GROUP ".kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"        \
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)         \
+                     : "memory");                                                                                              \
     } else {                                                                                                                   \
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                                                       \
                      "tcgen05.mma.cta_group::" GROUP ".kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}" \
