@@ -181,9 +181,10 @@ class Step:
         self.codes = [torch.empty(cb, dtype=torch.uint8, device=dev) for _ in range(2)]
         self.scales = [torch.empty(sb // 4, dtype=torch.float32, device=dev) for _ in range(2)]
         self.qws = torch.empty(wb, dtype=torch.uint8, device=dev)
+        self.sf = [torch.empty(cb // 32 + 4096, dtype=torch.uint8, device=dev) for _ in range(2)]   # UE8M0 atoms (power-of-two option)
         self.gws = torch.zeros(1024, dtype=torch.uint8, device=dev)
 
-    def run_decomposed(self, events=None):
+    def run_decomposed(self, events=None, mx=False):
         api, torch = self.api, self.torch
         if not hasattr(self, "codes"):
             self._alloc_decomposed()
@@ -193,8 +194,12 @@ class Step:
 
         def quant(x, fmt, block, flags, slot, stats):
             r, c = x.shape
-            api._check("snip_quantize", lib.snip_quantize(p(x), r, c, c, fmt, block, flags | api.Q_STATS, p(self.codes[slot]), p(self.scales[slot]),
-                                                          p(stats), None, p(self.qws), self.qws.numel(), st))
+            if mx:
+                api._check("snip_quantize_mx", lib.snip_quantize_mx(p(x), r, c, c, fmt, block, flags | api.Q_STATS, p(self.codes[slot]), p(self.scales[slot]),
+                                                                    p(self.sf[slot]), p(stats), p(self.qws), self.qws.numel(), st))
+            else:
+                api._check("snip_quantize", lib.snip_quantize(p(x), r, c, c, fmt, block, flags | api.Q_STATS, p(self.codes[slot]), p(self.scales[slot]),
+                                                              p(stats), None, p(self.qws), self.qws.numel(), st))
 
         def gemm(op, fmt, ra, ca, blka, ta, rb, cb_, blkb, tb, out, flops):
             a = api.make_qtensor(self.codes[0], self.scales[0], ra, ca, fmt, blka, ta)
@@ -202,7 +207,10 @@ class Step:
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-            api._check("snip_gemm_quantized", lib.snip_gemm_quantized(op, a, b, p(out), api.OUT_BF16, 0, p(self.gws), self.gws.numel(), st))
+            if mx:
+                api._check("snip_gemm_mx", lib.snip_gemm_mx(op, a, p(self.sf[0]), b, p(self.sf[1]), p(out), api.OUT_BF16, p(self.gws), self.gws.numel(), st))
+            else:
+                api._check("snip_gemm_quantized", lib.snip_gemm_quantized(op, a, b, p(out), api.OUT_BF16, 0, p(self.gws), self.gws.numel(), st))
             if events is not None:
                 e1.record()
                 events.append((fmt, op, flops, e0, e1))
@@ -432,6 +440,30 @@ def main():
     ms_per_step = ms_total / args.steps
     value = flops_job / (ms_per_step * 1e-3) / 1e12
 
+    # ---- the same step under the power-of-two scale option (hardware-applied scales) ----------------
+    for _ in range(3):
+        step.run_decomposed(mx=True)
+    barrier()
+    mx_events = []
+    m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    m0.record()
+    for _ in range(args.steps):
+        step.run_decomposed(mx_events, mx=True)
+    m1.record()
+    barrier()
+    ms_mx, flops_mx = combine_replicas(m0.elapsed_time(m1), step.flops, dist if world > 1 else None, device)
+    assert api.snip_poll_status(step.gws) == 0, "device-side timeout reported"
+    mx_region = {}
+    for fmt, op, fl, a, b in mx_events:
+        d = mx_region.setdefault(fmt, {"flops": 0.0, "ms": 0.0})
+        d["flops"] += fl; d["ms"] += a.elapsed_time(b)
+    pow2_option = {"value": flops_mx / (ms_mx / args.steps * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_mx / args.steps,
+                   "note": "same step with S = 2^e scales applied by the tensor core (snip_quantize_mx + snip_gemm_mx); an added quantization option, not the paper's rule",
+                   "gemm": {FMT_NAME[f]: {"tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12,
+                                          "frac_of_sustained_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f]),
+                                          "frac_of_burst_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops"] * NOMINAL_RATIO[f])}
+                            for f, d in mx_region.items()}}
+
     # ---- end to end: inputs start in pinned host memory, statistics come back -------------------
     e2e = None
     if rank == 0 or world > 1:
@@ -466,7 +498,7 @@ def main():
     # ---- kernel legs: the GEMM and quantizer kernels alone, events around each launch ---------------
     roofline, kernels = None, {}
     if not args.no_kernel_legs:
-        del step.inputs, step.out, step.codes, step.scales
+        del step.inputs, step.out, step.codes, step.scales, step.sf
         torch.cuda.empty_cache()
         kt = KernelTimer(api, torch, cfg, device)
         qkv = 0
@@ -513,7 +545,7 @@ def main():
             "config": {"workload": f"{cfg.name}: one block (qkv,o,gate,up,down) x (fwd,dgrad,wgrad) all-FP4 then all-FP8, tokens {cfg.M}, quantize+stats every GEMM",
                        "l2": "inputs larger than L2", "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": step.launches_per_step * args.steps,
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+            "roofline": roofline, "kernels": kernels, "pow2_option": pow2_option, "cpu_baseline": cpu}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

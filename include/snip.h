@@ -248,6 +248,17 @@ int snip_linear_wgrad(const void *dY, const void *X, void *dW, int64_t M, int64_
                       snip_stats_t *stats_dy, snip_stats_t *stats_x, void *ws, size_t ws_bytes,
                       void *stream);
 
+/*
+ * The three products of a linear layer under the power-of-two scale option: op = SNIP_OP_FWD (A = X,
+ * B = W, out = Y), SNIP_OP_DGRAD (A = dY, B = W, out = dX) or SNIP_OP_WGRAD (A = dY, B = X, out = dW).
+ * Quantizes both operands with snip_quantize_mx's rule and the tile kinds of the paper-rule calls
+ * above, then runs snip_gemm_mx.  FP8 / FP4 tags only.  Workspace from snip_linear_mx_workspace.
+ */
+int snip_linear_mx(int op, const void *A, const void *B, void *out, int64_t M, int64_t N, int64_t K,
+                   int fmt_a, int fmt_b, int out_dtype, snip_stats_t *stats_a, snip_stats_t *stats_b,
+                   void *ws, size_t ws_bytes, void *stream);
+int snip_linear_mx_workspace(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b, size_t *bytes_host);
+
 /* ---- statistics (paper Sec. 3.1, Step 1) -------------------------------------------------- */
 
 /*

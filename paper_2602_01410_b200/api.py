@@ -25,7 +25,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
     "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
-    "snip_linear_dgrad", "snip_linear_wgrad", "snip_layer_stats", "snip_layer_stats_workspace",
+    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_layer_stats", "snip_layer_stats_workspace",
     "snip_poll_status",
 )
 
@@ -71,6 +71,8 @@ def _load():
     lib.snip_linear_fwd.argtypes = lin
     lib.snip_linear_dgrad.argtypes = lin
     lib.snip_linear_wgrad.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.snip_linear_mx.argtypes = [i32, vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.snip_linear_mx_workspace.argtypes = [i32, i64, i64, i64, i32, i32, psz]
     lib.snip_layer_stats.argtypes = [ctypes.POINTER(LayerTensors), u32, vp, vp, sz, vp]
     lib.snip_layer_stats_workspace.argtypes = [i64, i64, i64, psz]
     lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -252,6 +254,33 @@ def snip_linear_wgrad(dY, X, fmt_dy, fmt_x, out_dtype=OUT_BF16, accumulate=False
     K = X.shape[1]
     return _linear("snip_linear_wgrad", dY, X, (N, K), M, N, K, fmt_dy, fmt_x, out_dtype, OP_WGRAD, out, ws,
                    want_stats, extra=(int(accumulate),))
+
+
+def snip_linear_mx_workspace(op, M, N, K, fmt_a, fmt_b):
+    w = ctypes.c_size_t()
+    _check("snip_linear_mx_workspace", _lib.snip_linear_mx_workspace(op, M, N, K, fmt_a, fmt_b, ctypes.byref(w)))
+    return w.value
+
+
+def snip_linear_mx(op, A, B, fmt_a, fmt_b, out_dtype=OUT_BF16, *, out=None, ws=None, want_stats=False):
+    """Power-of-two scale option.  op FWD: (X, W) -> Y; DGRAD: (dY, W) -> dX; WGRAD: (dY, X) -> dW."""
+    if op == OP_FWD:
+        (M, K), N = A.shape, B.shape[0]
+        shape = (M, N)
+    elif op == OP_DGRAD:
+        (M, N), K = A.shape, B.shape[1]
+        shape = (M, K)
+    else:
+        (M, N), K = A.shape, B.shape[1]
+        shape = (N, K)
+    out = _out(shape, out_dtype, A.device, out)
+    if ws is None:
+        ws = torch.zeros(snip_linear_mx_workspace(op, M, N, K, fmt_a, fmt_b), dtype=torch.uint8, device=A.device)
+    sa = torch.empty(32, dtype=torch.uint8, device=A.device) if want_stats else None
+    sb = torch.empty(32, dtype=torch.uint8, device=A.device) if want_stats else None
+    _check("snip_linear_mx", _lib.snip_linear_mx(op, _p(A), _p(B), _p(out), M, N, K, fmt_a, fmt_b, out_dtype, _p(sa), _p(sb), _p(ws),
+                                                 ws.numel(), _stream()))
+    return out, sa, sb
 
 
 def snip_layer_stats_workspace(M, N, K):

@@ -11,6 +11,10 @@ int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
 int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
               int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
               int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st);
+int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf,
+                     void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st);
+int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, const void *sfa, const void *sfb, int64_t Mo, int64_t No,
+                 int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st);
 int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st);
 size_t gemm_ws_bytes();
 
@@ -72,7 +76,9 @@ LinearPlan plan_for(int op, int64_t M, int64_t N, int64_t K)
     return p;
 }
 
-size_t linear_ws_bytes(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b)
+size_t sf_bytes(int64_t rows, int64_t cols) { return (size_t)(ceil_div(rows, 128) * ceil_div(cols, 128)) * 512; }
+
+size_t linear_ws_bytes(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b, bool mx = false)
 {
     const LinearPlan p = plan_for(op, M, N, K);
     Carve c(nullptr, 0);
@@ -82,17 +88,19 @@ size_t linear_ws_bytes(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int f
     if (need_b) { c.take(code_bytes(fmt_b, p.rows_b, p.cols_b)); c.take(scale_bytes(p.block_b, p.rows_b, p.cols_b)); }
     c.take(stats_bytes(p.rows_a, p.cols_a));
     c.take(stats_bytes(p.rows_b, p.cols_b));
+    if (mx) { c.take(sf_bytes(p.rows_a, p.cols_a)); c.take(sf_bytes(p.rows_b, p.cols_b)); }
     return c.off;
 }
 
 int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b, int out_dtype,
-                int accumulate, snip_stats_t *stats_a, snip_stats_t *stats_b, void *ws, size_t ws_bytes, cudaStream_t st)
+                int accumulate, snip_stats_t *stats_a, snip_stats_t *stats_b, void *ws, size_t ws_bytes, cudaStream_t st, bool mx = false)
 {
+    if (mx && (fmt_a == SNIP_FMT_BF16 || fmt_b == SNIP_FMT_BF16 || accumulate)) return SNIP_ERR_UNSUPPORTED;
     if (!A || !B || !out) return SNIP_ERR_ARG;
     if (!valid_fmt(fmt_a) || !valid_fmt(fmt_b)) return SNIP_ERR_ARG;
     if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
     if ((fmt_a == SNIP_FMT_BF16) != (fmt_b == SNIP_FMT_BF16)) return SNIP_ERR_UNSUPPORTED;
-    if (!ws || ws_bytes < linear_ws_bytes(op, M, N, K, fmt_a, fmt_b)) return SNIP_ERR_WORKSPACE;
+    if (!ws || ws_bytes < linear_ws_bytes(op, M, N, K, fmt_a, fmt_b, mx)) return SNIP_ERR_WORKSPACE;
     if (!aligned16(ws)) return SNIP_ERR_ALIGN;
     const LinearPlan p = plan_for(op, M, N, K);
     Carve c(ws, ws_bytes);
@@ -105,17 +113,20 @@ int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int6
     if (need_b) { codes_b = c.take(code_bytes(fmt_b, p.rows_b, p.cols_b)); scales_b = static_cast<float *>(c.take(scale_bytes(p.block_b, p.rows_b, p.cols_b))); }
     const size_t sws_a_bytes = stats_bytes(p.rows_a, p.cols_a), sws_b_bytes = stats_bytes(p.rows_b, p.cols_b);
     void *sws_a = c.take(sws_a_bytes), *sws_b = c.take(sws_b_bytes);
+    void *sf_a = nullptr, *sf_b = nullptr;
+    if (mx) { sf_a = c.take(sf_bytes(p.rows_a, p.cols_a)); sf_b = c.take(sf_bytes(p.rows_b, p.cols_b)); }
 
     int rc;
     const void *ga = A, *gb = B;
     if (q) {
-        rc = quantize_impl(A, p.rows_a, p.cols_a, p.cols_a, fmt_a, p.block_a, (p.tr_a ? SNIP_Q_TRANSPOSED : 0u) | (stats_a ? SNIP_Q_STATS : 0u),
-                           codes_a, scales_a, stats_a, nullptr, sws_a, sws_a_bytes, st);
+        rc = quantize_impl_ex(A, p.rows_a, p.cols_a, p.cols_a, fmt_a, p.block_a, (p.tr_a ? SNIP_Q_TRANSPOSED : 0u) | (stats_a ? SNIP_Q_STATS : 0u),
+                              mx ? 1 : 0, sf_a, codes_a, scales_a, stats_a, nullptr, sws_a, sws_a_bytes, st);
         if (rc) return rc;
-        rc = quantize_impl(B, p.rows_b, p.cols_b, p.cols_b, fmt_b, p.block_b, (p.tr_b ? SNIP_Q_TRANSPOSED : 0u) | (stats_b ? SNIP_Q_STATS : 0u),
-                           codes_b, scales_b, stats_b, nullptr, sws_b, sws_b_bytes, st);
+        rc = quantize_impl_ex(B, p.rows_b, p.cols_b, p.cols_b, fmt_b, p.block_b, (p.tr_b ? SNIP_Q_TRANSPOSED : 0u) | (stats_b ? SNIP_Q_STATS : 0u),
+                              mx ? 1 : 0, sf_b, codes_b, scales_b, stats_b, nullptr, sws_b, sws_b_bytes, st);
         if (rc) return rc;
         ga = codes_a; gb = codes_b;
+        if (mx) return gemm_mx_impl(fmt_a, fmt_b, ga, gb, sf_a, sf_b, p.Mo, p.No, p.Kc, out, out_dtype, gws, gemm_ws_bytes(), st);
     } else {
         // BF16 tag: identity quantization; only operands whose contraction index is not contiguous are copied
         if (p.tr_a) { rc = transpose_bf16(A, codes_a, p.rows_a, p.cols_a, st); if (rc) return rc; ga = codes_a; }
@@ -164,6 +175,23 @@ extern "C" int snip_linear_wgrad(const void *dY, const void *X, void *dW, int64_
 {
     return snip::linear_impl(SNIP_OP_WGRAD, dY, X, dW, M, N, K, fmt_dy, fmt_x, out_dtype, accumulate, stats_dy, stats_x, ws, ws_bytes,
                              static_cast<cudaStream_t>(stream));
+}
+
+// Power-of-two scale option of the three calls above in one entry point (op selects the product).
+extern "C" int snip_linear_mx(int op, const void *A, const void *B, void *out, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b,
+                              int out_dtype, snip_stats_t *stats_a, snip_stats_t *stats_b, void *ws, size_t ws_bytes, void *stream)
+{
+    if (op < SNIP_OP_FWD || op > SNIP_OP_WGRAD) return SNIP_ERR_ARG;
+    return snip::linear_impl(op, A, B, out, M, N, K, fmt_a, fmt_b, out_dtype, 0, stats_a, stats_b, ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
+}
+
+extern "C" int snip_linear_mx_workspace(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b, size_t *bytes)
+{
+    using namespace snip;
+    if (!bytes || op < SNIP_OP_FWD || op > SNIP_OP_WGRAD || !valid_fmt(fmt_a) || !valid_fmt(fmt_b)) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    *bytes = linear_ws_bytes(op, M, N, K, fmt_a, fmt_b, true);
+    return SNIP_OK;
 }
 
 // ---- layer statistics ---------------------------------------------------------------------

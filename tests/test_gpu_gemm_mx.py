@@ -67,3 +67,36 @@ def test_same_operands_through_the_promotion_gemm():
     y2 = api.snip_gemm_mx(api.OP_FWD, a, fx, b, fw, (M, N), api.OUT_FP32)
     ref = orc.linear_fwd(x, w, FP8, FP8, True)[0]
     assert rel_fro(y1.cpu().numpy(), ref) <= 1e-5 and rel_fro(y2.cpu().numpy(), ref) <= 1e-5
+
+
+@pytest.mark.parametrize("fmt", [FP8, FP4])
+def test_linear_mx_entry_point_with_stats(fmt):
+    from paper_2602_01410_b200 import api
+    M, K, N = 384, 640, 448
+    rng = np.random.default_rng(11)
+    x, w, dy = wl.make_x(rng, M, K), wl.make_w(rng, N, K), wl.make_dy(rng, M, N)
+    X, W, DY = to_dev(x), to_dev(w), to_dev(dy)
+    y, sx, sw = api.snip_linear_mx(api.OP_FWD, X, W, fmt, fmt, api.OUT_FP32, want_stats=True)
+    dx, _, _ = api.snip_linear_mx(api.OP_DGRAD, DY, W, fmt, fmt, api.OUT_FP32)
+    dw, _, _ = api.snip_linear_mx(api.OP_WGRAD, DY, X, fmt, fmt, api.OUT_FP32)
+    torch.cuda.synchronize()
+    ref, qx, qw = orc.linear_fwd(x, w, fmt, fmt, True)
+    assert rel_fro(y.cpu().numpy(), ref) <= 1e-5
+    assert rel_fro(dx.cpu().numpy(), orc.linear_dgrad(dy, w, fmt, fmt, True)[0]) <= 1e-5
+    assert rel_fro(dw.cpu().numpy(), orc.linear_wgrad(dy, x, fmt, fmt, True)[0]) <= 1e-5
+    assert api.stats_to_host(sx)["sumsq_err"] == pytest.approx(qx.sumsq_err, rel=1e-4)
+    assert api.stats_to_host(sw)["sumsq_err"] == pytest.approx(qw.sumsq_err, rel=1e-4)
+
+
+def test_7b_qkv_sampled_rows_hardware_scaled():
+    from paper_2602_01410_b200 import api
+    cfg = wl.CONFIGS[3]
+    x, w, dy = wl.linear_inputs(cfg, 0, 0)
+    X, W = to_dev(x), to_dev(w)
+    y, _, _ = api.snip_linear_mx(api.OP_FWD, X, W, FP4, FP4, api.OUT_BF16)
+    torch.cuda.synchronize()
+    rows = np.array([0, 17, 4095, 8191, 16383])
+    qx = orc.quantize(np.ascontiguousarray(x[rows]), FP4, orc.BLOCK_ROW, True)
+    qw = orc.quantize(w, FP4, orc.BLOCK_BLK, True)
+    ref16 = orc.bf16_to_float(orc.round_to_bf16(orc.gemm_fwd(qx.xhat, qw.xhat)))
+    assert rel_fro(bf16_out_to_f64(y[torch.from_numpy(rows).cuda()]), ref16) <= 1e-3
