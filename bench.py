@@ -325,6 +325,8 @@ def run_profile_case(name):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     parts = name.split("_")
+    if name.startswith("layer_stats"):
+        return run_layer_stats_case(api, torch, device, parts[2] if len(parts) > 2 else "x")
     mx = parts[1].startswith("mx")
     fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4, "mxfp8": FMT_FP8, "mxfp4": FMT_FP4}[parts[1]]
     if parts[0] == "quantize":
@@ -343,6 +345,32 @@ def run_profile_case(name):
             raise SystemExit("bf16 GEMM cases run through snip_linear_*; use fp8/fp4 here")
         fl, times = kt.gemm(fmt, op, 0, iters=3, warmup=1, mx=mx)
         print(f"{name}: {fl / (min(times) * 1e-3) / 1e12:.0f} TFLOP/s best of {len(times)}")
+
+
+def run_layer_stats_case(api, torch, device, which, rows=16384, cols=4096, copies=4, iters=5):
+    """snip_layer_stats on one 7B-sized tensor (x: all four options of an activation; w: both options of a
+    weight; plain: norm only), rotating over `copies` buffers so that L2 cannot serve the reads."""
+    xs = [torch.randn(rows, cols, device=device, dtype=torch.bfloat16) for _ in range(copies)]
+    ws = torch.empty(api.snip_layer_stats_workspace(rows, cols, cols), dtype=torch.uint8, device=device)
+    out = torch.zeros(24, dtype=torch.float64, device=device)
+    times = []
+    for i in range(iters + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        x = xs[i % copies]
+        e0.record()
+        if which == "x":
+            api.snip_layer_stats(X=x, M=rows, N=cols, K=cols, out=out, ws=ws)
+        elif which == "w":
+            api.snip_layer_stats(dX=None, W=x, M=cols, N=rows, K=cols, out=out, ws=ws)
+        else:
+            api.snip_layer_stats(dX=x, M=rows, N=cols, K=cols, out=out, ws=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            times.append(e0.elapsed_time(e1))
+    by = 2.0 * rows * cols
+    print(f"layer_stats_{which}: {min(times) * 1e3:.1f} us best of {len(times)} (memset + kernel + reduction), "
+          f"{by / (min(times) * 1e-3) / 1e9:.0f} GB/s of tensor read")
 
 
 def run_reference(args):
@@ -381,7 +409,7 @@ def main():
     ap.add_argument("--no-kernel-legs", action="store_true")
     ap.add_argument("--profile-case", default=None,
                     help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t> "
-                         "or gemm_<bf16|fp8|fp4>_<fwd|dgrad|wgrad>[_MxNxK]")
+                         "or gemm_<fp8|fp4|mxfp8|mxfp4>_<fwd|dgrad|wgrad>[_MxNxK] or layer_stats_<x|w|plain>")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

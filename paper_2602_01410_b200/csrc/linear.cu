@@ -1,7 +1,6 @@
 // The three GEMMs of one linear layer under a precision choice (paper Fig. 5): quantize the two
 // operands with the tile kind their contraction calls for, then run the block-scaled GEMM.
-// Also snip_layer_stats (Sec. 3.1, Step 1).  Host-side composition only; all arithmetic is in
-// the kernels of quantize.cu and gemm.cu.
+// Host-side composition only; all arithmetic is in the kernels of quantize.cu, gemm.cu and gemm_mx.cu.
 #include "common.cuh"
 
 namespace snip {
@@ -191,77 +190,5 @@ extern "C" int snip_linear_mx_workspace(int op, int64_t M, int64_t N, int64_t K,
     if (!bytes || op < SNIP_OP_FWD || op > SNIP_OP_WGRAD || !valid_fmt(fmt_a) || !valid_fmt(fmt_b)) return SNIP_ERR_ARG;
     if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
     *bytes = linear_ws_bytes(op, M, N, K, fmt_a, fmt_b, true);
-    return SNIP_OK;
-}
-
-// ---- layer statistics ---------------------------------------------------------------------
-
-extern "C" int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes)
-{
-    using namespace snip;
-    if (!ws_bytes) return SNIP_ERR_ARG;
-    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
-    size_t w = stats_bytes(M, K);
-    size_t t = stats_bytes(N, K); if (t > w) w = t;
-    t = stats_bytes(M, N); if (t > w) w = t;
-    *ws_bytes = align_up(w, 256) + 256;  // + one snip_stats_t slot
-    return SNIP_OK;
-}
-
-namespace snip {
-namespace {
-__global__ void gather_stat_kernel(const snip_stats_t *s, double *dst_x, double *dst_err)
-{
-    if (dst_x) *dst_x = s->sumsq_x;
-    if (dst_err) *dst_err = s->sumsq_err;
-}
-}  // namespace
-}  // namespace snip
-
-extern "C" int snip_layer_stats(const snip_layer_tensors_t *t, uint32_t fmt_mask, snip_layer_stats_t *out, void *ws, size_t ws_bytes,
-                                void *stream)
-{
-    using namespace snip;
-    if (!t || !out || !ws) return SNIP_ERR_ARG;
-    size_t need = 0;
-    int rc = snip_layer_stats_workspace(t->M, t->N, t->K, &need);
-    if (rc) return rc;
-    if (ws_bytes < need) return SNIP_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    SNIP_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(snip_layer_stats_t), st));
-    snip_stats_t *slot = reinterpret_cast<snip_stats_t *>(static_cast<uint8_t *>(ws));
-    void *sws = static_cast<uint8_t *>(ws) + 256;
-    const size_t sws_bytes = ws_bytes - 256;
-    const int64_t M = t->M, N = t->N, K = t->K;
-    struct T { const void *p; int64_t r, c; int qidx; } tens[6] = {
-        {t->X, M, K, 0}, {t->W, N, K, 1}, {t->Y, M, N, -1}, {t->dY, M, N, 2}, {t->dX, M, K, -1}, {t->dW, N, K, -1}};
-    for (int i = 0; i < 6; ++i) {
-        if (!tens[i].p) continue;
-        bool have_plain = false;
-        if (tens[i].qidx >= 0) {
-            const int blocks_xdy[2] = {SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_COL_128x1};
-            const int blocks_w[1] = {SNIP_BLOCK_BLK_128x128};
-            const int *blocks = tens[i].qidx == 1 ? blocks_w : blocks_xdy;
-            const int nb = tens[i].qidx == 1 ? 1 : 2;
-            for (int f = 0; f < 2; ++f) {
-                if (!(fmt_mask & (2u << f))) continue;
-                for (int b = 0; b < nb; ++b) {
-                    rc = quantize_impl(tens[i].p, tens[i].r, tens[i].c, tens[i].c, f == 0 ? SNIP_FMT_FP8_E4M3 : SNIP_FMT_FP4_E2M1, blocks[b],
-                                       SNIP_Q_STATS | SNIP_Q_NO_CODES, nullptr, nullptr, slot, nullptr, sws, sws_bytes, st);
-                    if (rc) return rc;
-                    gather_stat_kernel<<<1, 1, 0, st>>>(slot, have_plain ? nullptr : &out->sumsq[i], &out->sumsq_err[tens[i].qidx][f][blocks[b]]);
-                    SNIP_CUDA_TRY(cudaGetLastError());
-                    have_plain = true;
-                }
-            }
-        }
-        if (!have_plain) {
-            rc = quantize_impl(tens[i].p, tens[i].r, tens[i].c, tens[i].c, SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, SNIP_Q_STATS, nullptr,
-                               nullptr, slot, nullptr, sws, sws_bytes, st);
-            if (rc) return rc;
-            gather_stat_kernel<<<1, 1, 0, st>>>(slot, &out->sumsq[i], nullptr);
-            SNIP_CUDA_TRY(cudaGetLastError());
-        }
-    }
     return SNIP_OK;
 }

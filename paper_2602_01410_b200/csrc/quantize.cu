@@ -14,6 +14,7 @@
 #include <float.h>
 
 #include "common.cuh"
+#include "quant_device.cuh"
 
 namespace snip {
 
@@ -39,120 +40,6 @@ struct QuantArgs {
     int pow2;             // 1: power-of-two scale rule (largest 2^e with amax * 2^e <= FPX_MAX)
     uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
 };
-
-__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
-__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
-
-__device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t v)
-{
-    // packed bf16 max of |v| against a non-negative accumulator
-    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&acc);
-    uint32_t av = v & 0x7FFF7FFFu;
-    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&av);
-    __nv_bfloat162 m = __hmax2(a, b);
-    return *reinterpret_cast<uint32_t *>(&m);
-}
-
-__device__ __forceinline__ uint32_t max2(uint32_t x, uint32_t y)
-{
-    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&x);
-    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162 *>(&y);
-    __nv_bfloat162 m = __hmax2(a, b);
-    return *reinterpret_cast<uint32_t *>(&m);
-}
-
-// Scale of a tile from its amax.  Paper's rule: IEEE binary32 quotient FPX_MAX / amax, 1 for an empty
-// tile, clamped to FLT_MAX.  Power-of-two option: the largest 2^e with amax * 2^e <= FPX_MAX, worked out
-// on the exponent and significand bits (no division), e clamped to [-126, 127].
-template <int FMT>
-__device__ __forceinline__ float tile_scale(float amax, int pow2)
-{
-    constexpr float kMax = (FMT == SNIP_FMT_FP8_E4M3) ? 448.0f : 6.0f;
-    if (amax == 0.0f) return 1.0f;
-    if (pow2) {
-        constexpr int kMaxExp = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 2;                       // FPX_MAX = m_f * 2^kMaxExp
-        constexpr uint32_t kMaxMant = (FMT == SNIP_FMT_FP8_E4M3) ? 0x600000u : 0x400000u;  // m_f = 1.75 / 1.5
-        const uint32_t b = __float_as_uint(amax);
-        const int ef = (int)(b >> 23);                 // biased exponent; 0 for a (bf16) subnormal amax
-        if (ef == 0) return __uint_as_float(254u << 23);   // amax < 2^-126: the clamp e = 127 applies
-        int e = kMaxExp - (ef - 127) - (((b & 0x7FFFFFu) > kMaxMant) ? 1 : 0);
-        e = max(-126, min(127, e));
-        return __uint_as_float((uint32_t)(e + 127) << 23);
-    }
-    float s = __fdiv_rn(kMax, amax);
-    return fminf(s, FLT_MAX);  // +inf -> FLT_MAX
-}
-// -1/S for the error term.  Paper's rule: amax/FPX_MAX equals 1/S to within one rounding, which the
-// statistics (1e-4) do not see; power-of-two rule: exact.  For an empty tile the value is irrelevant.
-template <int FMT>
-__device__ __forceinline__ float neg_inv_scale(float amax, float s, int pow2)
-{
-    constexpr float kMax = (FMT == SNIP_FMT_FP8_E4M3) ? 448.0f : 6.0f;
-    return pow2 ? -__fdiv_rn(1.0f, s) : -amax * (1.0f / kMax);
-}
-// UE8M0 byte of 1/S for a power-of-two S, replicated into the four bytes of a word
-__device__ __forceinline__ uint32_t sf_word(float s) { return (254u - (__float_as_uint(s) >> 23)) * 0x01010101u; }
-
-// Two binary32 values -> two codes.  `lo` lands in the low byte / nibble.
-__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
-{
-    uint16_t r;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
-{
-    uint16_t r;
-    asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; mov.b16 %0, {t, 0}; }"
-        : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-// Two codes -> two binary32 values (exact).
-__device__ __forceinline__ float2 dec_e4m3x2(uint32_t c)
-{
-    uint32_t h2;
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)c));
-    return __half22float2(*reinterpret_cast<__half2 *>(&h2));
-}
-__device__ __forceinline__ float2 dec_e2m1x2(uint32_t c)
-{
-    uint32_t h2;
-    asm("{ .reg .b8 t, u; mov.b16 {t, u}, %1; cvt.rn.f16x2.e2m1x2 %0, t; }"
-        : "=r"(h2) : "h"((uint16_t)c));
-    return __half22float2(*reinterpret_cast<__half2 *>(&h2));
-}
-
-// Quantize 8 consecutive elements (one 128-bit load).  s2[i] / ninv2[i]: scale and negated
-// reciprocal scale of elements (2i, 2i+1).  Returns the packed codes (FP8: 8 bytes in out[0..1];
-// FP4: 4 bytes in out[0]) and adds to the statistics.  The products x*S are IEEE binary32
-// products (packed mul.rn.f32x2), exactly what the scalar definition asks for.
-template <int FMT, bool STATS>
-__device__ __forceinline__ void quant8(const uint4 &v, const float2 (&s2)[4], const float2 (&ninv2)[4],
-                                       uint32_t out[2], float2 &sx2, float2 &se2)
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t c[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float2 x = make_float2(bf16lo(w[i]), bf16hi(w[i]));
-        const float2 t = __fmul2_rn(x, s2[i]);
-        if (FMT == SNIP_FMT_FP8_E4M3) c[i] = cvt_e4m3x2(t.x, t.y);
-        else c[i] = cvt_e2m1x2(t.x, t.y);
-        if (STATS) {
-            const float2 d = (FMT == SNIP_FMT_FP8_E4M3) ? dec_e4m3x2(c[i]) : dec_e2m1x2(c[i]);
-            const float2 e = __ffma2_rn(d, ninv2[i], x);  // x - value(code)/S
-            sx2 = __ffma2_rn(x, x, sx2);
-            se2 = __ffma2_rn(e, e, se2);
-        }
-    }
-    if (FMT == SNIP_FMT_FP8_E4M3) {
-        out[0] = c[0] | (c[1] << 16);
-        out[1] = c[2] | (c[3] << 16);
-    } else {
-        out[0] = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
-        out[1] = 0;
-    }
-}
 
 // FMT: target format (BF16 = statistics only).  BLOCK: tile kind.  TRANSPOSED: codes stored as
 // the transpose.  CODES: write codes and scales.  STATS: accumulate sums.  ROWSTATS: per-row sums.
