@@ -2,9 +2,11 @@
 """Benchmark of the SNIP mixed-precision linear hot path on B200.
 
 A step = one transformer block of the Llama-7B-shaped workload (tokens 16384; fused QKV, O,
-gate, up, down): for every linear the forward, input-gradient and weight-gradient GEMMs, each
-preceded by the quantization of its two operands with fused error-norm statistics, run once with
-every GEMM in FP4 E2M1 and once with every GEMM in FP8 E4M3.
+gate, up, down): for every linear the quantization of X, W and dY (each read once, both quantized
+copies written: the tile kind of each of the two GEMMs that consume the tensor, with fused error-norm
+statistics per copy) and the forward, input-gradient and weight-gradient GEMMs, run once with every
+GEMM in FP4 E2M1 and once with every GEMM in FP8 E4M3.  `--quantizer single` runs one quantizer call
+per GEMM operand instead (six reads per linear).
 
 Prints ONE JSON line (rank 0).  `value` is GEMM TFLOP/s (2*M*N*K per GEMM) over the whole step,
 quantizers and statistics included, with inputs resident in HBM.  `roofline` describes the
@@ -131,8 +133,8 @@ def make_device_inputs(cfg, torch, device, seed):
 class Step:
     """Device buffers and the call sequence of one step."""
 
-    def __init__(self, api, torch, cfg, device, formats):
-        self.api, self.torch, self.cfg, self.formats = api, torch, cfg, formats
+    def __init__(self, api, torch, cfg, device, formats, dual=True):
+        self.api, self.torch, self.cfg, self.formats, self.dual = api, torch, cfg, formats, dual
         self.inputs = make_device_inputs(cfg, torch, device, 260201410)
         M = cfg.M
         self.out = []
@@ -144,16 +146,31 @@ class Step:
             for op in (api.OP_FWD, api.OP_DGRAD, api.OP_WGRAD):
                 for f in formats:
                     ws_bytes = max(ws_bytes, api.snip_workspace_size(op, M, L.N, L.K, f, f)[1])
+            for f in formats:
+                for pow2 in (False, True):
+                    ws_bytes = max(ws_bytes, api.snip_linear_fwd_bwd_workspace(M, L.N, L.K, f, f, f, pow2))
         self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
         n_gemm = len(cfg.linears) * 3 * len(formats)
         self.stats = torch.zeros(n_gemm * 2, 32, dtype=torch.uint8, device=device)  # one 16-byte-aligned snip_stats_t per row
+        self.stats6 = torch.zeros(len(cfg.linears) * len(formats), 6 * 24, dtype=torch.uint8, device=device)
         self.flops = sum(2.0 * M * L.N * L.K * 3 for L in cfg.linears) * len(formats)
-        self.launches_per_step = n_gemm * 5  # 2 quantizers + 2 statistics reductions + 1 GEMM
+        # per GEMM: dual = 1 quantizer + 1 statistics reduction + 1 GEMM; single = 2 + 2 + 1
+        self.launches_per_step = n_gemm * (3 if dual else 5)
 
     # -- the step through the snip_linear_* entry points (what a user calls) -------------
-    def run_linear_calls(self):
+    def run_linear_calls(self, mx=False):
         api = self.api
         i = 0
+        if self.dual:
+            lib, p, st = api._lib, api._p, api._stream()
+            for f in self.formats:
+                for (x, w, dy), (y, dx, dw) in zip(self.inputs, self.out):
+                    M, K = x.shape
+                    N = w.shape[0]
+                    api._check("snip_linear_fwd_bwd", lib.snip_linear_fwd_bwd(p(x), p(w), p(dy), p(y), p(dx), p(dw), M, N, K, f, f, f, api.OUT_BF16,
+                                                                              int(mx), p(self.stats6[i]), p(self.ws), self.ws.numel(), st))
+                    i += 1
+            return
         for f in self.formats:
             for (x, w, dy), (y, dx, dw) in zip(self.inputs, self.out):
                 M, K = x.shape
@@ -178,10 +195,11 @@ class Step:
                     a, b, w = api.snip_quantize_sizes(r, c, FMT_FP8, blk, api.Q_STATS)
                     cb, sb, wb = max(cb, a), max(sb, b), max(wb, w)
         dev = self.ws.device
-        self.codes = [torch.empty(cb, dtype=torch.uint8, device=dev) for _ in range(2)]
-        self.scales = [torch.empty(sb // 4, dtype=torch.float32, device=dev) for _ in range(2)]
-        self.qws = torch.empty(wb, dtype=torch.uint8, device=dev)
-        self.sf = [torch.empty(cb // 32 + 4096, dtype=torch.uint8, device=dev) for _ in range(2)]   # UE8M0 atoms (power-of-two option)
+        nbuf = 6 if self.dual else 2
+        self.codes = [torch.empty(cb, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
+        self.scales = [torch.empty(sb // 4, dtype=torch.float32, device=dev) for _ in range(nbuf)]
+        self.qws = torch.empty(2 * wb, dtype=torch.uint8, device=dev)
+        self.sf = [torch.empty(cb // 32 + 4096, dtype=torch.uint8, device=dev) for _ in range(nbuf)]   # UE8M0 atoms (power-of-two option)
         self.gws = torch.zeros(1024, dtype=torch.uint8, device=dev)
 
     def run_decomposed(self, events=None, mx=False):
@@ -201,14 +219,20 @@ class Step:
                 api._check("snip_quantize", lib.snip_quantize(p(x), r, c, c, fmt, block, flags | api.Q_STATS, p(self.codes[slot]), p(self.scales[slot]),
                                                               p(stats), None, p(self.qws), self.qws.numel(), st))
 
-        def gemm(op, fmt, ra, ca, blka, ta, rb, cb_, blkb, tb, out, flops):
-            a = api.make_qtensor(self.codes[0], self.scales[0], ra, ca, fmt, blka, ta)
-            b = api.make_qtensor(self.codes[1], self.scales[1], rb, cb_, fmt, blkb, tb)
+        def dual(x, fmt, kind, slot, stats_row):
+            r, c = x.shape
+            outs = [api.QOut(fmt, 0, p(self.codes[slot + j]), p(self.scales[slot + j]), p(self.sf[slot + j]) if mx else None,
+                             p(stats_row[24 * j:24 * j + 24])) for j in range(2)]
+            api._check("snip_quantize_dual", lib.snip_quantize_dual(p(x), r, c, c, kind, int(mx), outs[0], outs[1], p(self.qws), self.qws.numel(), st))
+
+        def gemm(op, fmt, ra, ca, blka, ta, rb, cb_, blkb, tb, out, flops, sa=0, sb_=1):
+            a = api.make_qtensor(self.codes[sa], self.scales[sa], ra, ca, fmt, blka, ta)
+            b = api.make_qtensor(self.codes[sb_], self.scales[sb_], rb, cb_, fmt, blkb, tb)
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
             if mx:
-                api._check("snip_gemm_mx", lib.snip_gemm_mx(op, a, p(self.sf[0]), b, p(self.sf[1]), p(out), api.OUT_BF16, p(self.gws), self.gws.numel(), st))
+                api._check("snip_gemm_mx", lib.snip_gemm_mx(op, a, p(self.sf[sa]), b, p(self.sf[sb_]), p(out), api.OUT_BF16, p(self.gws), self.gws.numel(), st))
             else:
                 api._check("snip_gemm_quantized", lib.snip_gemm_quantized(op, a, b, p(out), api.OUT_BF16, 0, p(self.gws), self.gws.numel(), st))
             if events is not None:
@@ -220,6 +244,16 @@ class Step:
                 M, K = x.shape
                 N = w.shape[0]
                 fl = 2.0 * M * N * K
+                if self.dual:
+                    # slots: 0 X/ROW, 1 X/COL^T, 2 W/BLK, 3 W/BLK^T, 4 dY/ROW, 5 dY/COL^T
+                    srow = self.stats6[i // 3].view(-1)
+                    i += 3
+                    dual(x, f, api.DUAL_ROW_COLT, 0, srow[0:48]); dual(w, f, api.DUAL_BLK_BLKT, 2, srow[48:96])
+                    gemm(api.OP_FWD, f, M, K, api.BLOCK_ROW, 0, N, K, api.BLOCK_BLK, 0, y, fl, 0, 2)
+                    dual(dy, f, api.DUAL_ROW_COLT, 4, srow[96:144])
+                    gemm(api.OP_DGRAD, f, M, N, api.BLOCK_ROW, 0, N, K, api.BLOCK_BLK, 1, dx, fl, 4, 3)
+                    gemm(api.OP_WGRAD, f, M, N, api.BLOCK_COL, 1, M, K, api.BLOCK_COL, 1, dw, fl, 5, 1)
+                    continue
                 quant(x, f, api.BLOCK_ROW, 0, 0, self.stats[2 * i]); quant(w, f, api.BLOCK_BLK, 0, 1, self.stats[2 * i + 1]); i += 1
                 gemm(api.OP_FWD, f, M, K, api.BLOCK_ROW, 0, N, K, api.BLOCK_BLK, 0, y, fl)
                 quant(dy, f, api.BLOCK_ROW, 0, 0, self.stats[2 * i]); quant(w, f, api.BLOCK_BLK, T, 1, self.stats[2 * i + 1]); i += 1
@@ -299,6 +333,28 @@ class KernelTimer:
         return bytes_per_elt * rows * cols, times
 
 
+    def quantizer_dual(self, fmt, kind, rows, cols, iters=20, warmup=3):
+        """snip_quantize_dual with statistics, timed like quantizer(); bytes = one read + two outputs."""
+        api, torch = self.api, self.torch
+        g = torch.Generator(device=self.device); g.manual_seed(2)
+        xs = [torch.randn(rows, cols, generator=g, device=self.device, dtype=torch.float32).to(torch.bfloat16) for _ in range(3)]
+        bufs = api.snip_quantize_dual(xs[0], kind, fmt, fmt)
+        ws = torch.empty(api.snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=self.device)
+        times = []
+        batch = 6
+        for i in range(warmup + iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for j in range(batch):
+                api.snip_quantize_dual(xs[j % 3], kind, fmt, fmt, bufs=bufs, ws=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= warmup:
+                times.append(e0.elapsed_time(e1) / batch)
+        bytes_per_elt = 2.0 + 2.0 * ((1.0 if fmt == FMT_FP8 else 0.5) + 4.0 / 128.0)
+        return bytes_per_elt * rows * cols, times
+
+
 def cpu_baseline_sample(cfg, tokens=4096):
     """The CPU oracle, as it stands, on a bounded sample: `tokens` rows of the O projection
     (K -> K) through quantize + fwd + dgrad + wgrad in FP8.  Returns (TFLOP/s, cores, text)."""
@@ -329,7 +385,12 @@ def run_profile_case(name):
         return run_layer_stats_case(api, torch, device, parts[2] if len(parts) > 2 else "x")
     mx = parts[1].startswith("mx")
     fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4, "mxfp8": FMT_FP8, "mxfp4": FMT_FP4}[parts[1]]
-    if parts[0] == "quantize":
+    if parts[0] == "quantize" and parts[2] == "dual":
+        kt = KernelTimer(api, torch, wl.CONFIGS[3], device)
+        kind = api.DUAL_BLK_BLKT if parts[-1] == "blk" else api.DUAL_ROW_COLT
+        by, times = kt.quantizer_dual(fmt, kind, 16384, 4096, iters=3, warmup=1)
+        print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
+    elif parts[0] == "quantize":
         kind = "_".join(parts[2:])
         block, tr = {"row": (api.BLOCK_ROW, False), "col_t": (api.BLOCK_COL, True), "blk_t": (api.BLOCK_BLK, True),
                      "blk": (api.BLOCK_BLK, False), "col": (api.BLOCK_COL, False)}[kind]
@@ -405,10 +466,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="snip")
     ap.add_argument("--workload", default="7b", choices=sorted(WORKLOADS))
+    ap.add_argument("--quantizer", default="dual", choices=("dual", "single"),
+                    help="dual: X, W, dY each read once, both quantized copies written; single: one quantizer call per GEMM operand")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-legs", action="store_true")
     ap.add_argument("--profile-case", default=None,
-                    help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t> "
+                    help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t|dual_rowcol|dual_blk> "
                          "or gemm_<fp8|fp4|mxfp8|mxfp4>_<fwd|dgrad|wgrad>[_MxNxK] or layer_stats_<x|w|plain>")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -437,7 +500,7 @@ def main():
 
     cfg = wl.CONFIGS[WORKLOADS[args.workload][0]]
     formats = (FMT_FP4, FMT_FP8)
-    step = Step(api, torch, cfg, device, formats)
+    step = Step(api, torch, cfg, device, formats, dual=(args.quantizer == "dual"))
     peaks = load_peaks()
 
     # ---- timed region: K steps, inputs resident in HBM ------------------------------------------
@@ -497,13 +560,14 @@ def main():
     if rank == 0 or world > 1:
         host = [tuple(t.cpu().pin_memory() for t in trip) for trip in step.inputs]
         h2d = sum(t.numel() * 2 for trip in host for t in trip)
-        stats_host = torch.empty_like(step.stats, device="cpu").pin_memory()
+        stats_dev = step.stats6 if step.dual else step.stats
+        stats_host = torch.empty_like(stats_dev, device="cpu").pin_memory()
         def e2e_step():
             for trip_d, trip_h in zip(step.inputs, host):
                 for d, h in zip(trip_d, trip_h):
                     d.copy_(h, non_blocking=True)
             step.run_linear_calls()
-            stats_host.copy_(step.stats, non_blocking=True)
+            stats_host.copy_(stats_dev, non_blocking=True)
         e2e_step(); barrier()
         n_e2e = max(1, min(args.steps, 3))
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -561,6 +625,10 @@ def main():
                 by, times = kt.quantizer(f, block, tr, cfg.M, 4096)
                 avg = sum(times) / len(times)
                 kernels[f"quantize_{FMT_NAME[f]}_{name}"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
+            for kind, name in ((api.DUAL_ROW_COLT, "row+col_t"), (api.DUAL_BLK_BLKT, "blk+blk_t")):
+                by, times = kt.quantizer_dual(f, kind, cfg.M, 4096)
+                avg = sum(times) / len(times)
+                kernels[f"quantize_dual_{FMT_NAME[f]}_{name}"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -570,7 +638,8 @@ def main():
     line = {"metric": "mixed-precision linear fwd+dgrad+wgrad TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4_e2m1+fp8_e4m3 (fp32 accumulate)", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: one block (qkv,o,gate,up,down) x (fwd,dgrad,wgrad) all-FP4 then all-FP8, tokens {cfg.M}, quantize+stats every GEMM",
+            "config": {"workload": f"{cfg.name}: one block (qkv,o,gate,up,down) x (fwd,dgrad,wgrad) all-FP4 then all-FP8, tokens {cfg.M}, quantize+stats of both operands of every GEMM "
+                                   + ("(X, W, dY read once each, two quantized copies per read)" if step.dual else "(one quantizer call per operand)"),
                        "l2": "inputs larger than L2", "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": step.launches_per_step * args.steps,
             "roofline": roofline, "kernels": kernels, "pow2_option": pow2_option, "cpu_baseline": cpu}

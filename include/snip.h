@@ -107,6 +107,24 @@ typedef struct {
     double sumsq_err[3][2][3];
 } snip_layer_stats_t;
 
+/* One output of snip_quantize_dual: format (FP8 or FP4), destination buffers (device), optional UE8M0
+ * scale-factor atoms (power-of-two rule only, else NULL) and optional statistics (device; give both
+ * outputs' or neither). */
+typedef struct {
+    int32_t fmt;
+    int32_t reserved;
+    void *codes;
+    float *scales;
+    void *sf;
+    snip_stats_t *stats;
+} snip_qout_t;
+
+/* Tile kinds of the two outputs of snip_quantize_dual. */
+typedef enum {
+    SNIP_DUAL_ROW_COLT = 0, /* as stored: 1x128 tiles along the columns; transposed: 128x1 tiles along the rows */
+    SNIP_DUAL_BLK_BLKT = 1  /* 128x128 blocks, as stored and transposed */
+} snip_dual_kind_t;
+
 /* ---- library information ----------------------------------------------------------------- */
 
 /* Version of this ABI as major*10000 + minor*100 + patch.  (No counterpart in the paper.) */
@@ -166,6 +184,25 @@ int snip_quantize(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
  */
 int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,
                           uint32_t flags, void *codes, float *scales, snip_stats_t *stats, void *stream);
+
+/*
+ * Both quantized copies of a tensor from one read.  Every tensor of a linear layer is consumed by
+ * two GEMMs with different contraction indices (paper Fig. 5): X by fwd (tiles along K) and wgrad
+ * (tiles along M), dY by dgrad (along N) and wgrad (along M), W by fwd and dgrad (the 128x128 block
+ * grid serves both, but dgrad wants the transposed storage).  This call produces, from a single pass
+ * over x[rows][ld], exactly what two snip_quantize calls would:
+ *   as_stored:  kind ROW_COLT -> (fmt, SNIP_BLOCK_ROW_1x128, no flags); BLK_BLKT -> (fmt, SNIP_BLOCK_BLK_128x128, no flags)
+ *   transposed: kind ROW_COLT -> (fmt, SNIP_BLOCK_COL_128x1, SNIP_Q_TRANSPOSED); BLK_BLKT -> (fmt, BLK, SNIP_Q_TRANSPOSED)
+ * with independent formats, so codes, scales and statistics are bit-identical to those calls.
+ * pow2_scale != 0 selects the power-of-two rule of snip_quantize_mx (and allows sf != NULL).
+ * Algorithmic bytes per element: 2 + the two outputs' code and scale bytes, instead of 4 + those.
+ * The paper does not prescribe how the copies are produced; it only fixes what they contain (Sec. 2.3).
+ * ws_bytes >= snip_quantize_dual_workspace() when statistics are requested (else ws may be NULL).
+ */
+int snip_quantize_dual_workspace(int64_t rows, int64_t cols, size_t *ws_bytes_host);
+int snip_quantize_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, int kind, int pow2_scale,
+                       const snip_qout_t *as_stored_host, const snip_qout_t *transposed_host,
+                       void *ws, size_t ws_bytes, void *stream);
 
 /*
  * Power-of-two scale option (an added quantization option in the sense of paper Sec. 3.2, which lets
@@ -271,6 +308,27 @@ int snip_linear_mx_workspace(int op, int64_t M, int64_t N, int64_t K, int fmt_a,
 int snip_layer_stats(const snip_layer_tensors_t *t_host, uint32_t fmt_mask,
                      snip_layer_stats_t *out, void *ws, size_t ws_bytes, void *stream);
 int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes_host);
+
+/*
+ * One linear layer, forward and both gradients, under a precision triple (one tag per GEMM, FP8 or FP4;
+ * paper Fig. 5) with every tensor read once: X, W and dY each go through snip_quantize_dual, which
+ * leaves the copy for the second GEMM that consumes the tensor, then Y = X W^T, dX = dY W, dW = dY^T X.
+ *   X:  1x128 tiles, fmt_fwd (fwd)    + 128x1 tiles transposed, fmt_wgrad (wgrad)
+ *   W:  128x128 blocks, fmt_fwd (fwd) + the same blocks transposed, fmt_dgrad (dgrad)
+ *   dY: 1x128 tiles, fmt_dgrad (dgrad) + 128x1 tiles transposed, fmt_wgrad (wgrad)
+ * Results equal those of snip_linear_fwd / _dgrad / _wgrad (pow2_scale = 0) or snip_linear_mx
+ * (pow2_scale != 0) called with the same tags.  stats6 (device, may be NULL): six snip_stats_t in the
+ * order X/1x128, X/128x1, W/fwd format, W/dgrad format, dY/1x128, dY/128x1.  out_dtype applies to all
+ * three outputs.  BF16 tags are not offered here (use the three separate calls).  A training loop that
+ * separates forward and backward in time keeps the quantized copies instead of the bf16 activations;
+ * this entry point runs the two halves back to back.
+ */
+int snip_linear_fwd_bwd_workspace(int64_t M, int64_t N, int64_t K, int fmt_fwd, int fmt_dgrad, int fmt_wgrad,
+                                  int pow2_scale, size_t *ws_bytes_host);
+int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY, void *Y, void *dX, void *dW,
+                        int64_t M, int64_t N, int64_t K, int fmt_fwd, int fmt_dgrad, int fmt_wgrad,
+                        int out_dtype, int pow2_scale, snip_stats_t *stats6, void *ws, size_t ws_bytes,
+                        void *stream);
 
 /* ---- device status ------------------------------------------------------------------------ */
 

@@ -24,8 +24,8 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
-    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_layer_stats", "snip_layer_stats_workspace",
+    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
+    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace",
     "snip_poll_status",
 )
 
@@ -42,6 +42,14 @@ class QTensor(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("rows", ctypes.c_int64),
                 ("cols", ctypes.c_int64), ("fmt", ctypes.c_int32), ("block", ctypes.c_int32),
                 ("transposed", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class QOut(ctypes.Structure):
+    _fields_ = [("fmt", ctypes.c_int32), ("reserved", ctypes.c_int32), ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("sf", ctypes.c_void_p), ("stats", ctypes.c_void_p)]
+
+
+DUAL_ROW_COLT, DUAL_BLK_BLKT = 0, 1
 
 
 class LayerTensors(ctypes.Structure):
@@ -64,6 +72,8 @@ def _load():
     lib.snip_quantize_noalloc.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp]
     lib.snip_quantize_mx_sizes.argtypes = [i64, i64, psz]
     lib.snip_quantize_mx.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
+    lib.snip_quantize_dual_workspace.argtypes = [i64, i64, psz]
+    lib.snip_quantize_dual.argtypes = [vp, i64, i64, i64, i32, i32, ctypes.POINTER(QOut), ctypes.POINTER(QOut), vp, sz, vp]
     lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
     lib.snip_gemm_mx.argtypes = [i32, ctypes.POINTER(QTensor), vp, ctypes.POINTER(QTensor), vp, vp, i32, vp, sz, vp]
@@ -73,6 +83,8 @@ def _load():
     lib.snip_linear_wgrad.argtypes = [vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_mx.argtypes = [i32, vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_mx_workspace.argtypes = [i32, i64, i64, i64, i32, i32, psz]
+    lib.snip_linear_fwd_bwd_workspace.argtypes = [i64, i64, i64, i32, i32, i32, i32, psz]
+    lib.snip_linear_fwd_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp, vp, sz, vp]
     lib.snip_layer_stats.argtypes = [ctypes.POINTER(LayerTensors), u32, vp, vp, sz, vp]
     lib.snip_layer_stats_workspace.argtypes = [i64, i64, i64, psz]
     lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -175,6 +187,41 @@ def snip_quantize_mx(x: torch.Tensor, fmt: int, block: int, flags: int = 0, *, w
     _check("snip_quantize_mx", _lib.snip_quantize_mx(_p(x), rows, cols, x.stride(0), fmt, block, flags, _p(codes), _p(scales), _p(sf),
                                                      _p(stats), _p(ws), 0 if ws is None else ws.numel(), _stream()))
     return codes, scales, sf, stats
+
+
+def snip_quantize_dual_workspace(rows, cols):
+    n = ctypes.c_size_t()
+    _check("snip_quantize_dual_workspace", _lib.snip_quantize_dual_workspace(rows, cols, ctypes.byref(n)))
+    return n.value
+
+
+def snip_quantize_dual(x: torch.Tensor, kind: int, fmt_stored: int, fmt_transposed: int, *, pow2_scale=False, want_stats=True,
+                       want_sf=False, bufs=None, ws=None):
+    """One read, two outputs.  Returns two dicts (as stored, transposed) with codes / scales / sf / stats
+    tensors (sf, stats None unless asked for).  bufs = (dict, dict) reuses buffers of an earlier call."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    dev = x.device
+    blocks = (BLOCK_ROW, BLOCK_COL) if kind == DUAL_ROW_COLT else (BLOCK_BLK, BLOCK_BLK)
+    outs, structs = [], []
+    for i, fmt in enumerate((fmt_stored, fmt_transposed)):
+        if bufs is not None:
+            o = bufs[i]
+        else:
+            cb, sb, _ = snip_quantize_sizes(rows, cols, fmt, blocks[i], Q_TRANSPOSED if i else 0)
+            o = {"codes": torch.empty(cb, dtype=torch.uint8, device=dev), "scales": torch.empty(sb // 4, dtype=torch.float32, device=dev),
+                 "sf": None, "stats": torch.empty(32, dtype=torch.uint8, device=dev) if want_stats else None}
+            if want_sf:
+                n = ctypes.c_size_t()
+                _check("snip_quantize_mx_sizes", _lib.snip_quantize_mx_sizes(rows, cols, ctypes.byref(n)))
+                o["sf"] = torch.empty(n.value, dtype=torch.uint8, device=dev)
+        outs.append(o)
+        structs.append(QOut(fmt, 0, _p(o["codes"]), _p(o["scales"]), _p(o["sf"]), _p(o["stats"])))
+    if ws is None and outs[0]["stats"] is not None:
+        ws = torch.empty(snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=dev)
+    _check("snip_quantize_dual", _lib.snip_quantize_dual(_p(x), rows, cols, x.stride(0), kind, int(pow2_scale), ctypes.byref(structs[0]),
+                                                         ctypes.byref(structs[1]), _p(ws), 0 if ws is None else ws.numel(), _stream()))
+    return outs[0], outs[1]
 
 
 def snip_workspace_size(op, M, N, K, fmt_a, fmt_b):
@@ -281,6 +328,30 @@ def snip_linear_mx(op, A, B, fmt_a, fmt_b, out_dtype=OUT_BF16, *, out=None, ws=N
     _check("snip_linear_mx", _lib.snip_linear_mx(op, _p(A), _p(B), _p(out), M, N, K, fmt_a, fmt_b, out_dtype, _p(sa), _p(sb), _p(ws),
                                                  ws.numel(), _stream()))
     return out, sa, sb
+
+
+def snip_linear_fwd_bwd_workspace(M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad, pow2_scale=False):
+    n = ctypes.c_size_t()
+    _check("snip_linear_fwd_bwd_workspace", _lib.snip_linear_fwd_bwd_workspace(M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad, int(pow2_scale),
+                                                                               ctypes.byref(n)))
+    return n.value
+
+
+def snip_linear_fwd_bwd(x, w, dy, fmt_fwd, fmt_dgrad, fmt_wgrad, out_dtype=OUT_BF16, *, pow2_scale=False, y=None, dx=None, dw=None,
+                        stats=None, ws=None):
+    """Forward and both gradients of one linear layer, each tensor read once.  Returns (y, dx, dw, stats)
+    with stats a uint8 tensor holding six 24-byte snip_stats_t."""
+    M, K = x.shape
+    N = w.shape[0]
+    dev = x.device
+    y, dx, dw = _out((M, N), out_dtype, dev, y), _out((M, K), out_dtype, dev, dx), _out((N, K), out_dtype, dev, dw)
+    if stats is None:
+        stats = torch.zeros(6 * 24, dtype=torch.uint8, device=dev)
+    if ws is None:
+        ws = torch.zeros(snip_linear_fwd_bwd_workspace(M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad, pow2_scale), dtype=torch.uint8, device=dev)
+    _check("snip_linear_fwd_bwd", _lib.snip_linear_fwd_bwd(_p(x), _p(w), _p(dy), _p(y), _p(dx), _p(dw), M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad,
+                                                           out_dtype, int(pow2_scale), _p(stats), _p(ws), ws.numel(), _stream()))
+    return y, dx, dw, stats
 
 
 def snip_layer_stats_workspace(M, N, K):

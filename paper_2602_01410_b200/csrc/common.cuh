@@ -28,6 +28,15 @@ static inline bool valid_fmt(int f) { return f >= SNIP_FMT_BF16 && f <= SNIP_FMT
 static inline bool valid_block(int b) { return b >= SNIP_BLOCK_ROW_1x128 && b <= SNIP_BLOCK_BLK_128x128; }
 static inline bool valid_dim(int64_t d) { return d > 0 && (d % 64) == 0; }
 
+// One output of the two-output quantizer (quantize.cu: quantize_dual_impl).
+struct DualOut {
+    int fmt;
+    void *codes;
+    float *scales;
+    void *sf;             // optional UE8M0 atoms (power-of-two rule only)
+    snip_stats_t *stats;  // optional; both outputs or neither
+};
+
 // Fails with SNIP_ERR_UNSUPPORTED unless the current device is compute capability 10.x.
 int require_sm100();
 

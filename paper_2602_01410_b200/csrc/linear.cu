@@ -16,6 +16,8 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
                  int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st);
 int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st);
 size_t gemm_ws_bytes();
+int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bool blk, int pow2, const DualOut &oa, const DualOut &ob,
+                       void *ws, size_t ws_bytes, cudaStream_t st);
 
 namespace {
 
@@ -141,6 +143,46 @@ int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int6
                      out_dtype, accumulate, gws, gemm_ws_bytes(), st);
 }
 
+
+// ---- forward + both gradients of one linear layer with each tensor read once ------------------
+
+// Buffers of the six quantized copies: X as stored (fwd) / transposed (wgrad), W as stored (fwd) /
+// transposed (dgrad), dY as stored (dgrad) / transposed (wgrad).
+struct FwdBwdCarve {
+    void *gws;
+    void *codes[6];
+    float *scales[6];
+    void *sf[6];
+    void *stats_ws;
+    size_t stats_ws_bytes;
+    size_t total;
+};
+
+FwdBwdCarve carve_fwd_bwd(void *ws, int64_t M, int64_t N, int64_t K, const int (&fmt)[6], bool mx)
+{
+    // index: 0 X/ROW, 1 X/COL^T, 2 W/BLK, 3 W/BLK^T, 4 dY/ROW, 5 dY/COL^T
+    const int64_t rows[6] = {M, M, N, N, M, M}, cols[6] = {K, K, K, K, N, N};
+    const int block[6] = {SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_COL_128x1, SNIP_BLOCK_BLK_128x128, SNIP_BLOCK_BLK_128x128, SNIP_BLOCK_ROW_1x128,
+                          SNIP_BLOCK_COL_128x1};
+    FwdBwdCarve f{};
+    Carve c(ws, 0);
+    f.gws = c.take(gemm_ws_bytes());
+    for (int i = 0; i < 6; ++i) {
+        f.codes[i] = c.take(code_bytes(fmt[i], rows[i], cols[i]));
+        f.scales[i] = static_cast<float *>(c.take(scale_bytes(block[i], rows[i], cols[i])));
+        f.sf[i] = mx ? c.take(sf_bytes(rows[i], cols[i])) : nullptr;
+    }
+    size_t sb = 0;
+    for (int i = 0; i < 6; i += 2) {
+        size_t w = 0;
+        snip_quantize_dual_workspace(rows[i], cols[i], &w);
+        if (w > sb) sb = w;
+    }
+    f.stats_ws = c.take(sb);
+    f.stats_ws_bytes = sb;
+    f.total = c.off;
+    return f;
+}
 }  // namespace
 }  // namespace snip
 
@@ -191,4 +233,59 @@ extern "C" int snip_linear_mx_workspace(int op, int64_t M, int64_t N, int64_t K,
     if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
     *bytes = linear_ws_bytes(op, M, N, K, fmt_a, fmt_b, true);
     return SNIP_OK;
+}
+
+// One linear layer, forward and both gradients, under a precision triple (one tag per GEMM).
+extern "C" int snip_linear_fwd_bwd_workspace(int64_t M, int64_t N, int64_t K, int fmt_fwd, int fmt_dgrad, int fmt_wgrad, int pow2_scale,
+                                             size_t *bytes)
+{
+    using namespace snip;
+    if (!bytes) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    const int fmt[6] = {fmt_fwd, fmt_wgrad, fmt_fwd, fmt_dgrad, fmt_dgrad, fmt_wgrad};
+    for (int f : fmt)
+        if (f != SNIP_FMT_FP8_E4M3 && f != SNIP_FMT_FP4_E2M1) return SNIP_ERR_UNSUPPORTED;
+    *bytes = carve_fwd_bwd(nullptr, M, N, K, fmt, pow2_scale != 0).total;
+    return SNIP_OK;
+}
+
+extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY, void *Y, void *dX, void *dW, int64_t M, int64_t N, int64_t K,
+                                   int fmt_fwd, int fmt_dgrad, int fmt_wgrad, int out_dtype, int pow2_scale, snip_stats_t *stats6, void *ws,
+                                   size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    if (!X || !W || !dY || !Y || !dX || !dW) return SNIP_ERR_ARG;
+    size_t need = 0;
+    int rc = snip_linear_fwd_bwd_workspace(M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad, pow2_scale, &need);
+    if (rc) return rc;
+    if (!ws || ws_bytes < need) return SNIP_ERR_WORKSPACE;
+    if (!aligned16(ws) || (stats6 && (reinterpret_cast<uintptr_t>(stats6) & 7u))) return SNIP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool mx = pow2_scale != 0;
+    const int fmt[6] = {fmt_fwd, fmt_wgrad, fmt_fwd, fmt_dgrad, fmt_dgrad, fmt_wgrad};
+    const FwdBwdCarve f = carve_fwd_bwd(ws, M, N, K, fmt, mx);
+    auto out_of = [&](int i) { return DualOut{fmt[i], f.codes[i], f.scales[i], f.sf[i], stats6 ? stats6 + i : nullptr}; };
+    auto gemm = [&](int op, int ia, int ib, void *out) -> int {
+        const LinearPlan p = plan_for(op, M, N, K);
+        if (mx) return gemm_mx_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], f.sf[ia], f.sf[ib], p.Mo, p.No, p.Kc, out, out_dtype, f.gws, gemm_ws_bytes(), st);
+        int64_t sb_cs, sb_bs;
+        if (op == SNIP_OP_FWD) { sb_bs = ceil_div(K, 128); sb_cs = 1; }
+        else if (op == SNIP_OP_DGRAD) { sb_bs = 1; sb_cs = ceil_div(K, 128); }
+        else { sb_bs = 0; sb_cs = p.No; }
+        return gemm_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], p.Mo, p.No, p.Kc, f.scales[ia], p.Mo, f.scales[ib], sb_cs, sb_bs, p.scale_mode, out,
+                         out_dtype, 0, f.gws, gemm_ws_bytes(), st);
+    };
+    // forward: X and W are read once each and leave both of their quantized copies behind
+    rc = quantize_dual_impl(X, M, K, K, false, mx, out_of(0), out_of(1), f.stats_ws, f.stats_ws_bytes, st);
+    if (rc) return rc;
+    rc = quantize_dual_impl(W, N, K, K, true, mx, out_of(2), out_of(3), f.stats_ws, f.stats_ws_bytes, st);
+    if (rc) return rc;
+    rc = gemm(SNIP_OP_FWD, 0, 2, Y);
+    if (rc) return rc;
+    // backward: dY is read once; dgrad and wgrad consume the stored copies
+    rc = quantize_dual_impl(dY, M, N, N, false, mx, out_of(4), out_of(5), f.stats_ws, f.stats_ws_bytes, st);
+    if (rc) return rc;
+    rc = gemm(SNIP_OP_DGRAD, 4, 3, dX);
+    if (rc) return rc;
+    return gemm(SNIP_OP_WGRAD, 5, 1, dW);
 }

@@ -18,6 +18,8 @@
 
 namespace snip {
 
+int gemm_sm_count();  // gemm.cu: SM count of the current device (cached per device)
+
 namespace {
 
 constexpr int kTile = 128;
@@ -37,48 +39,74 @@ struct QuantArgs {
     float *scales;        // may be null (NO_CODES)
     CtaPartial *partials; // may be null (no stats)
     float2 *row_partials; // [col tiles][rows] {sum x^2, sum err^2}; may be null
+    int64_t tiles_r, tiles_c, ntiles;
     int pow2;             // 1: power-of-two scale rule (largest 2^e with amax * 2^e <= FPX_MAX)
     uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
 };
 
+// Shared memory of one CTA (one 128x128 tile).
+struct QuantShared {
+    __align__(16) uint8_t stage[kTile * kTile];  // transposed codes of the tile (FP8 uses all 16 KB)
+    uint32_t col_amax[8][kTile / 2];              // packed bf16 pairs, one row per warp
+    float col_scale[kTile];
+    float col_ninv[kTile];
+    float red_f[8][3];
+};
+
+// Tile (r, c) of an nr x nc grid of 128x128 tiles.
+struct Tile {
+    int r, c, nr, nc;
+};
+// Running sums of one CTA over the tiles it processes (held by thread 0).
+struct StatsAcc {
+    double x = 0.0, e = 0.0;
+    float m = 0.0f;
+};
+
+// The kernels are persistent: a CTA walks over tiles t = blockIdx.x, blockIdx.x + gridDim.x, ... (row-major
+// tile order).  Each thread fetches its own 8x8 sub-block (eight 16-byte cp.async) into a private slot of
+// shared memory and reads it back itself, so the hand-off needs no barrier: cp.async.wait_group is the
+// only wait.  The next tile's fetch is issued as soon as the current one has been encoded, so it is in
+// flight during the write-out and while the other resident CTAs compute.
+constexpr int kStageBytes = kTile * kTile * 2;
+
+__device__ __forceinline__ void prefetch_tile(const QuantArgs &a, int tr, int tc, uint8_t *stage_base)
+{
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int64_t rbase = (int64_t)tr * kTile + 8 * ty, cbase = (int64_t)tc * kTile + 8 * tx;
+    const bool ok = cbase < a.cols && rbase < a.rows;       // dims are multiples of 64: all 64 elements or none
+    const uint16_t *xb = a.x + (ok ? rbase * a.ld + cbase : 0);
+    const uint32_t ld32 = (uint32_t)a.ld;
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage_base) + tid * 16;
+    const int nbytes = ok ? 16 : 0;                          // 0: the slot is zero-filled, nothing is read
+#pragma unroll
+    for (int p = 0; p < 8; ++p)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + p * (kThreads * 16)), "l"(xb + (ok ? p * ld32 : 0)), "r"(nbytes) : "memory");
+}
+__device__ __forceinline__ void prefetch_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void prefetch_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// One output of the tile whose 8x8 sub-block of this thread sits in slot[p * kThreads], p = 0..7 (shared memory;
+// re-read where needed instead of held in registers, which keeps four CTAs resident per SM).
 // FMT: target format (BF16 = statistics only).  BLOCK: tile kind.  TRANSPOSED: codes stored as
 // the transpose.  CODES: write codes and scales.  STATS: accumulate sums.  ROWSTATS: per-row sums.
 template <int FMT, int BLOCK, bool TRANSPOSED, bool CODES, bool STATS, bool ROWSTATS>
-__global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
+__device__ __forceinline__ void quantize_tile(const QuantArgs &a, const Tile &tl, const uint4 *slot, QuantShared &sh, StatsAcc &acc)
 {
     constexpr bool kQuant = (FMT != SNIP_FMT_BF16);
     constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;  // bytes per 8 elements
     constexpr int kRowBytes = kTile * kCodeBytes8 / 8;               // staged bytes per line
+    uint8_t *const stage = sh.stage;
+    auto &col_amax = sh.col_amax;
+    auto &col_scale = sh.col_scale;
+    auto &col_ninv = sh.col_ninv;
+    auto &red_f = sh.red_f;
 
-    __shared__ __align__(16) uint8_t stage[TRANSPOSED && CODES && kQuant ? kTile * kRowBytes : 16];
-    __shared__ uint32_t col_amax[8][kTile / 2];  // packed bf16 pairs, one row per warp
-    __shared__ float col_scale[kTile];
-    __shared__ float col_ninv[kTile];
-    __shared__ float red_f[8][3];
-
-    // the statistics reduction that follows on the stream may be scheduled now; it waits for this
-    // grid to finish before it reads anything (programmatic dependent launch)
-    if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tx = tid & 15, ty = tid >> 4;
-    const int64_t r0 = (int64_t)blockIdx.y * kTile, c0 = (int64_t)blockIdx.x * kTile;
+    const int64_t r0 = (int64_t)tl.r * kTile, c0 = (int64_t)tl.c * kTile;
     const int64_t rbase = r0 + 8 * ty, cbase = c0 + 8 * tx;
     const bool col_ok = cbase < a.cols;  // cols is a multiple of 64, so 8-groups never straddle
-
-    // ---- load the 8x8 sub-block: eight independent 128-bit loads ------------------------
-    uint4 v[8];
-    {
-        const uint16_t *xb = a.x + rbase * a.ld + cbase;   // 64-bit arithmetic once per thread
-        const bool rows_ok = rbase < a.rows;               // rows is a multiple of 64: all 8 rows or none
-        const uint32_t ld32 = (uint32_t)a.ld;
-#pragma unroll
-        for (int p = 0; p < 8; ++p) {
-            if (col_ok && rows_ok)
-                v[p] = __ldg(reinterpret_cast<const uint4 *>(xb + p * ld32));
-            else
-                v[p] = make_uint4(0, 0, 0, 0);
-        }
-    }
 
     // ---- block amax -> scales --------------------------------------------------------
     float s_row[8], s_col[8];  // scale per row p (ROW) / per column j (COL); BLK uses s_row[0]
@@ -89,10 +117,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
         uint32_t rmax[8];      // per row: packed max over the 8 columns (as 4 pairs folded)
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
-            uint32_t m = absmax2(0u, v[p].x);
-            m = absmax2(m, v[p].y);
-            m = absmax2(m, v[p].z);
-            m = absmax2(m, v[p].w);
+            const uint4 vp = slot[p * kThreads];
+            uint32_t m = absmax2(0u, vp.x);
+            m = absmax2(m, vp.y);
+            m = absmax2(m, vp.z);
+            m = absmax2(m, vp.w);
             rmax[p] = m;
         }
         if (BLOCK == SNIP_BLOCK_ROW_1x128 && kQuant) {
@@ -128,7 +157,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             }
             if (CODES && tx == 0 && a.sf) {
                 // atom [row tile][column tile]: word (r % 32) * 4 + r / 32 holds row r's byte four times
-                uint32_t *atom = a.sf + ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * 128;
+                uint32_t *atom = a.sf + ((int64_t)tl.r * tl.nc + tl.c) * 128;
 #pragma unroll
                 for (int p = 0; p < 8; ++p) {
                     const int r = 8 * ty + p;
@@ -137,7 +166,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             }
             if (CODES && tx == 0) {
                 // scales[tile j][row]: eight consecutive rows per thread
-                float *dst = a.scales + (int64_t)blockIdx.x * a.rows + rbase;
+                float *dst = a.scales + (int64_t)tl.c * a.rows + rbase;
                 if (rbase < a.rows) {
                     *reinterpret_cast<float4 *>(dst) = make_float4(s_row[0], s_row[1], s_row[2], s_row[3]);
                     *reinterpret_cast<float4 *>(dst + 4) = make_float4(s_row[4], s_row[5], s_row[6], s_row[7]);
@@ -148,10 +177,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             uint32_t cm[4] = {0, 0, 0, 0};
 #pragma unroll
             for (int p = 0; p < 8; ++p) {
-                cm[0] = absmax2(cm[0], v[p].x);
-                cm[1] = absmax2(cm[1], v[p].y);
-                cm[2] = absmax2(cm[2], v[p].z);
-                cm[3] = absmax2(cm[3], v[p].w);
+                const uint4 vp = slot[p * kThreads];
+                cm[0] = absmax2(cm[0], vp.x);
+                cm[1] = absmax2(cm[1], vp.y);
+                cm[2] = absmax2(cm[2], vp.z);
+                cm[3] = absmax2(cm[3], vp.w);
             }
             if (BLOCK == SNIP_BLOCK_COL_128x1 && kQuant) {
                 // the two row groups of a warp, then the 8 warps through shared memory
@@ -170,8 +200,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
                     col_scale[tid] = s;
                     col_ninv[tid] = neg_inv_scale<FMT>(am, s, a.pow2);
                     // atom [column tile][row tile] (the operand is consumed transposed): one word per column
-                    if (CODES && a.sf) a.sf[((int64_t)blockIdx.x * gridDim.y + blockIdx.y) * 128 + (tid & 31) * 4 + (tid >> 5)] = (c0 + tid < a.cols) ? sf_word(s) : 0x7F7F7F7Fu;
-                    if (CODES && c0 + tid < a.cols) a.scales[(int64_t)blockIdx.y * a.cols + c0 + tid] = s;
+                    if (CODES && a.sf) a.sf[((int64_t)tl.c * tl.nr + tl.r) * 128 + (tid & 31) * 4 + (tid >> 5)] = (c0 + tid < a.cols) ? sf_word(s) : 0x7F7F7F7Fu;
+                    if (CODES && c0 + tid < a.cols) a.scales[(int64_t)tl.r * a.cols + c0 + tid] = s;
                     if (STATS) my_amax = am;
                 }
                 __syncthreads();
@@ -201,10 +231,10 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
                     s_row[0] = tile_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm, a.pow2);
                     n_row[0] = neg_inv_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm, s_row[0], a.pow2);
                     if (CODES && a.sf && tid < kTile) {
-                        const int64_t atom = TRANSPOSED ? (int64_t)blockIdx.x * gridDim.y + blockIdx.y : (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+                        const int64_t atom = TRANSPOSED ? (int64_t)tl.c * tl.nr + tl.r : (int64_t)tl.r * tl.nc + tl.c;
                         a.sf[atom * 128 + tid] = sf_word(s_row[0]);
                     }
-                    if (CODES && tid == 0) a.scales[(int64_t)blockIdx.y * gridDim.x + blockIdx.x] = s_row[0];
+                    if (CODES && tid == 0) a.scales[(int64_t)tl.r * tl.nc + tl.c] = s_row[0];
                 }
                 __syncthreads();  // red_f is reused below
             }
@@ -234,11 +264,11 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             }
             if (ROWSTATS) {
                 float2 px = make_float2(0.0f, 0.0f), pe = make_float2(0.0f, 0.0f);
-                quant8<FMT, STATS>(v[p], sc, ni, codes[p], px, pe);
+                quant8<FMT, STATS>(slot[p * kThreads], sc, ni, codes[p], px, pe);
                 rsx[p] = px.x + px.y; rse[p] = pe.x + pe.y;
                 sx += rsx[p]; se += rse[p];
             } else {
-                quant8<FMT, STATS>(v[p], sc, ni, codes[p], sx2, se2);
+                quant8<FMT, STATS>(slot[p * kThreads], sc, ni, codes[p], sx2, se2);
             }
         }
         if (STATS && !ROWSTATS) { sx = sx2.x + sx2.y; se = se2.x + se2.y; }
@@ -312,7 +342,8 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
         // BF16: identity, only sum x^2
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
-            const uint32_t w[4] = {v[p].x, v[p].y, v[p].z, v[p].w};
+            const uint4 vp = slot[p * kThreads];
+            const uint32_t w[4] = {vp.x, vp.y, vp.z, vp.w};
             float px = 0.0f;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -337,7 +368,7 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             }
         }
         if (tx == 0 && rbase < a.rows) {
-            float2 *dst = a.row_partials + (int64_t)blockIdx.x * a.rows + rbase;
+            float2 *dst = a.row_partials + (int64_t)tl.c * a.rows + rbase;
 #pragma unroll
             for (int p = 0; p < 8; ++p) dst[p] = make_float2(rsx[p], rse[p]);
         }
@@ -356,22 +387,113 @@ __global__ void __launch_bounds__(kThreads) quantize_kernel(const QuantArgs a)
             float am = 0.0f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) { dx += (double)red_f[w][0]; de += (double)red_f[w][1]; am = fmaxf(am, red_f[w][2]); }
-            CtaPartial *dst = a.partials + (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
-            dst->sumsq_x = dx;
-            dst->sumsq_err = de;
-            dst->amax = am;
+            acc.x += dx;
+            acc.e += de;
+            acc.m = fmaxf(acc.m, am);
         }
     }
+}
+
+// Dynamic shared memory of the kernels: the tile slot, then the QuantShared scratch.
+constexpr size_t kSmemBytes = (size_t)kStageBytes + sizeof(QuantShared);
+constexpr int kCtasPerSm = 4;
+
+__device__ __forceinline__ void write_partial(CtaPartial *partials, const StatsAcc &acc)
+{
+    if (threadIdx.x == 0) {
+        CtaPartial *dst = partials + blockIdx.x;
+        dst->sumsq_x = acc.x;
+        dst->sumsq_err = acc.e;
+        dst->amax = acc.m;
+    }
+}
+
+// Walk of one CTA over its tiles without divisions in the loop.
+struct TileWalk {
+    int r, c, step_r, step_c, nr, nc;
+    __device__ __forceinline__ TileWalk(int nr_, int nc_) : nr(nr_), nc(nc_)
+    {
+        r = (int)blockIdx.x / nc_; c = (int)blockIdx.x % nc_;
+        step_r = (int)gridDim.x / nc_; step_c = (int)gridDim.x % nc_;
+    }
+    __device__ __forceinline__ bool valid() const { return r < nr; }
+    __device__ __forceinline__ void next()
+    {
+        r += step_r; c += step_c;
+        if (c >= nc) { c -= nc; ++r; }
+    }
+};
+
+template <int FMT, int BLOCK, bool TRANSPOSED, bool CODES, bool STATS, bool ROWSTATS>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const QuantArgs a)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
+    const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
+    // the statistics reduction that follows on the stream may be scheduled now; it waits for this
+    // grid to finish before it reads anything (programmatic dependent launch)
+    if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    StatsAcc acc;
+    TileWalk w((int)a.tiles_r, (int)a.tiles_c);
+    if (w.valid()) prefetch_tile(a, w.r, w.c, smem);
+    prefetch_commit();
+    while (w.valid()) {
+        prefetch_wait<0>();
+        const Tile tl = {w.r, w.c, w.nr, w.nc};
+        quantize_tile<FMT, BLOCK, TRANSPOSED, CODES, STATS, ROWSTATS>(a, tl, slot, sh, acc);
+        w.next();
+        if (w.valid()) prefetch_tile(a, w.r, w.c, smem);   // this thread's reads of its slot are done
+        prefetch_commit();
+        __syncthreads();  // the scratch arrays are reused by the next tile
+    }
+    if (STATS) write_partial(a.partials, acc);
+}
+
+// Two outputs from one read (the tile kinds a tensor is consumed with, paper Fig. 5): `a` as stored
+// (1x128 tiles along the columns, or 128x128 blocks) and `b` transposed (128x1 tiles along the rows, or
+// the same 128x128 blocks), each with its own format, scales and statistics.
+struct DualArgs {
+    QuantArgs a, b;
+};
+template <int FMT_A, int FMT_B, bool BLK, bool STATS>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_dual_kernel(const DualArgs d)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
+    const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
+    if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    StatsAcc acc_a, acc_b;
+    TileWalk w((int)d.a.tiles_r, (int)d.a.tiles_c);
+    if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
+    prefetch_commit();
+    while (w.valid()) {
+        prefetch_wait<0>();
+        const Tile tl = {w.r, w.c, w.nr, w.nc};
+        quantize_tile<FMT_A, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true, STATS, false>(d.a, tl, slot, sh, acc_a);
+        __syncthreads();  // the scratch arrays are reused by the second output
+        quantize_tile<FMT_B, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true, STATS, false>(d.b, tl, slot, sh, acc_b);
+        w.next();
+        if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
+        prefetch_commit();
+        __syncthreads();
+    }
+    if (STATS) { write_partial(d.a.partials, acc_a); write_partial(d.b.partials, acc_b); }
 }
 
 // Fixed-order reduction of the per-CTA partials into one snip_stats_t (deterministic: every thread
 // owns a fixed strided subset, warps combine with shuffles, warp results are added in warp order).
 // Launched with programmatic stream serialization: it may start while the quantizer still runs and
 // blocks in griddepcontrol.wait until that grid has completed and its writes are visible.
-__global__ void __launch_bounds__(1024) stats_reduce_kernel(const CtaPartial *partials, int64_t n, snip_stats_t *out)
+struct ReduceSets {
+    const CtaPartial *partials[2];
+    snip_stats_t *out[2];
+};
+__global__ void __launch_bounds__(1024) stats_reduce_kernel(const ReduceSets sets, int64_t n)
 {
     __shared__ double sh_x[32], sh_e[32];
     __shared__ float sh_m[32];
+    const CtaPartial *partials = sets.partials[blockIdx.x];
+    snip_stats_t *out = sets.out[blockIdx.x];
     asm volatile("griddepcontrol.wait;" ::: "memory");
     double dx = 0.0, de = 0.0;
     float am = 0.0f;
@@ -416,14 +538,23 @@ __global__ void row_stats_reduce_kernel(const float2 *row_partials, int64_t rows
     row_stats[2 * r + 1] = de;
 }
 
+// Launch of a persistent kernel: its dynamic shared memory exceeds the default limit, so the limit is
+// raised first (a per-function, per-device attribute; setting it again is cheap).
+template <typename Kernel, typename Args>
+void launch_persistent(Kernel kernel, const Args &args, dim3 grid, cudaStream_t st)
+{
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) return;  // left in cudaGetLastError
+    kernel<<<grid, kThreads, kSmemBytes, st>>>(args);
+}
+
 template <int FMT, int BLOCK, bool TRANSPOSED>
 void launch_variant(const QuantArgs &a, bool codes, bool stats, bool rowstats, dim3 grid, cudaStream_t st)
 {
-    if (codes && stats && rowstats) quantize_kernel<FMT, BLOCK, TRANSPOSED, true, true, true><<<grid, kThreads, 0, st>>>(a);
-    else if (codes && stats) quantize_kernel<FMT, BLOCK, TRANSPOSED, true, true, false><<<grid, kThreads, 0, st>>>(a);
-    else if (codes) quantize_kernel<FMT, BLOCK, TRANSPOSED, true, false, false><<<grid, kThreads, 0, st>>>(a);
-    else if (rowstats) quantize_kernel<FMT, BLOCK, false, false, true, true><<<grid, kThreads, 0, st>>>(a);
-    else quantize_kernel<FMT, BLOCK, false, false, true, false><<<grid, kThreads, 0, st>>>(a);
+    if (codes && stats && rowstats) launch_persistent(quantize_kernel<FMT, BLOCK, TRANSPOSED, true, true, true>, a, grid, st);
+    else if (codes && stats) launch_persistent(quantize_kernel<FMT, BLOCK, TRANSPOSED, true, true, false>, a, grid, st);
+    else if (codes) launch_persistent(quantize_kernel<FMT, BLOCK, TRANSPOSED, true, false, false>, a, grid, st);
+    else if (rowstats) launch_persistent(quantize_kernel<FMT, BLOCK, false, false, true, true>, a, grid, st);
+    else launch_persistent(quantize_kernel<FMT, BLOCK, false, false, true, false>, a, grid, st);
 }
 
 template <int FMT>
@@ -439,6 +570,14 @@ void launch_fmt(const QuantArgs &a, int block, bool transposed, bool codes, bool
         if (transposed) launch_variant<FMT, SNIP_BLOCK_BLK_128x128, true>(a, codes, stats, rowstats, grid, st);
         else launch_variant<FMT, SNIP_BLOCK_BLK_128x128, false>(a, codes, stats, rowstats, grid, st);
     }
+}
+
+// CTAs of a persistent launch over ntiles tiles: kCtasPerSm per SM (what the kernels' shared memory and
+// registers allow), never more than there are tiles.
+int64_t persistent_ctas(int64_t ntiles)
+{
+    const int64_t cap = kCtasPerSm * (int64_t)gemm_sm_count();
+    return ntiles < cap ? ntiles : cap;
 }
 
 size_t stats_ws_bytes(int64_t rows, int64_t cols, bool rowstats)
@@ -491,7 +630,6 @@ int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
     if (rc != SNIP_OK) return rc;
 
     const int64_t tr = ceil_div(rows, kTile), tc = ceil_div(cols, kTile);
-    if (tr > 65535) return SNIP_ERR_SHAPE;
     QuantArgs a;
     a.x = static_cast<const uint16_t *>(x);
     a.rows = rows; a.cols = cols; a.ld = ld;
@@ -500,7 +638,9 @@ int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
     a.scales = want_codes ? scales : nullptr;
     a.partials = any_stats ? static_cast<CtaPartial *>(ws) : nullptr;
     a.row_partials = want_rows ? reinterpret_cast<float2 *>(static_cast<uint8_t *>(ws) + align_up((size_t)(tr * tc) * sizeof(CtaPartial), 256)) : nullptr;
-    dim3 grid((unsigned)tc, (unsigned)tr);
+    a.tiles_r = tr; a.tiles_c = tc; a.ntiles = tr * tc;
+    const int64_t nparts = persistent_ctas(tr * tc);
+    dim3 grid((unsigned)nparts);
     if (fmt == SNIP_FMT_FP8_E4M3) launch_fmt<SNIP_FMT_FP8_E4M3>(a, block, transposed, want_codes, any_stats, want_rows, grid, st);
     else if (fmt == SNIP_FMT_FP4_E2M1) launch_fmt<SNIP_FMT_FP4_E2M1>(a, block, transposed, want_codes, any_stats, want_rows, grid, st);
     else launch_variant<SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, false>(a, false, true, want_rows, grid, st);
@@ -515,13 +655,83 @@ int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        const CtaPartial *parts = a.partials;
-        const int64_t nparts = tr * tc;
-        SNIP_CUDA_TRY(cudaLaunchKernelEx(&cfg, stats_reduce_kernel, parts, nparts, stats));
+        const ReduceSets sets = {{a.partials, nullptr}, {stats, nullptr}};
+        SNIP_CUDA_TRY(cudaLaunchKernelEx(&cfg, stats_reduce_kernel, sets, nparts));
     }
     if (want_rows) {
         row_stats_reduce_kernel<<<(unsigned)ceil_div(rows, 256), 256, 0, st>>>(a.row_partials, rows, tc, row_stats);
         SNIP_CUDA_TRY(cudaGetLastError());
+    }
+    return SNIP_OK;
+}
+
+// One read, two outputs.  blk = false: a = 1x128 tiles as stored, b = 128x1 tiles transposed;
+// blk = true: a = 128x128 blocks as stored, b = the same blocks transposed.
+template <int FMT_A, int FMT_B>
+static void launch_dual(const DualArgs &d, bool blk, bool stats, dim3 grid, cudaStream_t st)
+{
+    if (blk && stats) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, true, true>, d, grid, st);
+    else if (blk) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, true, false>, d, grid, st);
+    else if (stats) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, true>, d, grid, st);
+    else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false>, d, grid, st);
+}
+
+int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bool blk, int pow2, const DualOut &oa, const DualOut &ob,
+                       void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    if (!x) return SNIP_ERR_ARG;
+    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0) return SNIP_ERR_SHAPE;
+    const DualOut *o[2] = {&oa, &ob};
+    for (int i = 0; i < 2; ++i) {
+        if (o[i]->fmt != SNIP_FMT_FP8_E4M3 && o[i]->fmt != SNIP_FMT_FP4_E2M1) return SNIP_ERR_UNSUPPORTED;
+        if (!o[i]->codes || !o[i]->scales) return SNIP_ERR_ARG;
+        if (o[i]->sf && !pow2) return SNIP_ERR_UNSUPPORTED;
+        if (!aligned16(o[i]->codes) || !aligned16(o[i]->scales) || (o[i]->sf && !aligned16(o[i]->sf)) ||
+            (o[i]->stats && (reinterpret_cast<uintptr_t>(o[i]->stats) & 7u)))
+            return SNIP_ERR_ALIGN;
+    }
+    if ((oa.stats == nullptr) != (ob.stats == nullptr)) return SNIP_ERR_ARG;
+    if (!aligned16(x)) return SNIP_ERR_ALIGN;
+    const bool stats = oa.stats != nullptr;
+    const size_t one = stats_ws_bytes(rows, cols, false);
+    if (stats && (!ws || ws_bytes < 2 * one)) return SNIP_ERR_WORKSPACE;
+    if (stats && !aligned16(ws)) return SNIP_ERR_ALIGN;
+    int rc = require_sm100();
+    if (rc != SNIP_OK) return rc;
+    const int64_t tr = ceil_div(rows, kTile), tc = ceil_div(cols, kTile);
+    DualArgs d;
+    for (int i = 0; i < 2; ++i) {
+        QuantArgs &q = i ? d.b : d.a;
+        q.x = static_cast<const uint16_t *>(x);
+        q.rows = rows; q.cols = cols; q.ld = ld;
+        q.codes = static_cast<uint8_t *>(o[i]->codes);
+        q.scales = o[i]->scales;
+        q.partials = stats ? reinterpret_cast<CtaPartial *>(static_cast<uint8_t *>(ws) + i * one) : nullptr;
+        q.row_partials = nullptr;
+        q.pow2 = pow2;
+        q.sf = static_cast<uint32_t *>(o[i]->sf);
+        q.tiles_r = tr; q.tiles_c = tc; q.ntiles = tr * tc;
+    }
+    const int64_t nparts = persistent_ctas(tr * tc);
+    dim3 grid((unsigned)nparts);
+    const bool a8 = oa.fmt == SNIP_FMT_FP8_E4M3, b8 = ob.fmt == SNIP_FMT_FP8_E4M3;
+    if (a8 && b8) launch_dual<SNIP_FMT_FP8_E4M3, SNIP_FMT_FP8_E4M3>(d, blk, stats, grid, st);
+    else if (a8) launch_dual<SNIP_FMT_FP8_E4M3, SNIP_FMT_FP4_E2M1>(d, blk, stats, grid, st);
+    else if (b8) launch_dual<SNIP_FMT_FP4_E2M1, SNIP_FMT_FP8_E4M3>(d, blk, stats, grid, st);
+    else launch_dual<SNIP_FMT_FP4_E2M1, SNIP_FMT_FP4_E2M1>(d, blk, stats, grid, st);
+    SNIP_CUDA_TRY(cudaGetLastError());
+    if (stats) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2);
+        cfg.blockDim = dim3(1024);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const ReduceSets sets = {{d.a.partials, d.b.partials}, {oa.stats, ob.stats}};
+        SNIP_CUDA_TRY(cudaLaunchKernelEx(&cfg, stats_reduce_kernel, sets, nparts));
     }
     return SNIP_OK;
 }
@@ -637,3 +847,26 @@ extern "C" int snip_quantize_mx(const void *x, int64_t rows, int64_t cols, int64
                             static_cast<cudaStream_t>(stream));
 }
 
+
+// ---- one read, two outputs -------------------------------------------------------------------
+
+extern "C" int snip_quantize_dual_workspace(int64_t rows, int64_t cols, size_t *ws_bytes)
+{
+    using namespace snip;
+    if (!ws_bytes) return SNIP_ERR_ARG;
+    if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
+    *ws_bytes = 2 * stats_ws_bytes(rows, cols, false);
+    return SNIP_OK;
+}
+
+extern "C" int snip_quantize_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, int kind, int pow2_scale,
+                                  const snip_qout_t *as_stored, const snip_qout_t *transposed, void *ws, size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    if (!as_stored || !transposed) return SNIP_ERR_ARG;
+    if (kind != SNIP_DUAL_ROW_COLT && kind != SNIP_DUAL_BLK_BLKT) return SNIP_ERR_ARG;
+    const DualOut oa = {as_stored->fmt, as_stored->codes, as_stored->scales, as_stored->sf, as_stored->stats};
+    const DualOut ob = {transposed->fmt, transposed->codes, transposed->scales, transposed->sf, transposed->stats};
+    return quantize_dual_impl(x, rows, cols, ld, kind == SNIP_DUAL_BLK_BLKT, pow2_scale ? 1 : 0, oa, ob, ws, ws_bytes,
+                              static_cast<cudaStream_t>(stream));
+}
