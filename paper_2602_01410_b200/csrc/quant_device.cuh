@@ -23,6 +23,14 @@ __device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t v)
     return *reinterpret_cast<uint32_t *>(&m);
 }
 
+// packed bf16: magnitude of each half = max(|a|, |b|); the sign bits are meaningless (mask them at the end)
+__device__ __forceinline__ uint32_t absmax2x(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t max2(uint32_t x, uint32_t y)
 {
     __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&x);

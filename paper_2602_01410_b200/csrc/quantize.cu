@@ -44,25 +44,22 @@ struct QuantArgs {
     uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
 };
 
-// Shared memory of one CTA (one 128x128 tile).
+// Scratch shared memory of one CTA (next to the tile slot).
 struct QuantShared {
     __align__(16) uint8_t stage[kTile * kTile];  // transposed codes of the tile (FP8 uses all 16 KB)
     uint32_t col_amax[8][kTile / 2];              // packed bf16 pairs, one row per warp
     float col_scale[kTile];
     float col_ninv[kTile];
-    float red_f[8][3];
+    float row_scale[kTile];
+    float row_ninv[kTile];
+    uint32_t red_m[8];
+    double red_d[8][4];
 };
 
 // Tile (r, c) of an nr x nc grid of 128x128 tiles.
 struct Tile {
     int r, c, nr, nc;
 };
-// Running sums of one CTA over the tiles it processes (held by thread 0).
-struct StatsAcc {
-    double x = 0.0, e = 0.0;
-    float m = 0.0f;
-};
-
 // The kernels are persistent: a CTA walks over tiles t = blockIdx.x, blockIdx.x + gridDim.x, ... (row-major
 // tile order).  Each thread fetches its own 8x8 sub-block (eight 16-byte cp.async) into a private slot of
 // shared memory and reads it back itself, so the hand-off needs no barrier: cp.async.wait_group is the
@@ -86,279 +83,378 @@ __device__ __forceinline__ void prefetch_tile(const QuantArgs &a, int tr, int tc
 __device__ __forceinline__ void prefetch_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void prefetch_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-// One output of the tile whose 8x8 sub-block of this thread sits in slot[p * kThreads], p = 0..7 (shared memory;
-// re-read where needed instead of held in registers, which keeps four CTAs resident per SM).
-// FMT: target format (BF16 = statistics only).  BLOCK: tile kind.  TRANSPOSED: codes stored as
-// the transpose.  CODES: write codes and scales.  STATS: accumulate sums.  ROWSTATS: per-row sums.
-template <int FMT, int BLOCK, bool TRANSPOSED, bool CODES, bool STATS, bool ROWSTATS>
-__device__ __forceinline__ void quantize_tile(const QuantArgs &a, const Tile &tl, const uint4 *slot, QuantShared &sh, StatsAcc &acc)
-{
-    constexpr bool kQuant = (FMT != SNIP_FMT_BF16);
-    constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;  // bytes per 8 elements
-    constexpr int kRowBytes = kTile * kCodeBytes8 / 8;               // staged bytes per line
-    uint8_t *const stage = sh.stage;
-    auto &col_amax = sh.col_amax;
-    auto &col_scale = sh.col_scale;
-    auto &col_ninv = sh.col_ninv;
-    auto &red_f = sh.red_f;
+// Compile-time description of one output of a tile pass.
+template <int FMT_, int BLOCK_, bool TRANSPOSED_, bool CODES_>
+struct Out {
+    static constexpr int FMT = FMT_, BLOCK = BLOCK_;
+    static constexpr bool TRANSPOSED = TRANSPOSED_, CODES = CODES_, kQuant = (FMT_ != SNIP_FMT_BF16);
+};
+struct NoOut {
+    static constexpr int FMT = SNIP_FMT_BF16, BLOCK = SNIP_BLOCK_BLK_128x128;
+    static constexpr bool TRANSPOSED = false, CODES = false, kQuant = false;
+};
 
+// Per-thread running sums over the tiles of a CTA (binary64: one add per tile and sum).
+struct ThreadStats {
+    double x = 0.0, ea = 0.0, eb = 0.0;
+    float amax = 0.0f;
+};
+
+// -1/S for the error term x - value(code)/S = x + value(code) * (-1/S).  Paper's rule: amax/FPX_MAX equals
+// 1/S to within one rounding, which the statistics (1e-4) do not see; power-of-two rule: exact, from the
+// exponent field.  For an empty tile the value is irrelevant (all codes are zero).
+template <int FMT>
+__device__ __forceinline__ float neg_inv(float amax, float s, int pow2)
+{
+    constexpr float kInvMax = (FMT == SNIP_FMT_FP8_E4M3) ? (1.0f / 448.0f) : (1.0f / 6.0f);
+    return pow2 ? __uint_as_float(0x80000000u | ((254u << 23) - __float_as_uint(s))) : -amax * kInvMax;
+}
+
+// Two binary32 products -> packed codes of an element pair (FP8: 16 bits, FP4: 8 bits) and, with STATS,
+// the squared error added to se2.
+template <int FMT, bool STATS>
+__device__ __forceinline__ uint32_t encode_pair(const float2 x, const float2 s, const float2 n, float2 &se2)
+{
+    const float2 t = __fmul2_rn(x, s);   // IEEE binary32 products, as the scalar definition asks for
+    uint32_t c;
+    if (FMT == SNIP_FMT_FP8_E4M3) c = cvt_e4m3x2(t.x, t.y);
+    else c = cvt_e2m1x2(t.x, t.y);
+    if (STATS) {
+        const float2 d = (FMT == SNIP_FMT_FP8_E4M3) ? dec_e4m3x2(c) : dec_e2m1x2(c);
+        const float2 e = __ffma2_rn(d, n, x);
+        se2 = __ffma2_rn(e, e, se2);
+    }
+    return c;
+}
+
+// Packs the four pair codes of 8 consecutive elements: FP8 -> two words, FP4 -> one word.
+template <int FMT>
+__device__ __forceinline__ void pack8(const uint32_t (&c)[4], uint32_t (&out)[2])
+{
+    if (FMT == SNIP_FMT_FP8_E4M3) {
+        out[0] = c[0] | (c[1] << 16);
+        out[1] = c[2] | (c[3] << 16);
+    } else {
+        out[0] = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
+        out[1] = 0;
+    }
+}
+
+// Stores this thread's 8x8 codes as stored (row-major): one 8-byte (FP8) or 4-byte (FP4) store per row.
+template <int FMT>
+__device__ __forceinline__ void store_row(const QuantArgs &a, int64_t rbase, int64_t cbase, int p, const uint32_t (&code)[2])
+{
+    constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;
+    const int64_t out_ld = a.cols * kCodeBytes8 / 8;
+    uint8_t *dst = a.codes + (rbase + p) * out_ld + cbase * kCodeBytes8 / 8;
+    if (FMT == SNIP_FMT_FP8_E4M3) *reinterpret_cast<uint2 *>(dst) = make_uint2(code[0], code[1]);
+    else *reinterpret_cast<uint32_t *>(dst) = code[0];
+}
+
+// 4x4 byte transpose: t[j] byte i = a[i] byte j (eight byte permutes).
+__device__ __forceinline__ void transpose4x4_bytes(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t (&t)[4])
+{
+    const uint32_t x0 = __byte_perm(a0, a1, 0x5140), x1 = __byte_perm(a0, a1, 0x7362);
+    const uint32_t y0 = __byte_perm(a2, a3, 0x5140), y1 = __byte_perm(a2, a3, 0x7362);
+    t[0] = __byte_perm(x0, y0, 0x5410);
+    t[1] = __byte_perm(x0, y0, 0x7632);
+    t[2] = __byte_perm(x1, y1, 0x5410);
+    t[3] = __byte_perm(x1, y1, 0x7632);
+}
+
+// Transposes this thread's 8x8 codes in registers and stages them: line (8*tx + j) of the transposed tile
+// gets the codes of rows 8*ty .. 8*ty+7 of column 8*tx + j.  The chunk index ty is XOR-ed with tx so that
+// the 16 lanes of a row group hit distinct banks.
+template <int FMT>
+__device__ __forceinline__ void stage_transposed(uint8_t *stage, int tx, int ty, const uint32_t (&codes)[8][2])
+{
+    constexpr int kRowBytes = (FMT == SNIP_FMT_FP8_E4M3) ? kTile : kTile / 2;
+    if (FMT == SNIP_FMT_FP8_E4M3) {
+        // codes[p][h]: bytes of columns 4h .. 4h+3 of row p; four 4x4 byte transposes
+        uint32_t lo[2][4], hi[2][4];   // [h][j]: rows 0-3 / rows 4-7 of column 4h + j
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            transpose4x4_bytes(codes[0][h], codes[1][h], codes[2][h], codes[3][h], lo[h]);
+            transpose4x4_bytes(codes[4][h], codes[5][h], codes[6][h], codes[7][h], hi[h]);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            reinterpret_cast<uint2 *>(stage + (8 * tx + j) * kRowBytes)[ty ^ tx] = make_uint2(lo[j >> 2][j & 3], hi[j >> 2][j & 3]);
+    } else {
+        // codes[p][0]: eight nibbles (columns 0..7) of row p.  Pair rows (2q, 2q+1) into bytes, even and odd
+        // columns apart: ev[q] byte k = column 2k, od[q] byte k = column 2k+1 (low nibble = row 2q); a 4x4
+        // byte transpose of each then gives the eight-row word of every column.
+        uint32_t ev[4], od[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t r0 = codes[2 * q][0], r1 = codes[2 * q + 1][0];
+            ev[q] = (r0 & 0x0F0F0F0Fu) | ((r1 << 4) & 0xF0F0F0F0u);
+            od[q] = ((r0 >> 4) & 0x0F0F0F0Fu) | (r1 & 0xF0F0F0F0u);
+        }
+        uint32_t te[4], to[4];
+        transpose4x4_bytes(ev[0], ev[1], ev[2], ev[3], te);
+        transpose4x4_bytes(od[0], od[1], od[2], od[3], to);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            reinterpret_cast<uint32_t *>(stage + (8 * tx + 2 * k) * kRowBytes)[ty ^ tx] = te[k];
+            reinterpret_cast<uint32_t *>(stage + (8 * tx + 2 * k + 1) * kRowBytes)[ty ^ tx] = to[k];
+        }
+    }
+}
+
+// Writes the staged transposed tile: line c holds rows r0 .. r0+127 of column c0 + c; 16-byte stores.
+template <int FMT>
+__device__ __forceinline__ void write_transposed(const QuantArgs &a, const uint8_t *stage, int64_t r0, int64_t c0)
+{
+    constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;
+    constexpr int kRowBytes = kTile * kCodeBytes8 / 8;
+    constexpr int kChunks = kRowBytes / 16;
+    const int64_t out_ld = a.rows * kCodeBytes8 / 8;
+    const int valid_rows = (int)min((int64_t)kTile, a.rows - r0);   // rows is a multiple of 64
+    const int valid_cols = (int)min((int64_t)kTile, a.cols - c0);
+    uint8_t *base = a.codes + c0 * out_ld + r0 * kCodeBytes8 / 8;
+#pragma unroll
+    for (int idx = threadIdx.x; idx < kTile * kChunks; idx += kThreads) {
+        const int c = idx / kChunks, q = idx % kChunks;
+        const int key = (c >> 3) & 15;
+        uint4 o;
+        bool ok = c < valid_cols;
+        if (FMT == SNIP_FMT_FP8_E4M3) {
+            const uint2 *src = reinterpret_cast<const uint2 *>(stage + c * kRowBytes);
+            const uint2 h0 = src[(2 * q) ^ key], h1 = src[(2 * q + 1) ^ key];
+            o = make_uint4(h0.x, h0.y, h1.x, h1.y);
+            ok = ok && 16 * q < valid_rows;
+        } else {
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(stage + c * kRowBytes);
+            o = make_uint4(src[(4 * q) ^ key], src[(4 * q + 1) ^ key], src[(4 * q + 2) ^ key], src[(4 * q + 3) ^ key]);
+            ok = ok && 32 * q < valid_rows;
+        }
+        if (ok) *reinterpret_cast<uint4 *>(base + (int64_t)c * out_ld + 16 * q) = o;
+    }
+}
+
+// Scales of one output for this thread's 8x8 sub-block.
+struct SubScales {
+    float s_row[8], n_row[8];   // 1x128 tiles: one per row p
+    float s_col[8], n_col[8];   // 128x1 tiles: one per column j
+    float s_blk, n_blk;         // 128x128 block
+};
+
+template <class O>
+__device__ __forceinline__ float2 scale_pair(const SubScales &sc, int p, int i)
+{
+    if (O::BLOCK == SNIP_BLOCK_ROW_1x128) return make_float2(sc.s_row[p], sc.s_row[p]);
+    if (O::BLOCK == SNIP_BLOCK_COL_128x1) return make_float2(sc.s_col[2 * i], sc.s_col[2 * i + 1]);
+    return make_float2(sc.s_blk, sc.s_blk);
+}
+template <class O>
+__device__ __forceinline__ float2 ninv_pair(const SubScales &sc, int p, int i)
+{
+    if (O::BLOCK == SNIP_BLOCK_ROW_1x128) return make_float2(sc.n_row[p], sc.n_row[p]);
+    if (O::BLOCK == SNIP_BLOCK_COL_128x1) return make_float2(sc.n_col[2 * i], sc.n_col[2 * i + 1]);
+    return make_float2(sc.n_blk, sc.n_blk);
+}
+
+// Row scales.  rmax[p]: this thread's packed partial maxima of row p (sign bits meaningless).  The 16 lanes
+// of a row group combine them with an exchange-halving butterfly (5 shuffles instead of 16): after it, lane
+// tx holds the maxima of rows 2q and 2q+1, q = 2*bit3(tx) + bit2(tx).  Lane tx with bit1 = 0 then owns row
+// 2q + bit0: it derives the scale (one division per lane), writes the global scale / atom word and
+// publishes scale and -1/S through shared memory; every lane reads back its eight rows after a warp barrier.
+template <class O>
+__device__ __forceinline__ void row_scales(const QuantArgs &a, const Tile &tl, QuantShared &sh, const uint32_t (&rmax)[8], int tx, int ty,
+                                           int64_t rbase, SubScales &sc, float &amax_acc)
+{
+    uint32_t pk[4];   // rows 2q (low half) and 2q+1 (high half)
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        pk[q] = max2(__byte_perm(rmax[2 * q], rmax[2 * q + 1], 0x5410) & 0x7FFF7FFFu, __byte_perm(rmax[2 * q], rmax[2 * q + 1], 0x7632) & 0x7FFF7FFFu);
+    const bool b3 = (tx & 8) != 0, b2 = (tx & 4) != 0;
+    uint32_t k0 = b3 ? pk[2] : pk[0], k1 = b3 ? pk[3] : pk[1];
+    const uint32_t g0 = b3 ? pk[0] : pk[2], g1 = b3 ? pk[1] : pk[3];
+    k0 = max2(k0, __shfl_xor_sync(0xFFFFFFFFu, g0, 8));
+    k1 = max2(k1, __shfl_xor_sync(0xFFFFFFFFu, g1, 8));
+    uint32_t k = b2 ? k1 : k0;
+    const uint32_t g = b2 ? k0 : k1;
+    k = max2(k, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
+    k = max2(k, __shfl_xor_sync(0xFFFFFFFFu, k, 2));
+    k = max2(k, __shfl_xor_sync(0xFFFFFFFFu, k, 1));
+    const int myrow = ((tx >> 3) & 1) * 4 + ((tx >> 2) & 1) * 2 + (tx & 1);
+    const float am = (tx & 1) ? bf16hi(k) : bf16lo(k);
+    amax_acc = fmaxf(amax_acc, am);
+    const float s = tile_scale<O::FMT>(am, a.pow2);
+    if (!(tx & 2)) {
+        const int r = 8 * ty + myrow;
+        sh.row_scale[r] = s;
+        sh.row_ninv[r] = neg_inv<O::FMT>(am, s, a.pow2);
+        if (O::CODES) {
+            // atom [row tile][column tile]: word (r % 32) * 4 + r / 32 holds row r's byte four times
+            if (a.sf) a.sf[((int64_t)tl.r * tl.nc + tl.c) * 128 + (r & 31) * 4 + (r >> 5)] = (rbase + myrow < a.rows) ? sf_word(s) : 0x7F7F7F7Fu;
+            if (rbase + myrow < a.rows) a.scales[(int64_t)tl.c * a.rows + rbase + myrow] = s;   // scales[tile j][row]
+        }
+    }
+    __syncwarp();
+    const float4 s0 = *reinterpret_cast<const float4 *>(&sh.row_scale[8 * ty]);
+    const float4 s1 = *reinterpret_cast<const float4 *>(&sh.row_scale[8 * ty + 4]);
+    const float4 n0 = *reinterpret_cast<const float4 *>(&sh.row_ninv[8 * ty]);
+    const float4 n1 = *reinterpret_cast<const float4 *>(&sh.row_ninv[8 * ty + 4]);
+    sc.s_row[0] = s0.x; sc.s_row[1] = s0.y; sc.s_row[2] = s0.z; sc.s_row[3] = s0.w;
+    sc.s_row[4] = s1.x; sc.s_row[5] = s1.y; sc.s_row[6] = s1.z; sc.s_row[7] = s1.w;
+    sc.n_row[0] = n0.x; sc.n_row[1] = n0.y; sc.n_row[2] = n0.z; sc.n_row[3] = n0.w;
+    sc.n_row[4] = n1.x; sc.n_row[5] = n1.y; sc.n_row[6] = n1.z; sc.n_row[7] = n1.w;
+}
+
+// Column scales: thread tid < 128 owns column tid of the tile (its maximum is in sh.col_amax), publishes
+// scale and -1/S through shared memory and writes the global scale / atom word.  Two barriers inside.
+template <class O>
+__device__ __forceinline__ void col_scales(const QuantArgs &a, const Tile &tl, QuantShared &sh, int tid, int tx, int64_t c0, SubScales &sc)
+{
+    __syncthreads();   // sh.col_amax complete
+    if (tid < kTile) {
+        const uint16_t *h = reinterpret_cast<const uint16_t *>(&sh.col_amax[0][0]);
+        uint32_t m = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) m = max(m, (uint32_t)h[w * kTile + tid] & 0x7FFFu);  // non-negative bf16: integer order
+        const float am = __uint_as_float(m << 16);
+        const float s = tile_scale<O::FMT>(am, a.pow2);
+        sh.col_scale[tid] = s;
+        sh.col_ninv[tid] = neg_inv<O::FMT>(am, s, a.pow2);
+        // atom [column tile][row tile] (the operand is consumed transposed): one word per column
+        if (O::CODES && a.sf) a.sf[((int64_t)tl.c * tl.nr + tl.r) * 128 + (tid & 31) * 4 + (tid >> 5)] = (c0 + tid < a.cols) ? sf_word(s) : 0x7F7F7F7Fu;
+        if (O::CODES && c0 + tid < a.cols) a.scales[(int64_t)tl.r * a.cols + c0 + tid] = s;
+    }
+    __syncthreads();
+    const float4 s0 = *reinterpret_cast<const float4 *>(&sh.col_scale[8 * tx]);
+    const float4 s1 = *reinterpret_cast<const float4 *>(&sh.col_scale[8 * tx + 4]);
+    const float4 n0 = *reinterpret_cast<const float4 *>(&sh.col_ninv[8 * tx]);
+    const float4 n1 = *reinterpret_cast<const float4 *>(&sh.col_ninv[8 * tx + 4]);
+    sc.s_col[0] = s0.x; sc.s_col[1] = s0.y; sc.s_col[2] = s0.z; sc.s_col[3] = s0.w;
+    sc.s_col[4] = s1.x; sc.s_col[5] = s1.y; sc.s_col[6] = s1.z; sc.s_col[7] = s1.w;
+    sc.n_col[0] = n0.x; sc.n_col[1] = n0.y; sc.n_col[2] = n0.z; sc.n_col[3] = n0.w;
+    sc.n_col[4] = n1.x; sc.n_col[5] = n1.y; sc.n_col[6] = n1.z; sc.n_col[7] = n1.w;
+}
+
+template <class O>
+__device__ __forceinline__ void blk_scales(const QuantArgs &a, const Tile &tl, float blk_am, int tid, SubScales &sc)
+{
+    sc.s_blk = tile_scale<O::FMT>(blk_am, a.pow2);
+    sc.n_blk = neg_inv<O::FMT>(blk_am, sc.s_blk, a.pow2);
+    if (O::CODES && a.sf && tid < kTile) {
+        const int64_t atom = O::TRANSPOSED ? (int64_t)tl.c * tl.nr + tl.r : (int64_t)tl.r * tl.nc + tl.c;
+        a.sf[atom * 128 + tid] = sf_word(sc.s_blk);
+    }
+    if (O::CODES && tid == 0) a.scales[(int64_t)tl.r * tl.nc + tl.c] = sc.s_blk;
+}
+
+// One tile, up to two outputs (A, B), everything from the thread's 8x8 sub-block in slot[p * kThreads].
+// A and B: Out<...> or NoOut.  ROWSTATS (per-row sums) refers to output A.  after_reads() is called once
+// the last read of the slot has been issued (the caller starts the next tile's fetch there).
+template <class A, class B, bool STATS, bool ROWSTATS, class AfterReads>
+__device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArgs &qb, const Tile &tl, const uint4 *slot, QuantShared &sh,
+                                             ThreadStats &ts, AfterReads after_reads)
+{
+    static_assert(!(A::TRANSPOSED && B::TRANSPOSED), "one transposed output per pass");
+    constexpr bool kRow = (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128) || (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128);
+    constexpr bool kCol = (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_128x1) || (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_128x1);
+    constexpr bool kBlk = (A::kQuant && A::BLOCK == SNIP_BLOCK_BLK_128x128) || (B::kQuant && B::BLOCK == SNIP_BLOCK_BLK_128x128);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tx = tid & 15, ty = tid >> 4;
     const int64_t r0 = (int64_t)tl.r * kTile, c0 = (int64_t)tl.c * kTile;
     const int64_t rbase = r0 + 8 * ty, cbase = c0 + 8 * tx;
-    const bool col_ok = cbase < a.cols;  // cols is a multiple of 64, so 8-groups never straddle
+    const bool in_range = cbase < qa.cols && rbase < qa.rows;   // dims are multiples of 64: all 64 elements or none
 
-    // ---- block amax -> scales --------------------------------------------------------
-    float s_row[8], s_col[8];  // scale per row p (ROW) / per column j (COL); BLK uses s_row[0]
-    float n_row[8], n_col[8];  // matching -1/S for the error term
-    (void)s_row; (void)s_col; (void)n_row; (void)n_col;
-    float my_amax = 0.0f;      // this thread's amax, for the tensor-wide statistic
-    if (kQuant || STATS) {
-        uint32_t rmax[8];      // per row: packed max over the 8 columns (as 4 pairs folded)
+    // ---- maxima (signs are garbage until masked: max.xorsign.abs keeps magnitudes only) -----------
+    SubScales sa, sb;
+    {
+        uint32_t rmax[8], cm[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
             const uint4 vp = slot[p * kThreads];
-            uint32_t m = absmax2(0u, vp.x);
-            m = absmax2(m, vp.y);
-            m = absmax2(m, vp.z);
-            m = absmax2(m, vp.w);
-            rmax[p] = m;
+            if (kRow) rmax[p] = absmax2x(absmax2x(vp.x, vp.y), absmax2x(vp.z, vp.w));
+            if (kCol || kBlk || !kRow) {
+                cm[0] = absmax2x(cm[0], vp.x);
+                cm[1] = absmax2x(cm[1], vp.y);
+                cm[2] = absmax2x(cm[2], vp.z);
+                cm[3] = absmax2x(cm[3], vp.w);
+            }
         }
-        if (BLOCK == SNIP_BLOCK_ROW_1x128 && kQuant) {
-            // fold pairs, pack two rows per register, reduce across the 16 lanes of the row
-            uint32_t pk[4];
+        if (kRow) {
+            static_assert(!(A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128 && B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128), "one row-tiled output per pass");
+            float am = 0.0f;
+            if (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128) row_scales<A>(qa, tl, sh, rmax, tx, ty, rbase, sa, am);
+            if (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128) row_scales<B>(qb, tl, sh, rmax, tx, ty, rbase, sb, am);
+            if (STATS) ts.amax = fmaxf(ts.amax, am);
+        }
+        if (kCol) {
+            // the two row groups of a warp, then the 8 warps through shared memory
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t m0 = rmax[2 * q], m1 = rmax[2 * q + 1];
-                m0 = max2(m0, m0 >> 16);  // low half = row 2q
-                m1 = max2(m1, m1 << 16);  // high half = row 2q+1
-                pk[q] = (m0 & 0xFFFFu) | (m1 & 0xFFFF0000u);
-            }
-#pragma unroll
-            for (int off = 1; off < 16; off <<= 1)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) pk[q] = max2(pk[q], __shfl_xor_sync(0xFFFFFFFFu, pk[q], off));
-            // lane (tx & 7) derives the scale of row p = tx & 7, then the 8 scales are shared
-            const int myp = tx & 7;
-            uint32_t sel = pk[0];
-#pragma unroll
-            for (int q = 1; q < 4; ++q) sel = ((myp >> 1) == q) ? pk[q] : sel;
-            float am = (myp & 1) ? bf16hi(sel) : bf16lo(sel);
-            float mine = tile_scale<FMT>(am, a.pow2);
-            float mine_ninv = neg_inv_scale<FMT>(am, mine, a.pow2);
-#pragma unroll
-            for (int p = 0; p < 8; ++p) {
-                s_row[p] = __shfl_sync(0xFFFFFFFFu, mine, (lane & 16) | p);
-                if (STATS) n_row[p] = __shfl_sync(0xFFFFFFFFu, mine_ninv, (lane & 16) | p);
-            }
-            if (STATS) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) my_amax = fmaxf(my_amax, fmaxf(bf16lo(pk[q]), bf16hi(pk[q])));
-            }
-            if (CODES && tx == 0 && a.sf) {
-                // atom [row tile][column tile]: word (r % 32) * 4 + r / 32 holds row r's byte four times
-                uint32_t *atom = a.sf + ((int64_t)tl.r * tl.nc + tl.c) * 128;
-#pragma unroll
-                for (int p = 0; p < 8; ++p) {
-                    const int r = 8 * ty + p;
-                    atom[(r & 31) * 4 + (r >> 5)] = (rbase + p < a.rows) ? sf_word(s_row[p]) : 0x7F7F7F7Fu;
-                }
-            }
-            if (CODES && tx == 0) {
-                // scales[tile j][row]: eight consecutive rows per thread
-                float *dst = a.scales + (int64_t)tl.c * a.rows + rbase;
-                if (rbase < a.rows) {
-                    *reinterpret_cast<float4 *>(dst) = make_float4(s_row[0], s_row[1], s_row[2], s_row[3]);
-                    *reinterpret_cast<float4 *>(dst + 4) = make_float4(s_row[4], s_row[5], s_row[6], s_row[7]);
-                }
-            }
-        } else {
-            // column maxima over this thread's 8 rows (4 packed registers = 8 columns)
-            uint32_t cm[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (int p = 0; p < 8; ++p) {
-                const uint4 vp = slot[p * kThreads];
-                cm[0] = absmax2(cm[0], vp.x);
-                cm[1] = absmax2(cm[1], vp.y);
-                cm[2] = absmax2(cm[2], vp.z);
-                cm[3] = absmax2(cm[3], vp.w);
-            }
-            if (BLOCK == SNIP_BLOCK_COL_128x1 && kQuant) {
-                // the two row groups of a warp, then the 8 warps through shared memory
-#pragma unroll
-                for (int q = 0; q < 4; ++q) cm[q] = max2(cm[q], __shfl_xor_sync(0xFFFFFFFFu, cm[q], 16));
-                if (lane < 16)
-                    *reinterpret_cast<uint4 *>(&col_amax[warp][4 * tx]) = make_uint4(cm[0], cm[1], cm[2], cm[3]);
+            for (int q = 0; q < 4; ++q) cm[q] = absmax2x(cm[q], __shfl_xor_sync(0xFFFFFFFFu, cm[q], 16));
+            if (lane < 16) *reinterpret_cast<uint4 *>(&sh.col_amax[warp][4 * tx]) = make_uint4(cm[0], cm[1], cm[2], cm[3]);
+            if (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_128x1) col_scales<A>(qa, tl, sh, tid, tx, c0, sa);
+            if (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_128x1) col_scales<B>(qb, tl, sh, tid, tx, c0, sb);
+        }
+        if (kBlk || (!kRow && STATS)) {
+            uint32_t m = absmax2x(absmax2x(cm[0], cm[1]), absmax2x(cm[2], cm[3])) & 0x7FFF7FFFu;
+            m = max(m & 0xFFFFu, m >> 16);
+            if (!kRow && STATS) ts.amax = fmaxf(ts.amax, __uint_as_float(m << 16));
+            if (kBlk) {
+                m = __reduce_max_sync(0xFFFFFFFFu, m);
+                if (lane == 0) sh.red_m[warp] = m;
                 __syncthreads();
-                if (tid < kTile) {
-                    const uint16_t *h = reinterpret_cast<const uint16_t *>(&col_amax[0][0]);
-                    uint32_t m = 0;
+                uint32_t bm = sh.red_m[0];
 #pragma unroll
-                    for (int w = 0; w < 8; ++w) m = max(m, (uint32_t)h[w * kTile + tid]);  // non-negative bf16: integer order
-                    float am = __uint_as_float(m << 16);
-                    float s = tile_scale<FMT>(am, a.pow2);
-                    col_scale[tid] = s;
-                    col_ninv[tid] = neg_inv_scale<FMT>(am, s, a.pow2);
-                    // atom [column tile][row tile] (the operand is consumed transposed): one word per column
-                    if (CODES && a.sf) a.sf[((int64_t)tl.c * tl.nr + tl.r) * 128 + (tid & 31) * 4 + (tid >> 5)] = (c0 + tid < a.cols) ? sf_word(s) : 0x7F7F7F7Fu;
-                    if (CODES && c0 + tid < a.cols) a.scales[(int64_t)tl.r * a.cols + c0 + tid] = s;
-                    if (STATS) my_amax = am;
-                }
-                __syncthreads();
-                const float4 s0 = *reinterpret_cast<const float4 *>(&col_scale[8 * tx]);
-                const float4 s1 = *reinterpret_cast<const float4 *>(&col_scale[8 * tx + 4]);
-                s_col[0] = s0.x; s_col[1] = s0.y; s_col[2] = s0.z; s_col[3] = s0.w;
-                s_col[4] = s1.x; s_col[5] = s1.y; s_col[6] = s1.z; s_col[7] = s1.w;
-                if (STATS) {
-                    const float4 n0 = *reinterpret_cast<const float4 *>(&col_ninv[8 * tx]);
-                    const float4 n1 = *reinterpret_cast<const float4 *>(&col_ninv[8 * tx + 4]);
-                    n_col[0] = n0.x; n_col[1] = n0.y; n_col[2] = n0.z; n_col[3] = n0.w;
-                    n_col[4] = n1.x; n_col[5] = n1.y; n_col[6] = n1.z; n_col[7] = n1.w;
-                }
-            } else {
-                // BLK (or statistics-only): one amax for the whole CTA tile
-                uint32_t m = max2(max2(cm[0], cm[1]), max2(cm[2], cm[3]));
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) m = max2(m, __shfl_xor_sync(0xFFFFFFFFu, m, off));
-                float am = fmaxf(bf16lo(m), bf16hi(m));
-                if (lane == 0) red_f[warp][2] = am;
-                __syncthreads();
-                float bm = red_f[0][2];
-#pragma unroll
-                for (int w = 1; w < 8; ++w) bm = fmaxf(bm, red_f[w][2]);
-                my_amax = bm;
-                if (kQuant) {
-                    s_row[0] = tile_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm, a.pow2);
-                    n_row[0] = neg_inv_scale<FMT == SNIP_FMT_BF16 ? SNIP_FMT_FP8_E4M3 : FMT>(bm, s_row[0], a.pow2);
-                    if (CODES && a.sf && tid < kTile) {
-                        const int64_t atom = TRANSPOSED ? (int64_t)tl.c * tl.nr + tl.r : (int64_t)tl.r * tl.nc + tl.c;
-                        a.sf[atom * 128 + tid] = sf_word(s_row[0]);
-                    }
-                    if (CODES && tid == 0) a.scales[(int64_t)tl.r * tl.nc + tl.c] = s_row[0];
-                }
-                __syncthreads();  // red_f is reused below
+                for (int w = 1; w < 8; ++w) bm = max(bm, sh.red_m[w]);
+                const float blk_am = __uint_as_float(bm << 16);
+                if (A::kQuant && A::BLOCK == SNIP_BLOCK_BLK_128x128) blk_scales<A>(qa, tl, blk_am, tid, sa);
+                if (B::kQuant && B::BLOCK == SNIP_BLOCK_BLK_128x128) blk_scales<B>(qb, tl, blk_am, tid, sb);
             }
         }
     }
 
-    // ---- encode, statistics, store ------------------------------------------------------
-    float sx = 0.0f, se = 0.0f;
+    // ---- encode, statistics, as-stored codes ------------------------------------------------------
+    uint32_t keep[8][2];   // codes of the transposed output, held until the sub-block is complete
+    (void)keep;
+    float2 sx2 = make_float2(0.0f, 0.0f), sea2 = make_float2(0.0f, 0.0f), seb2 = make_float2(0.0f, 0.0f);
     float rsx[8], rse[8];
     (void)rsx; (void)rse;
-    if (kQuant) {
-        float2 sc[4], ni[4];
-        if (BLOCK == SNIP_BLOCK_COL_128x1) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { sc[j] = make_float2(s_col[2 * j], s_col[2 * j + 1]); ni[j] = make_float2(n_col[2 * j], n_col[2 * j + 1]); }
-        } else if (BLOCK == SNIP_BLOCK_BLK_128x128) {
+    for (int p = 0; p < 8; ++p) {
+        const uint4 vp = slot[p * kThreads];
+        const uint32_t w[4] = {vp.x, vp.y, vp.z, vp.w};
+        uint32_t ca[4], cb[4];
+        float2 px = make_float2(0.0f, 0.0f), pe = make_float2(0.0f, 0.0f);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { sc[j] = make_float2(s_row[0], s_row[0]); ni[j] = make_float2(n_row[0], n_row[0]); }
+        for (int i = 0; i < 4; ++i) {
+            const float2 x = make_float2(bf16lo(w[i]), bf16hi(w[i]));
+            if (STATS) { if (ROWSTATS) px = __ffma2_rn(x, x, px); else sx2 = __ffma2_rn(x, x, sx2); }
+            if (A::kQuant) ca[i] = encode_pair<A::FMT, STATS>(x, scale_pair<A>(sa, p, i), ninv_pair<A>(sa, p, i), ROWSTATS ? pe : sea2);
+            if (B::kQuant) cb[i] = encode_pair<B::FMT, STATS>(x, scale_pair<B>(sb, p, i), ninv_pair<B>(sb, p, i), seb2);
         }
-        uint32_t codes[8][2];
-        float2 sx2 = make_float2(0.0f, 0.0f), se2 = make_float2(0.0f, 0.0f);
-#pragma unroll
-        for (int p = 0; p < 8; ++p) {
-            if (BLOCK == SNIP_BLOCK_ROW_1x128) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { sc[j] = make_float2(s_row[p], s_row[p]); ni[j] = make_float2(n_row[p], n_row[p]); }
-            }
-            if (ROWSTATS) {
-                float2 px = make_float2(0.0f, 0.0f), pe = make_float2(0.0f, 0.0f);
-                quant8<FMT, STATS>(slot[p * kThreads], sc, ni, codes[p], px, pe);
-                rsx[p] = px.x + px.y; rse[p] = pe.x + pe.y;
-                sx += rsx[p]; se += rse[p];
-            } else {
-                quant8<FMT, STATS>(slot[p * kThreads], sc, ni, codes[p], sx2, se2);
-            }
+        if (ROWSTATS) {
+            rsx[p] = px.x + px.y; rse[p] = pe.x + pe.y;
+            sx2.x += rsx[p]; sea2.x += rse[p];
         }
-        if (STATS && !ROWSTATS) { sx = sx2.x + sx2.y; se = se2.x + se2.y; }
-        if (CODES) {
-            if (!TRANSPOSED) {
-                const int64_t out_ld = a.cols * kCodeBytes8 / 8;  // bytes per output row
-                if (col_ok && rbase < a.rows) {
-                    uint8_t *dst = a.codes + rbase * out_ld + cbase * kCodeBytes8 / 8;
-                    const uint32_t ld32 = (uint32_t)out_ld;
-#pragma unroll
-                    for (int p = 0; p < 8; ++p) {
-                        if (FMT == SNIP_FMT_FP8_E4M3)
-                            *reinterpret_cast<uint2 *>(dst + p * ld32) = make_uint2(codes[p][0], codes[p][1]);
-                        else
-                            *reinterpret_cast<uint32_t *>(dst + p * ld32) = codes[p][0];
-                    }
-                }
-            } else {
-                // Transpose the 8x8 sub-block of codes in registers: for column j collect the
-                // codes of rows p = 0..7, then stage line (8*tx + j) of the transposed tile.
-                // Chunk index ty is XOR-ed with tx so that the 16 lanes of a row group hit
-                // distinct banks.
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint32_t lo = 0, hi = 0;
-                    if (FMT == SNIP_FMT_FP8_E4M3) {
-#pragma unroll
-                        for (int p = 0; p < 8; ++p) {
-                            uint32_t b = (codes[p][j >> 2] >> (8 * (j & 3))) & 0xFFu;
-                            if (p < 4) lo |= b << (8 * p); else hi |= b << (8 * (p - 4));
-                        }
-                        uint2 *dst = reinterpret_cast<uint2 *>(stage + (8 * tx + j) * kRowBytes) + (ty ^ tx);
-                        *dst = make_uint2(lo, hi);
-                    } else {
-#pragma unroll
-                        for (int p = 0; p < 8; ++p) {
-                            uint32_t b = (codes[p][0] >> (4 * j)) & 0xFu;
-                            lo |= b << (4 * p);
-                        }
-                        uint32_t *dst = reinterpret_cast<uint32_t *>(stage + (8 * tx + j) * kRowBytes) + (ty ^ tx);
-                        *dst = lo;
-                    }
-                }
-                __syncthreads();
-                // write out: line c of the staged tile holds rows r0..r0+127 of column c0+c
-                const int64_t out_ld = a.rows * kCodeBytes8 / 8;  // bytes per transposed row
-                constexpr int kChunks = kRowBytes / 16;            // 16-byte chunks per line
-                const int valid_rows = (int)min((int64_t)kTile, a.rows - r0);
-                for (int idx = tid; idx < kTile * kChunks; idx += kThreads) {
-                    const int c = idx / kChunks, q = idx % kChunks;
-                    if (c0 + c >= a.cols) continue;
-                    const int key = (c >> 3) & 15;
-                    uint4 o;
-                    if (FMT == SNIP_FMT_FP8_E4M3) {
-                        const uint2 *src = reinterpret_cast<const uint2 *>(stage + c * kRowBytes);
-                        uint2 h0 = src[(2 * q) ^ key], h1 = src[(2 * q + 1) ^ key];
-                        o = make_uint4(h0.x, h0.y, h1.x, h1.y);
-                        if (16 * q >= valid_rows) continue;  // rows is a multiple of 64
-                    } else {
-                        const uint32_t *src = reinterpret_cast<const uint32_t *>(stage + c * kRowBytes);
-                        o = make_uint4(src[(4 * q) ^ key], src[(4 * q + 1) ^ key], src[(4 * q + 2) ^ key],
-                                       src[(4 * q + 3) ^ key]);
-                        if (32 * q >= valid_rows) continue;
-                    }
-                    uint8_t *dst = a.codes + (c0 + c) * out_ld + r0 * kCodeBytes8 / 8 + 16 * q;
-                    *reinterpret_cast<uint4 *>(dst) = o;
-                }
-            }
+        if (A::kQuant && A::CODES) {
+            uint32_t code[2];
+            pack8<A::FMT>(ca, code);
+            if (A::TRANSPOSED) { keep[p][0] = code[0]; keep[p][1] = code[1]; }
+            else if (in_range) store_row<A::FMT>(qa, rbase, cbase, p, code);
         }
-    } else if (STATS) {
-        // BF16: identity, only sum x^2
-#pragma unroll
-        for (int p = 0; p < 8; ++p) {
-            const uint4 vp = slot[p * kThreads];
-            const uint32_t w[4] = {vp.x, vp.y, vp.z, vp.w};
-            float px = 0.0f;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float x0 = bf16lo(w[i]), x1 = bf16hi(w[i]);
-                px = fmaf(x0, x0, px);
-                px = fmaf(x1, x1, px);
-            }
-            sx += px;
-            if (ROWSTATS) { rsx[p] = px; rse[p] = 0.0f; }
+        if (B::kQuant && B::CODES) {
+            uint32_t code[2];
+            pack8<B::FMT>(cb, code);
+            if (B::TRANSPOSED) { keep[p][0] = code[0]; keep[p][1] = code[1]; }
+            else if (in_range) store_row<B::FMT>(qb, rbase, cbase, p, code);
         }
     }
+    after_reads();
 
-    // ---- statistics: warp -> CTA -> one partial per CTA ------------------------------------
+    if (STATS) {
+        ts.x += (double)(sx2.x + sx2.y);
+        if (A::kQuant) ts.ea += (double)(sea2.x + sea2.y);
+        if (B::kQuant) ts.eb += (double)(seb2.x + seb2.y);
+    }
     if (ROWSTATS) {
-        // per row: add the 16 lanes that share the row, lane tx==0 writes {sum x^2, sum err^2}
+        // per row: add the 16 lanes that share the row, lane tx == 0 writes {sum x^2, sum err^2}
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
 #pragma unroll
@@ -367,29 +463,52 @@ __device__ __forceinline__ void quantize_tile(const QuantArgs &a, const Tile &tl
                 rse[p] += __shfl_xor_sync(0xFFFFFFFFu, rse[p], off);
             }
         }
-        if (tx == 0 && rbase < a.rows) {
-            float2 *dst = a.row_partials + (int64_t)tl.c * a.rows + rbase;
+        if (tx == 0 && rbase < qa.rows) {
+            float2 *dst = qa.row_partials + (int64_t)tl.c * qa.rows + rbase;
 #pragma unroll
             for (int p = 0; p < 8; ++p) dst[p] = make_float2(rsx[p], rse[p]);
         }
     }
-    if (STATS) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            sx += __shfl_xor_sync(0xFFFFFFFFu, sx, off);
-            se += __shfl_xor_sync(0xFFFFFFFFu, se, off);
-            my_amax = fmaxf(my_amax, __shfl_xor_sync(0xFFFFFFFFu, my_amax, off));
-        }
-        if (lane == 0) { red_f[warp][0] = sx; red_f[warp][1] = se; red_f[warp][2] = my_amax; }
+
+    // ---- transposed codes: registers -> swizzled shared tile -> coalesced 16-byte stores ------------
+    if (A::kQuant && A::CODES && A::TRANSPOSED) {
+        stage_transposed<A::FMT>(sh.stage, tx, ty, keep);
         __syncthreads();
-        if (tid == 0) {
-            double dx = 0.0, de = 0.0;
-            float am = 0.0f;
+        write_transposed<A::FMT>(qa, sh.stage, r0, c0);
+    }
+    if (B::kQuant && B::CODES && B::TRANSPOSED) {
+        stage_transposed<B::FMT>(sh.stage, tx, ty, keep);
+        __syncthreads();
+        write_transposed<B::FMT>(qb, sh.stage, r0, c0);
+    }
+}
+
+// End of a CTA's walk: its threads' sums -> one CtaPartial per output (warp shuffles, then warp order).
+template <bool HAS_B>
+__device__ __forceinline__ void finish_stats(const ThreadStats &ts, QuantShared &sh, CtaPartial *pa, CtaPartial *pb)
+{
+    double x = ts.x, ea = ts.ea, eb = ts.eb;
+    float am = ts.amax;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) { dx += (double)red_f[w][0]; de += (double)red_f[w][1]; am = fmaxf(am, red_f[w][2]); }
-            acc.x += dx;
-            acc.e += de;
-            acc.m = fmaxf(acc.m, am);
+    for (int off = 16; off > 0; off >>= 1) {
+        x += __shfl_xor_sync(0xFFFFFFFFu, x, off);
+        ea += __shfl_xor_sync(0xFFFFFFFFu, ea, off);
+        if (HAS_B) eb += __shfl_xor_sync(0xFFFFFFFFu, eb, off);
+        am = fmaxf(am, __shfl_xor_sync(0xFFFFFFFFu, am, off));
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();   // the scratch of the last tile is no longer in use
+    if (lane == 0) { sh.red_d[warp][0] = x; sh.red_d[warp][1] = ea; sh.red_d[warp][2] = eb; sh.red_d[warp][3] = (double)am; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double tx_ = 0.0, ta = 0.0, tb = 0.0, tm = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { tx_ += sh.red_d[w][0]; ta += sh.red_d[w][1]; tb += sh.red_d[w][2]; tm = fmax(tm, sh.red_d[w][3]); }
+        CtaPartial *d = pa + blockIdx.x;
+        d->sumsq_x = tx_; d->sumsq_err = ta; d->amax = (float)tm;
+        if (HAS_B) {
+            d = pb + blockIdx.x;
+            d->sumsq_x = tx_; d->sumsq_err = tb; d->amax = (float)tm;
         }
     }
 }
@@ -397,16 +516,6 @@ __device__ __forceinline__ void quantize_tile(const QuantArgs &a, const Tile &tl
 // Dynamic shared memory of the kernels: the tile slot, then the QuantShared scratch.
 constexpr size_t kSmemBytes = (size_t)kStageBytes + sizeof(QuantShared);
 constexpr int kCtasPerSm = 4;
-
-__device__ __forceinline__ void write_partial(CtaPartial *partials, const StatsAcc &acc)
-{
-    if (threadIdx.x == 0) {
-        CtaPartial *dst = partials + blockIdx.x;
-        dst->sumsq_x = acc.x;
-        dst->sumsq_err = acc.e;
-        dst->amax = acc.m;
-    }
-}
 
 // Walk of one CTA over its tiles without divisions in the loop.
 struct TileWalk {
@@ -433,20 +542,21 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
     // the statistics reduction that follows on the stream may be scheduled now; it waits for this
     // grid to finish before it reads anything (programmatic dependent launch)
     if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    StatsAcc acc;
+    ThreadStats ts;
     TileWalk w((int)a.tiles_r, (int)a.tiles_c);
     if (w.valid()) prefetch_tile(a, w.r, w.c, smem);
     prefetch_commit();
     while (w.valid()) {
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
-        quantize_tile<FMT, BLOCK, TRANSPOSED, CODES, STATS, ROWSTATS>(a, tl, slot, sh, acc);
         w.next();
-        if (w.valid()) prefetch_tile(a, w.r, w.c, smem);   // this thread's reads of its slot are done
-        prefetch_commit();
+        process_tile<Out<FMT, BLOCK, TRANSPOSED, CODES>, NoOut, STATS, ROWSTATS>(a, a, tl, slot, sh, ts, [&] {
+            if (w.valid()) prefetch_tile(a, w.r, w.c, smem);   // this thread's reads of its slot are done
+            prefetch_commit();
+        });
         __syncthreads();  // the scratch arrays are reused by the next tile
     }
-    if (STATS) write_partial(a.partials, acc);
+    if (STATS) finish_stats<false>(ts, sh, a.partials, nullptr);
 }
 
 // Two outputs from one read (the tile kinds a tensor is consumed with, paper Fig. 5): `a` as stored
@@ -462,22 +572,23 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_dual_kernel(con
     QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
     const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
     if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    StatsAcc acc_a, acc_b;
+    ThreadStats ts;
     TileWalk w((int)d.a.tiles_r, (int)d.a.tiles_c);
     if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
     prefetch_commit();
     while (w.valid()) {
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
-        quantize_tile<FMT_A, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true, STATS, false>(d.a, tl, slot, sh, acc_a);
-        __syncthreads();  // the scratch arrays are reused by the second output
-        quantize_tile<FMT_B, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true, STATS, false>(d.b, tl, slot, sh, acc_b);
         w.next();
-        if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
-        prefetch_commit();
+        using A = Out<FMT_A, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true>;
+        using B = Out<FMT_B, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true>;
+        process_tile<A, B, STATS, false>(d.a, d.b, tl, slot, sh, ts, [&] {
+            if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
+            prefetch_commit();
+        });
         __syncthreads();
     }
-    if (STATS) { write_partial(d.a.partials, acc_a); write_partial(d.b.partials, acc_b); }
+    if (STATS) finish_stats<true>(ts, sh, d.a.partials, d.b.partials);
 }
 
 // Fixed-order reduction of the per-CTA partials into one snip_stats_t (deterministic: every thread
