@@ -515,7 +515,11 @@ __device__ __forceinline__ void finish_stats(const ThreadStats &ts, QuantShared 
 
 // Dynamic shared memory of the kernels: the tile slot, then the QuantShared scratch.
 constexpr size_t kSmemBytes = (size_t)kStageBytes + sizeof(QuantShared);
+#ifndef SNIP_DUAL_CTAS
+#define SNIP_DUAL_CTAS 3
+#endif
 constexpr int kCtasPerSm = 4;
+constexpr int kDualCtasPerSm = SNIP_DUAL_CTAS;
 
 // Walk of one CTA over its tiles without divisions in the loop.
 struct TileWalk {
@@ -566,7 +570,7 @@ struct DualArgs {
     QuantArgs a, b;
 };
 template <int FMT_A, int FMT_B, bool BLK, bool STATS>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_dual_kernel(const DualArgs d)
+__global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel(const DualArgs d)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
@@ -685,9 +689,9 @@ void launch_fmt(const QuantArgs &a, int block, bool transposed, bool codes, bool
 
 // CTAs of a persistent launch over ntiles tiles: kCtasPerSm per SM (what the kernels' shared memory and
 // registers allow), never more than there are tiles.
-int64_t persistent_ctas(int64_t ntiles)
+int64_t persistent_ctas(int64_t ntiles, int per_sm = kCtasPerSm)
 {
-    const int64_t cap = kCtasPerSm * (int64_t)gemm_sm_count();
+    const int64_t cap = per_sm * (int64_t)gemm_sm_count();
     return ntiles < cap ? ntiles : cap;
 }
 
@@ -823,7 +827,7 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bo
         q.sf = static_cast<uint32_t *>(o[i]->sf);
         q.tiles_r = tr; q.tiles_c = tc; q.ntiles = tr * tc;
     }
-    const int64_t nparts = persistent_ctas(tr * tc);
+    const int64_t nparts = persistent_ctas(tr * tc, kDualCtasPerSm);
     dim3 grid((unsigned)nparts);
     const bool a8 = oa.fmt == SNIP_FMT_FP8_E4M3, b8 = ob.fmt == SNIP_FMT_FP8_E4M3;
     if (a8 && b8) launch_dual<SNIP_FMT_FP8_E4M3, SNIP_FMT_FP8_E4M3>(d, blk, stats, grid, st);
