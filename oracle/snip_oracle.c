@@ -200,6 +200,82 @@ float orc_tile_scale_pow2(int fmt, float amax)
 /* Quantizer                                                                                 */
 /* ---------------------------------------------------------------------------------------- */
 
+/* ---- stochastic rounding (Sec. 6.1: FP4 output gradients are rounded probabilistically to one of
+ * the two nearest representable values) ------------------------------------------------------
+ *
+ * The paper names the method and cites it; the concrete rule used here (a reading): with
+ * a = min(|t|, FPX_MAX) and lo <= a < hi the neighbouring representable magnitudes (subnormals
+ * included; a == FPX_MAX stays), round to hi iff (a - lo) / (hi - lo) > (u + 1/2) / 2^16, where u
+ * is a 16-bit uniform integer owned by the element; the sign bit is copied from t.  A representable
+ * a has fraction 0 and never moves.  P(round up) equals the fraction to within 2^-17.
+ *
+ * The uniforms come from the counter-based generator Philox4x32 with 10 rounds (Salmon, Moraes,
+ * Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", 2011): counter = (idx / 8 as two
+ * 32-bit words, 0, 0), key = the two words of the seed; its four output words hold the eight
+ * uniforms of elements 8*(idx/8) .. +7, element j in bits [16*(j%2), 16*(j%2)+16) of word j/2.
+ */
+static void orc_mulhilo32(uint32_t a, uint32_t b, uint32_t *hi, uint32_t *lo)
+{
+    uint64_t p = (uint64_t)a * (uint64_t)b;
+    *hi = (uint32_t)(p >> 32);
+    *lo = (uint32_t)p;
+}
+
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint32_t hi0, lo0, hi1, lo1;
+        orc_mulhilo32(0xD2511F53u, c0, &hi0, &lo0);
+        orc_mulhilo32(0xCD9E8D57u, c2, &hi1, &lo1);
+        uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u; /* key schedule: golden-ratio and sqrt(3)-1 increments */
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+uint32_t orc_sr_uniform16(uint64_t seed, uint64_t idx)
+{
+    uint64_t blk = idx / 8;
+    uint32_t ctr[4] = {(uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t w[4];
+    orc_philox4x32_10(ctr, key, w);
+    unsigned j = (unsigned)(idx % 8);
+    return (w[j / 2] >> (16 * (j % 2))) & 0xFFFFu;
+}
+
+/* Stochastically rounded code of the binary32 value t given the element's 16-bit uniform u.  The
+ * neighbours are found by scanning the table of representable magnitudes (obviously correct, slow). */
+static unsigned orc_encode_sr_fmt(const orc_minifloat_t *f, float t, uint32_t u)
+{
+    unsigned sign = signbit(t) ? 1u : 0u;
+    double a = fabs((double)t);
+    unsigned nmag = 1u << (f->ebits + f->mbits);      /* magnitude codes 0 .. nmag-1 */
+    unsigned top = 0;                                  /* largest magnitude code in use (E4M3: 0x7E, 0x7F is NaN) */
+    for (unsigned m = 0; m < nmag; ++m)
+        if (orc_decode(f, m) <= f->max_value) top = m;
+    double vmax = orc_decode(f, top);
+    if (a >= vmax) return (sign << (f->ebits + f->mbits)) | top;
+    unsigned lo = 0;
+    for (unsigned m = 0; m <= top; ++m)
+        if (orc_decode(f, m) <= a) lo = m;             /* magnitudes ascend with the code */
+    double vlo = orc_decode(f, lo), vhi = orc_decode(f, lo + 1);
+    double frac = (a - vlo) / (vhi - vlo);
+    double thr = ((double)u + 0.5) / 65536.0;
+    unsigned mag = frac > thr ? lo + 1 : lo;
+    return (sign << (f->ebits + f->mbits)) | mag;
+}
+
+uint8_t orc_encode_sr(int fmt, float t, uint32_t u16)
+{
+    const orc_minifloat_t *f = orc_format(fmt);
+    return f ? (uint8_t)orc_encode_sr_fmt(f, t, u16 & 0xFFFFu) : 0;
+}
+
 static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 /* Shape of the scale tensor for a rows x cols input (Sec. 2.3 granularity):
@@ -242,10 +318,31 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int blo
     return orc_quantize_rule(x, rows, cols, fmt, block, 0, codes, scales, xhat, sumsq, row_sumsq);
 }
 
+static int orc_quantize_impl(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block, int pow2_scale,
+                             int stochastic, uint64_t seed,
+                             uint8_t *codes, float *scales, double *xhat, double *sumsq, double *row_sumsq);
+
 /* Same with the scale rule selectable: pow2_scale = 0 is the paper's quotient FPX_MAX / amax,
  * pow2_scale = 1 the power-of-two option above.  Everything else is identical. */
 int orc_quantize_rule(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block, int pow2_scale,
                       uint8_t *codes, float *scales, double *xhat, double *sumsq, double *row_sumsq)
+{
+    return orc_quantize_impl(x, rows, cols, fmt, block, pow2_scale, 0, 0, codes, scales, xhat, sumsq, row_sumsq);
+}
+
+/* Same with stochastic rounding of the codes (Sec. 6.1: used for FP4 output gradients): element
+ * (r, c) draws the 16-bit uniform orc_sr_uniform16(seed, r * cols + c) and is rounded by
+ * orc_encode_sr.  Scales are unchanged (they depend on amax only). */
+int orc_quantize_sr(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block, int pow2_scale, uint64_t seed,
+                    uint8_t *codes, float *scales, double *xhat, double *sumsq, double *row_sumsq)
+{
+    if (!orc_format(fmt)) return -1;
+    return orc_quantize_impl(x, rows, cols, fmt, block, pow2_scale, 1, seed, codes, scales, xhat, sumsq, row_sumsq);
+}
+
+static int orc_quantize_impl(const uint16_t *x, int64_t rows, int64_t cols, int fmt, int block, int pow2_scale,
+                             int stochastic, uint64_t seed,
+                             uint8_t *codes, float *scales, double *xhat, double *sumsq, double *row_sumsq)
 {
     if (!x || rows < 0 || cols < 0) return -1;
     if (fmt != ORC_FMT_BF16 && !orc_format(fmt)) return -1;
@@ -291,7 +388,8 @@ int orc_quantize_rule(const uint16_t *x, int64_t rows, int64_t cols, int fmt, in
             if (f) {
                 float s = S[orc_scale_index(rows, cols, block, r, c)];
                 volatile float t = xf * s; /* one binary32 rounding, never fused */
-                unsigned code = orc_encode(f, t);
+                unsigned code = stochastic ? orc_encode_sr_fmt(f, t, orc_sr_uniform16(seed, (uint64_t)(r * cols + c)))
+                                           : orc_encode(f, t);
                 if (codes) codes[r * cols + c] = (uint8_t)code;
                 xh = orc_decode(f, code) / (double)s;
             } else {

@@ -61,6 +61,14 @@ def lib() -> ctypes.CDLL:
         L.orc_quantize.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp]
         L.orc_quantize_rule.restype = i32
         L.orc_quantize_rule.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.orc_quantize_sr.restype = i32
+        L.orc_quantize_sr.argtypes = [vp, i64, i64, i32, i32, i32, ctypes.c_uint64, vp, vp, vp, vp, vp]
+        L.orc_philox4x32_10.restype = None
+        L.orc_philox4x32_10.argtypes = [vp, vp, vp]
+        L.orc_sr_uniform16.restype = ctypes.c_uint32
+        L.orc_sr_uniform16.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
+        L.orc_encode_sr.restype = ctypes.c_uint8
+        L.orc_encode_sr.argtypes = [i32, ctypes.c_float, ctypes.c_uint32]
         L.orc_tile_scale_pow2.restype = ctypes.c_float
         L.orc_tile_scale_pow2.argtypes = [i32, ctypes.c_float]
         L.orc_dequantize.restype = i32
@@ -154,7 +162,27 @@ class Quantized:
         return pack_codes(self.codes, self.fmt, transposed)
 
 
-def quantize(x_bits: np.ndarray, fmt: int, block: int, pow2_scale: bool = False) -> Quantized:
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """Four 32-bit outputs of Philox4x32-10 for a 4-word counter and a 2-word key."""
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def sr_uniform16(seed: int, idx: int) -> int:
+    """The 16-bit uniform that element idx (row-major linear index) draws under `seed`."""
+    return int(lib().orc_sr_uniform16(seed, idx))
+
+
+def encode_sr(fmt: int, t: float, u16: int) -> int:
+    """Stochastically rounded code of the binary32 value t for the 16-bit uniform u16 (Sec. 6.1)."""
+    return int(lib().orc_encode_sr(fmt, float(np.float32(t)), u16))
+
+
+def quantize(x_bits: np.ndarray, fmt: int, block: int, pow2_scale: bool = False, sr_seed: int | None = None) -> Quantized:
+    """sr_seed = None: round to nearest even (Sec. 2.3); an integer: stochastic rounding with that seed (Sec. 6.1)."""
     x = np.ascontiguousarray(x_bits, dtype=np.uint16)
     assert x.ndim == 2
     rows, cols = x.shape
@@ -164,8 +192,12 @@ def quantize(x_bits: np.ndarray, fmt: int, block: int, pow2_scale: bool = False)
     xhat = np.empty((rows, cols), dtype=np.float64)
     sumsq = np.zeros(2, dtype=np.float64)
     row_sumsq = np.zeros((rows, 2), dtype=np.float64)
-    rc = lib().orc_quantize_rule(_ptr(x), rows, cols, fmt, block, int(pow2_scale), _ptr(codes), _ptr(scales),
-                                 _ptr(xhat), _ptr(sumsq), _ptr(row_sumsq))
+    if sr_seed is None:
+        rc = lib().orc_quantize_rule(_ptr(x), rows, cols, fmt, block, int(pow2_scale), _ptr(codes), _ptr(scales),
+                                     _ptr(xhat), _ptr(sumsq), _ptr(row_sumsq))
+    else:
+        rc = lib().orc_quantize_sr(_ptr(x), rows, cols, fmt, block, int(pow2_scale), sr_seed, _ptr(codes), _ptr(scales),
+                                   _ptr(xhat), _ptr(sumsq), _ptr(row_sumsq))
     if rc != 0:
         raise ValueError("orc_quantize: bad argument")
     return Quantized(fmt, block, rows, cols, codes, scales, xhat, float(sumsq[0]),
