@@ -168,7 +168,7 @@ class Step:
                     M, K = x.shape
                     N = w.shape[0]
                     api._check("snip_linear_fwd_bwd", lib.snip_linear_fwd_bwd(p(x), p(w), p(dy), p(y), p(dx), p(dw), M, N, K, f, f, f, api.OUT_BF16,
-                                                                              int(mx), p(self.stats6[i]), p(self.ws), self.ws.numel(), st))
+                                                                              int(mx), 0, 0, p(self.stats6[i]), p(self.ws), self.ws.numel(), st))
                     i += 1
             return
         for f in self.formats:
@@ -222,7 +222,7 @@ class Step:
         def dual(x, fmt, kind, slot, stats_row):
             r, c = x.shape
             outs = [api.QOut(fmt, 0, p(self.codes[slot + j]), p(self.scales[slot + j]), p(self.sf[slot + j]) if mx else None,
-                             p(stats_row[24 * j:24 * j + 24])) for j in range(2)]
+                             p(stats_row[24 * j:24 * j + 24]), 0) for j in range(2)]
             api._check("snip_quantize_dual", lib.snip_quantize_dual(p(x), r, c, c, kind, int(mx), outs[0], outs[1], p(self.qws), self.qws.numel(), st))
 
         def gemm(op, fmt, ra, ca, blka, ta, rb, cb_, blkb, tb, out, flops, sa=0, sb_=1):
@@ -390,6 +390,25 @@ def run_profile_case(name):
         kind = api.DUAL_BLK_BLKT if parts[-1] == "blk" else api.DUAL_ROW_COLT
         by, times = kt.quantizer_dual(fmt, kind, 16384, 4096, iters=3, warmup=1)
         print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
+    elif parts[0] == "quantize" and parts[2] == "sr":
+        # stochastic rounding (FP4): quantize_fp4_sr_row | quantize_fp4_sr_col_t
+        block, flags = (api.BLOCK_ROW, api.Q_STATS) if parts[3] == "row" else (api.BLOCK_COL, api.Q_STATS | api.Q_TRANSPOSED)
+        xs = [torch.randn(16384, 4096, device=device, dtype=torch.bfloat16) for _ in range(3)]
+        cb, sb, wb = api.snip_quantize_sizes(16384, 4096, FMT_FP4, block, flags)
+        codes = torch.empty(cb, dtype=torch.uint8, device=device); scales = torch.empty(sb // 4, dtype=torch.float32, device=device)
+        stats = torch.empty(32, dtype=torch.uint8, device=device); ws = torch.empty(wb, dtype=torch.uint8, device=device)
+        times = []
+        for i in range(4):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for j in range(6):
+                x = xs[j % 3]
+                api._check("snip_quantize_sr", api._lib.snip_quantize_sr(api._p(x), 16384, 4096, 4096, block, flags, 17 + j, 0, api._p(codes), api._p(scales),
+                                                                         None, api._p(stats), api._p(ws), ws.numel(), api._stream()))
+            e1.record(); torch.cuda.synchronize()
+            if i: times.append(e0.elapsed_time(e1) / 6)
+        by = 2.531 * 16384 * 4096
+        print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)} ({min(times) * 1e3:.1f} us per call)")
     elif parts[0] == "quantize":
         kind = "_".join(parts[2:])
         block, tr = {"row": (api.BLOCK_ROW, False), "col_t": (api.BLOCK_COL, True), "blk_t": (api.BLOCK_BLK, True),

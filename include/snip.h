@@ -107,16 +107,20 @@ typedef struct {
     double sumsq_err[3][2][3];
 } snip_layer_stats_t;
 
+/* Rounding of the codes: nearest-even (Sec. 2.3) or stochastic (Sec. 6.1, FP4 output gradients). */
+typedef enum { SNIP_ROUND_NEAREST_EVEN = 0, SNIP_ROUND_STOCHASTIC = 1 } snip_rounding_t;
+
 /* One output of snip_quantize_dual: format (FP8 or FP4), destination buffers (device), optional UE8M0
  * scale-factor atoms (power-of-two rule only, else NULL) and optional statistics (device; give both
  * outputs' or neither). */
 typedef struct {
     int32_t fmt;
-    int32_t reserved;
+    int32_t rounding; /* snip_rounding_t; stochastic needs fmt = FP4 and row / column tiles */
     void *codes;
     float *scales;
     void *sf;
     snip_stats_t *stats;
+    uint64_t seed;    /* stochastic rounding: key of the generator */
 } snip_qout_t;
 
 /* Tile kinds of the two outputs of snip_quantize_dual. */
@@ -203,6 +207,25 @@ int snip_quantize_dual_workspace(int64_t rows, int64_t cols, size_t *ws_bytes_ho
 int snip_quantize_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, int kind, int pow2_scale,
                        const snip_qout_t *as_stored_host, const snip_qout_t *transposed_host,
                        void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Stochastic rounding for FP4 E2M1 codes (paper Sec. 6.1: FP4 output gradients are rounded
+ * probabilistically to one of the two nearest representable values so that small gradients do not
+ * vanish systematically).  Same tiles, scales, layouts and statistics as snip_quantize with
+ * fmt = FP4; only the rounding of the binary32 product t = x*S differs.  The paper cites the method
+ * without fixing a rule or a generator; this library's rule: with a = min(|t|, 6) and lo <= a < hi
+ * the neighbouring representable magnitudes, the code is hi iff (a - lo)/(hi - lo) > (u + 1/2)/2^16,
+ * else lo, sign copied from t; u is the element's 16-bit uniform: Philox4x32 with 10 rounds, counter
+ * = (idx/8 as two 32-bit words, 0, 0) with idx = r*cols + c (position in x, whatever the storage of
+ * the codes), key = the two words of `seed`; element idx uses bits [16*(idx%2), +16) of output word
+ * (idx%8)/2.  The result is a pure function of (x, seed): reruns are bit-identical.
+ * block: SNIP_BLOCK_ROW_1x128 (flags without SNIP_Q_TRANSPOSED) or SNIP_BLOCK_COL_128x1 (with it),
+ * the two forms an output gradient is consumed in; SNIP_Q_STATS as in snip_quantize (sumsq_err is the
+ * squared distance to the stochastic values).  pow2_scale / sf as in snip_quantize_mx.
+ */
+int snip_quantize_sr(const void *x, int64_t rows, int64_t cols, int64_t ld, int block, uint32_t flags,
+                     uint64_t seed, int pow2_scale, void *codes, float *scales, void *sf,
+                     snip_stats_t *stats, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * Power-of-two scale option (an added quantization option in the sense of paper Sec. 3.2, which lets
@@ -319,7 +342,9 @@ int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes
  * Results equal those of snip_linear_fwd / _dgrad / _wgrad (pow2_scale = 0) or snip_linear_mx
  * (pow2_scale != 0) called with the same tags.  stats6 (device, may be NULL): six snip_stats_t in the
  * order X/1x128, X/128x1, W/fwd format, W/dgrad format, dY/1x128, dY/128x1.  out_dtype applies to all
- * three outputs.  BF16 tags are not offered here (use the three separate calls).  A training loop that
+ * three outputs.  dy_rounding = SNIP_ROUND_STOCHASTIC rounds the FP4 copies of dY stochastically with
+ * dy_seed (Sec. 6.1; see snip_quantize_sr), FP8 copies stay nearest-even.  BF16 tags are not offered
+ * here (use the three separate calls).  A training loop that
  * separates forward and backward in time keeps the quantized copies instead of the bf16 activations;
  * this entry point runs the two halves back to back.
  */
@@ -327,8 +352,8 @@ int snip_linear_fwd_bwd_workspace(int64_t M, int64_t N, int64_t K, int fmt_fwd, 
                                   int pow2_scale, size_t *ws_bytes_host);
 int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY, void *Y, void *dX, void *dW,
                         int64_t M, int64_t N, int64_t K, int fmt_fwd, int fmt_dgrad, int fmt_wgrad,
-                        int out_dtype, int pow2_scale, snip_stats_t *stats6, void *ws, size_t ws_bytes,
-                        void *stream);
+                        int out_dtype, int pow2_scale, int dy_rounding, uint64_t dy_seed,
+                        snip_stats_t *stats6, void *ws, size_t ws_bytes, void *stream);
 
 /* ---- device status ------------------------------------------------------------------------ */
 

@@ -24,7 +24,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
+    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace",
     "snip_poll_status",
 )
@@ -45,11 +45,12 @@ class QTensor(ctypes.Structure):
 
 
 class QOut(ctypes.Structure):
-    _fields_ = [("fmt", ctypes.c_int32), ("reserved", ctypes.c_int32), ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p),
-                ("sf", ctypes.c_void_p), ("stats", ctypes.c_void_p)]
+    _fields_ = [("fmt", ctypes.c_int32), ("rounding", ctypes.c_int32), ("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("sf", ctypes.c_void_p), ("stats", ctypes.c_void_p), ("seed", ctypes.c_uint64)]
 
 
 DUAL_ROW_COLT, DUAL_BLK_BLKT = 0, 1
+ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 
 
 class LayerTensors(ctypes.Structure):
@@ -74,6 +75,7 @@ def _load():
     lib.snip_quantize_mx.argtypes = [vp, i64, i64, i64, i32, i32, u32, vp, vp, vp, vp, vp, sz, vp]
     lib.snip_quantize_dual_workspace.argtypes = [i64, i64, psz]
     lib.snip_quantize_dual.argtypes = [vp, i64, i64, i64, i32, i32, ctypes.POINTER(QOut), ctypes.POINTER(QOut), vp, sz, vp]
+    lib.snip_quantize_sr.argtypes = [vp, i64, i64, i64, i32, u32, ctypes.c_uint64, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
     lib.snip_gemm_mx.argtypes = [i32, ctypes.POINTER(QTensor), vp, ctypes.POINTER(QTensor), vp, vp, i32, vp, sz, vp]
@@ -84,7 +86,7 @@ def _load():
     lib.snip_linear_mx.argtypes = [i32, vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_mx_workspace.argtypes = [i32, i64, i64, i64, i32, i32, psz]
     lib.snip_linear_fwd_bwd_workspace.argtypes = [i64, i64, i64, i32, i32, i32, i32, psz]
-    lib.snip_linear_fwd_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, vp, vp, sz, vp]
+    lib.snip_linear_fwd_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, i32, ctypes.c_uint64, vp, vp, sz, vp]
     lib.snip_layer_stats.argtypes = [ctypes.POINTER(LayerTensors), u32, vp, vp, sz, vp]
     lib.snip_layer_stats_workspace.argtypes = [i64, i64, i64, psz]
     lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -195,8 +197,28 @@ def snip_quantize_dual_workspace(rows, cols):
     return n.value
 
 
+def snip_quantize_sr(x: torch.Tensor, block: int, flags: int, seed: int, *, pow2_scale=False, want_sf=False):
+    """FP4 codes with stochastic rounding.  Returns (codes, scales, sf, stats) like snip_quantize_mx."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    cb, sb, wb = snip_quantize_sizes(rows, cols, FMT_FP4_E2M1, block, flags)
+    dev = x.device
+    codes = torch.empty(cb, dtype=torch.uint8, device=dev)
+    scales = torch.empty(sb // 4, dtype=torch.float32, device=dev)
+    sf = None
+    if want_sf:
+        n = ctypes.c_size_t()
+        _check("snip_quantize_mx_sizes", _lib.snip_quantize_mx_sizes(rows, cols, ctypes.byref(n)))
+        sf = torch.empty(n.value, dtype=torch.uint8, device=dev)
+    stats = torch.empty(32, dtype=torch.uint8, device=dev) if (flags & Q_STATS) else None
+    ws = torch.empty(wb, dtype=torch.uint8, device=dev) if (flags & Q_STATS) else None
+    _check("snip_quantize_sr", _lib.snip_quantize_sr(_p(x), rows, cols, x.stride(0), block, flags, seed, int(pow2_scale), _p(codes), _p(scales),
+                                                     _p(sf), _p(stats), _p(ws), 0 if ws is None else ws.numel(), _stream()))
+    return codes, scales, sf, stats
+
+
 def snip_quantize_dual(x: torch.Tensor, kind: int, fmt_stored: int, fmt_transposed: int, *, pow2_scale=False, want_stats=True,
-                       want_sf=False, bufs=None, ws=None):
+                       want_sf=False, bufs=None, ws=None, sr_seeds=(None, None)):
     """One read, two outputs.  Returns two dicts (as stored, transposed) with codes / scales / sf / stats
     tensors (sf, stats None unless asked for).  bufs = (dict, dict) reuses buffers of an earlier call."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
@@ -216,7 +238,9 @@ def snip_quantize_dual(x: torch.Tensor, kind: int, fmt_stored: int, fmt_transpos
                 _check("snip_quantize_mx_sizes", _lib.snip_quantize_mx_sizes(rows, cols, ctypes.byref(n)))
                 o["sf"] = torch.empty(n.value, dtype=torch.uint8, device=dev)
         outs.append(o)
-        structs.append(QOut(fmt, 0, _p(o["codes"]), _p(o["scales"]), _p(o["sf"]), _p(o["stats"])))
+        seed = sr_seeds[i]
+        structs.append(QOut(fmt, ROUND_NEAREST_EVEN if seed is None else ROUND_STOCHASTIC, _p(o["codes"]), _p(o["scales"]), _p(o["sf"]),
+                            _p(o["stats"]), 0 if seed is None else seed))
     if ws is None and outs[0]["stats"] is not None:
         ws = torch.empty(snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=dev)
     _check("snip_quantize_dual", _lib.snip_quantize_dual(_p(x), rows, cols, x.stride(0), kind, int(pow2_scale), ctypes.byref(structs[0]),
@@ -337,8 +361,8 @@ def snip_linear_fwd_bwd_workspace(M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad, pow2_s
     return n.value
 
 
-def snip_linear_fwd_bwd(x, w, dy, fmt_fwd, fmt_dgrad, fmt_wgrad, out_dtype=OUT_BF16, *, pow2_scale=False, y=None, dx=None, dw=None,
-                        stats=None, ws=None):
+def snip_linear_fwd_bwd(x, w, dy, fmt_fwd, fmt_dgrad, fmt_wgrad, out_dtype=OUT_BF16, *, pow2_scale=False, dy_sr_seed=None, y=None,
+                        dx=None, dw=None, stats=None, ws=None):
     """Forward and both gradients of one linear layer, each tensor read once.  Returns (y, dx, dw, stats)
     with stats a uint8 tensor holding six 24-byte snip_stats_t."""
     M, K = x.shape
@@ -350,7 +374,8 @@ def snip_linear_fwd_bwd(x, w, dy, fmt_fwd, fmt_dgrad, fmt_wgrad, out_dtype=OUT_B
     if ws is None:
         ws = torch.zeros(snip_linear_fwd_bwd_workspace(M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad, pow2_scale), dtype=torch.uint8, device=dev)
     _check("snip_linear_fwd_bwd", _lib.snip_linear_fwd_bwd(_p(x), _p(w), _p(dy), _p(y), _p(dx), _p(dw), M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad,
-                                                           out_dtype, int(pow2_scale), _p(stats), _p(ws), ws.numel(), _stream()))
+                                                           out_dtype, int(pow2_scale), ROUND_NEAREST_EVEN if dy_sr_seed is None else ROUND_STOCHASTIC,
+                                                           0 if dy_sr_seed is None else dy_sr_seed, _p(stats), _p(ws), ws.numel(), _stream()))
     return y, dx, dw, stats
 
 

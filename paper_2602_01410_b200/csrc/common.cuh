@@ -35,6 +35,8 @@ struct DualOut {
     float *scales;
     void *sf;             // optional UE8M0 atoms (power-of-two rule only)
     snip_stats_t *stats;  // optional; both outputs or neither
+    int sr = 0;           // 1: stochastic rounding (FP4 only)
+    uint64_t seed = 0;
 };
 
 // Fails with SNIP_ERR_UNSUPPORTED unless the current device is compute capability 10.x.

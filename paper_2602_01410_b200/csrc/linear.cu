@@ -250,8 +250,8 @@ extern "C" int snip_linear_fwd_bwd_workspace(int64_t M, int64_t N, int64_t K, in
 }
 
 extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY, void *Y, void *dX, void *dW, int64_t M, int64_t N, int64_t K,
-                                   int fmt_fwd, int fmt_dgrad, int fmt_wgrad, int out_dtype, int pow2_scale, snip_stats_t *stats6, void *ws,
-                                   size_t ws_bytes, void *stream)
+                                   int fmt_fwd, int fmt_dgrad, int fmt_wgrad, int out_dtype, int pow2_scale, int dy_rounding, uint64_t dy_seed,
+                                   snip_stats_t *stats6, void *ws, size_t ws_bytes, void *stream)
 {
     using namespace snip;
     if (!X || !W || !dY || !Y || !dX || !dW) return SNIP_ERR_ARG;
@@ -264,7 +264,12 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
     const bool mx = pow2_scale != 0;
     const int fmt[6] = {fmt_fwd, fmt_wgrad, fmt_fwd, fmt_dgrad, fmt_dgrad, fmt_wgrad};
     const FwdBwdCarve f = carve_fwd_bwd(ws, M, N, K, fmt, mx);
-    auto out_of = [&](int i) { return DualOut{fmt[i], f.codes[i], f.scales[i], f.sf[i], stats6 ? stats6 + i : nullptr}; };
+    if (dy_rounding != SNIP_ROUND_NEAREST_EVEN && dy_rounding != SNIP_ROUND_STOCHASTIC) return SNIP_ERR_ARG;
+    // stochastic rounding applies to the FP4 copies of dY (indices 4 and 5); an FP8 copy keeps nearest-even
+    auto out_of = [&](int i) {
+        const int sr = (i >= 4 && dy_rounding == SNIP_ROUND_STOCHASTIC && fmt[i] == SNIP_FMT_FP4_E2M1) ? 1 : 0;
+        return DualOut{fmt[i], f.codes[i], f.scales[i], f.sf[i], stats6 ? stats6 + i : nullptr, sr, dy_seed};
+    };
     auto gemm = [&](int op, int ia, int ib, void *out) -> int {
         const LinearPlan p = plan_for(op, M, N, K);
         if (mx) return gemm_mx_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], f.sf[ia], f.sf[ib], p.Mo, p.No, p.Kc, out, out_dtype, f.gws, gemm_ws_bytes(), st);

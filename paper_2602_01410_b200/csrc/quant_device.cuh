@@ -132,4 +132,36 @@ __device__ __forceinline__ void quant8(const uint4 &v, const float2 (&s2)[4], co
     }
 }
 
+// ---- stochastic rounding (paper Sec. 6.1: FP4 output gradients) ------------------------------------
+
+// Philox4x32 with 10 rounds (Salmon et al., SC'11): counter (c0, c1, 0, 0), key (k0, k1).
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1, uint32_t (&out)[4])
+{
+    uint32_t c2 = 0, c3 = 0;
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Stochastically rounded E2M1 value of t for the 16-bit uniform u: with a = min(|t|, 6), g the grid step
+// at a (0.5 below 2, 1 below 4, else 2) and lo = floor(a/g)*g, the result is lo + g iff
+// (a - lo)/g > (u + 1/2)/2^16, else lo; the sign of t is kept.  Every operation below is exact in
+// binary32, so the decision equals the one taken in exact arithmetic.
+__device__ __forceinline__ float sr_e2m1_value(float t, uint32_t u)
+{
+    const float a = fminf(fabsf(t), 6.0f);
+    const float g = a < 2.0f ? 0.5f : (a < 4.0f ? 1.0f : 2.0f);
+    const float inv_g = a < 2.0f ? 2.0f : (a < 4.0f ? 1.0f : 0.5f);
+    const float y = a * inv_g;
+    const float k = floorf(y);
+    const float thr = (float)(2u * u + 1u) * (1.0f / 131072.0f);
+    const float v = (k + ((y - k) > thr ? 1.0f : 0.0f)) * g;
+    return copysignf(v, t);
+}
+
 }  // namespace snip

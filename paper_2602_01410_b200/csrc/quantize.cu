@@ -40,6 +40,7 @@ struct QuantArgs {
     CtaPartial *partials; // may be null (no stats)
     float2 *row_partials; // [col tiles][rows] {sum x^2, sum err^2}; may be null
     int64_t tiles_r, tiles_c, ntiles;
+    uint64_t seed;        // stochastic rounding: key of the generator
     int pow2;             // 1: power-of-two scale rule (largest 2^e with amax * 2^e <= FPX_MAX)
     uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
 };
@@ -84,14 +85,15 @@ __device__ __forceinline__ void prefetch_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void prefetch_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 // Compile-time description of one output of a tile pass.
-template <int FMT_, int BLOCK_, bool TRANSPOSED_, bool CODES_>
+template <int FMT_, int BLOCK_, bool TRANSPOSED_, bool CODES_, bool SR_ = false>
 struct Out {
     static constexpr int FMT = FMT_, BLOCK = BLOCK_;
-    static constexpr bool TRANSPOSED = TRANSPOSED_, CODES = CODES_, kQuant = (FMT_ != SNIP_FMT_BF16);
+    static constexpr bool TRANSPOSED = TRANSPOSED_, CODES = CODES_, kQuant = (FMT_ != SNIP_FMT_BF16), SR = SR_;
+    static_assert(!SR_ || FMT_ == SNIP_FMT_FP4_E2M1, "stochastic rounding is offered for FP4 E2M1 only");
 };
 struct NoOut {
     static constexpr int FMT = SNIP_FMT_BF16, BLOCK = SNIP_BLOCK_BLK_128x128;
-    static constexpr bool TRANSPOSED = false, CODES = false, kQuant = false;
+    static constexpr bool TRANSPOSED = false, CODES = false, kQuant = false, SR = false;
 };
 
 // Per-thread running sums over the tiles of a CTA (binary64: one add per tile and sum).
@@ -125,6 +127,20 @@ __device__ __forceinline__ uint32_t encode_pair(const float2 x, const float2 s, 
         se2 = __ffma2_rn(e, e, se2);
     }
     return c;
+}
+
+// Stochastic-rounding form for FP4: u2 holds the two 16-bit uniforms of the pair (first element low).
+// The rounded values are at hand in binary32, so the error term needs no decode.
+template <bool STATS>
+__device__ __forceinline__ uint32_t encode_pair_sr_fp4(const float2 x, const float2 s, const float2 n, uint32_t u2, float2 &se2)
+{
+    const float2 t = __fmul2_rn(x, s);
+    const float2 v = make_float2(sr_e2m1_value(t.x, u2 & 0xFFFFu), sr_e2m1_value(t.y, u2 >> 16));
+    if (STATS) {
+        const float2 e = __ffma2_rn(v, n, x);
+        se2 = __ffma2_rn(e, e, se2);
+    }
+    return cvt_e2m1x2(v.x, v.y);   // exact: v is representable
 }
 
 // Packs the four pair codes of 8 consecutive elements: FP8 -> two words, FP4 -> one word.
@@ -421,13 +437,27 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
         const uint4 vp = slot[p * kThreads];
         const uint32_t w[4] = {vp.x, vp.y, vp.z, vp.w};
         uint32_t ca[4], cb[4];
+        uint32_t ua[4], ub[4];   // stochastic rounding: the eight 16-bit uniforms of this row segment
+        (void)ua; (void)ub;
+        if (A::SR || B::SR) {
+            // element index r * cols + c, eight consecutive columns per generator call
+            const uint64_t blk = ((uint64_t)(rbase + p) * (uint64_t)qa.cols + (uint64_t)cbase) >> 3;
+            if (A::SR) philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)qa.seed, (uint32_t)(qa.seed >> 32), ua);
+            if (B::SR) philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)qb.seed, (uint32_t)(qb.seed >> 32), ub);
+        }
         float2 px = make_float2(0.0f, 0.0f), pe = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const float2 x = make_float2(bf16lo(w[i]), bf16hi(w[i]));
             if (STATS) { if (ROWSTATS) px = __ffma2_rn(x, x, px); else sx2 = __ffma2_rn(x, x, sx2); }
-            if (A::kQuant) ca[i] = encode_pair<A::FMT, STATS>(x, scale_pair<A>(sa, p, i), ninv_pair<A>(sa, p, i), ROWSTATS ? pe : sea2);
-            if (B::kQuant) cb[i] = encode_pair<B::FMT, STATS>(x, scale_pair<B>(sb, p, i), ninv_pair<B>(sb, p, i), seb2);
+            if (A::kQuant) {
+                if (A::SR) ca[i] = encode_pair_sr_fp4<STATS>(x, scale_pair<A>(sa, p, i), ninv_pair<A>(sa, p, i), ua[i], ROWSTATS ? pe : sea2);
+                else ca[i] = encode_pair<A::FMT, STATS>(x, scale_pair<A>(sa, p, i), ninv_pair<A>(sa, p, i), ROWSTATS ? pe : sea2);
+            }
+            if (B::kQuant) {
+                if (B::SR) cb[i] = encode_pair_sr_fp4<STATS>(x, scale_pair<B>(sb, p, i), ninv_pair<B>(sb, p, i), ub[i], seb2);
+                else cb[i] = encode_pair<B::FMT, STATS>(x, scale_pair<B>(sb, p, i), ninv_pair<B>(sb, p, i), seb2);
+            }
         }
         if (ROWSTATS) {
             rsx[p] = px.x + px.y; rse[p] = pe.x + pe.y;
@@ -537,7 +567,7 @@ struct TileWalk {
     }
 };
 
-template <int FMT, int BLOCK, bool TRANSPOSED, bool CODES, bool STATS, bool ROWSTATS>
+template <int FMT, int BLOCK, bool TRANSPOSED, bool CODES, bool STATS, bool ROWSTATS, bool SR = false>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const QuantArgs a)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -554,7 +584,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
         w.next();
-        process_tile<Out<FMT, BLOCK, TRANSPOSED, CODES>, NoOut, STATS, ROWSTATS>(a, a, tl, slot, sh, ts, [&] {
+        process_tile<Out<FMT, BLOCK, TRANSPOSED, CODES, SR>, NoOut, STATS, ROWSTATS>(a, a, tl, slot, sh, ts, [&] {
             if (w.valid()) prefetch_tile(a, w.r, w.c, smem);   // this thread's reads of its slot are done
             prefetch_commit();
         });
@@ -569,7 +599,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
 struct DualArgs {
     QuantArgs a, b;
 };
-template <int FMT_A, int FMT_B, bool BLK, bool STATS>
+template <int FMT_A, int FMT_B, bool BLK, bool STATS, bool SR_A = false, bool SR_B = false>
 __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel(const DualArgs d)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -584,8 +614,8 @@ __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
         w.next();
-        using A = Out<FMT_A, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true>;
-        using B = Out<FMT_B, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true>;
+        using A = Out<FMT_A, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true, SR_A>;
+        using B = Out<FMT_B, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true, SR_B>;
         process_tile<A, B, STATS, false>(d.a, d.b, tl, slot, sh, ts, [&] {
             if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
             prefetch_commit();
@@ -716,9 +746,21 @@ int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
     return quantize_impl_ex(x, rows, cols, ld, fmt, block, flags, 0, nullptr, codes, scales, stats, row_stats, ws, ws_bytes, st);
 }
 
+int quantize_impl_full(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf, int sr,
+                       uint64_t seed, void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes,
+                       cudaStream_t st);
+
 // pow2 = 1 selects the power-of-two scale rule; sf (optional, needs pow2) receives the UE8M0 atoms.
 int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf,
                      void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    return quantize_impl_full(x, rows, cols, ld, fmt, block, flags, pow2, sf, 0, 0, codes, scales, stats, row_stats, ws, ws_bytes, st);
+}
+
+// sr = 1: stochastic rounding with `seed` (FP4 codes, 1x128 tiles as stored or 128x1 tiles transposed, no per-row sums).
+int quantize_impl_full(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf, int sr,
+                       uint64_t seed, void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes,
+                       cudaStream_t st)
 {
     if (sf) {
         const bool tr = (flags & SNIP_Q_TRANSPOSED) != 0;
@@ -749,6 +791,7 @@ int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
     a.x = static_cast<const uint16_t *>(x);
     a.rows = rows; a.cols = cols; a.ld = ld;
     a.pow2 = pow2; a.sf = static_cast<uint32_t *>(sf);
+    a.seed = seed;
     a.codes = want_codes ? static_cast<uint8_t *>(codes) : nullptr;
     a.scales = want_codes ? scales : nullptr;
     a.partials = any_stats ? static_cast<CtaPartial *>(ws) : nullptr;
@@ -756,6 +799,15 @@ int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
     a.tiles_r = tr; a.tiles_c = tc; a.ntiles = tr * tc;
     const int64_t nparts = persistent_ctas(tr * tc);
     dim3 grid((unsigned)nparts);
+    if (sr) {
+        const bool row = block == SNIP_BLOCK_ROW_1x128 && !transposed, colt = block == SNIP_BLOCK_COL_128x1 && transposed;
+        if (fmt != SNIP_FMT_FP4_E2M1 || !want_codes || want_rows || !(row || colt)) return SNIP_ERR_UNSUPPORTED;
+        constexpr int F4 = SNIP_FMT_FP4_E2M1;
+        if (row && any_stats) launch_persistent(quantize_kernel<F4, SNIP_BLOCK_ROW_1x128, false, true, true, false, true>, a, grid, st);
+        else if (row) launch_persistent(quantize_kernel<F4, SNIP_BLOCK_ROW_1x128, false, true, false, false, true>, a, grid, st);
+        else if (any_stats) launch_persistent(quantize_kernel<F4, SNIP_BLOCK_COL_128x1, true, true, true, false, true>, a, grid, st);
+        else launch_persistent(quantize_kernel<F4, SNIP_BLOCK_COL_128x1, true, true, false, false, true>, a, grid, st);
+    } else
     if (fmt == SNIP_FMT_FP8_E4M3) launch_fmt<SNIP_FMT_FP8_E4M3>(a, block, transposed, want_codes, any_stats, want_rows, grid, st);
     else if (fmt == SNIP_FMT_FP4_E2M1) launch_fmt<SNIP_FMT_FP4_E2M1>(a, block, transposed, want_codes, any_stats, want_rows, grid, st);
     else launch_variant<SNIP_FMT_BF16, SNIP_BLOCK_BLK_128x128, false>(a, false, true, want_rows, grid, st);
@@ -782,6 +834,14 @@ int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
 
 // One read, two outputs.  blk = false: a = 1x128 tiles as stored, b = 128x1 tiles transposed;
 // blk = true: a = 128x128 blocks as stored, b = the same blocks transposed.
+// Two-output launch with stochastic rounding on the FP4 outputs that ask for it (row/column kinds only).
+template <int FMT_A, int FMT_B, bool SR_A, bool SR_B>
+static void launch_dual_sr(const DualArgs &d, bool stats, dim3 grid, cudaStream_t st)
+{
+    if (stats) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, true, SR_A, SR_B>, d, grid, st);
+    else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false, SR_A, SR_B>, d, grid, st);
+}
+
 template <int FMT_A, int FMT_B>
 static void launch_dual(const DualArgs &d, bool blk, bool stats, dim3 grid, cudaStream_t st)
 {
@@ -824,12 +884,22 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bo
         q.partials = stats ? reinterpret_cast<CtaPartial *>(static_cast<uint8_t *>(ws) + i * one) : nullptr;
         q.row_partials = nullptr;
         q.pow2 = pow2;
+        q.seed = o[i]->seed;
         q.sf = static_cast<uint32_t *>(o[i]->sf);
         q.tiles_r = tr; q.tiles_c = tc; q.ntiles = tr * tc;
     }
     const int64_t nparts = persistent_ctas(tr * tc, kDualCtasPerSm);
     dim3 grid((unsigned)nparts);
     const bool a8 = oa.fmt == SNIP_FMT_FP8_E4M3, b8 = ob.fmt == SNIP_FMT_FP8_E4M3;
+    constexpr int F8 = SNIP_FMT_FP8_E4M3, F4 = SNIP_FMT_FP4_E2M1;
+    if (oa.sr || ob.sr) {
+        if (blk || (oa.sr && a8) || (ob.sr && b8)) return SNIP_ERR_UNSUPPORTED;   // FP4 row / column tiles only
+        if (oa.sr && ob.sr) launch_dual_sr<F4, F4, true, true>(d, stats, grid, st);
+        else if (oa.sr && b8) launch_dual_sr<F4, F8, true, false>(d, stats, grid, st);
+        else if (oa.sr) launch_dual_sr<F4, F4, true, false>(d, stats, grid, st);
+        else if (a8) launch_dual_sr<F8, F4, false, true>(d, stats, grid, st);
+        else launch_dual_sr<F4, F4, false, true>(d, stats, grid, st);
+    } else
     if (a8 && b8) launch_dual<SNIP_FMT_FP8_E4M3, SNIP_FMT_FP8_E4M3>(d, blk, stats, grid, st);
     else if (a8) launch_dual<SNIP_FMT_FP8_E4M3, SNIP_FMT_FP4_E2M1>(d, blk, stats, grid, st);
     else if (b8) launch_dual<SNIP_FMT_FP4_E2M1, SNIP_FMT_FP8_E4M3>(d, blk, stats, grid, st);
@@ -980,8 +1050,19 @@ extern "C" int snip_quantize_dual(const void *x, int64_t rows, int64_t cols, int
     using namespace snip;
     if (!as_stored || !transposed) return SNIP_ERR_ARG;
     if (kind != SNIP_DUAL_ROW_COLT && kind != SNIP_DUAL_BLK_BLKT) return SNIP_ERR_ARG;
-    const DualOut oa = {as_stored->fmt, as_stored->codes, as_stored->scales, as_stored->sf, as_stored->stats};
-    const DualOut ob = {transposed->fmt, transposed->codes, transposed->scales, transposed->sf, transposed->stats};
+    if ((as_stored->rounding & ~1) || (transposed->rounding & ~1)) return SNIP_ERR_ARG;
+    const DualOut oa = {as_stored->fmt, as_stored->codes, as_stored->scales, as_stored->sf, as_stored->stats, as_stored->rounding, as_stored->seed};
+    const DualOut ob = {transposed->fmt, transposed->codes, transposed->scales, transposed->sf, transposed->stats, transposed->rounding, transposed->seed};
     return quantize_dual_impl(x, rows, cols, ld, kind == SNIP_DUAL_BLK_BLKT, pow2_scale ? 1 : 0, oa, ob, ws, ws_bytes,
                               static_cast<cudaStream_t>(stream));
+}
+
+// ---- stochastic rounding (paper Sec. 6.1) ------------------------------------------------------
+
+extern "C" int snip_quantize_sr(const void *x, int64_t rows, int64_t cols, int64_t ld, int block, uint32_t flags, uint64_t seed, int pow2_scale,
+                                void *codes, float *scales, void *sf, snip_stats_t *stats, void *ws, size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    return quantize_impl_full(x, rows, cols, ld, SNIP_FMT_FP4_E2M1, block, flags, pow2_scale ? 1 : 0, sf, 1, seed, codes, scales, stats, nullptr, ws,
+                              ws_bytes, static_cast<cudaStream_t>(stream));
 }
