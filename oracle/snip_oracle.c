@@ -518,6 +518,27 @@ double orc_sumsq_bf16(const uint16_t *x, int64_t n)
     return s;
 }
 
+/* ---- AdamW sensitivity term (Sec. 4.3: weight divergence) --------------------------------------
+ *
+ * Step 1 also collects the Frobenius norm of the elementwise term
+ *     T = (1 - beta1) / (sqrt(v) + eps)  -  (1 - beta2) m g / ( sqrt(v) (sqrt(v) + eps)^2 ),
+ * the derivative of the AdamW direction m / (sqrt(v) + eps) with respect to the gradient g (m, v are
+ * the moments after they absorbed g).  Returns sum T^2 in binary64.  m, v, g: binary64 copies of the
+ * inputs.  Reading: where v == 0 (then g == 0 and m == 0 in AdamW) the second term is taken as 0. */
+double orc_adamw_sensitivity_sumsq(const double *m, const double *v, const double *g, int64_t n, double beta1, double beta2, double eps)
+{
+    double acc = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double s = sqrt(v[i]);
+        double d = s + eps;
+        double first = (1.0 - beta1) / d;
+        double second = v[i] == 0.0 ? 0.0 : (1.0 - beta2) * m[i] * g[i] / (s * d * d);
+        double t = first - second;
+        acc += t * t;
+    }
+    return acc;
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.orc_round_to_bf16.argtypes = [vp, i64, vp]
         L.orc_sumsq_bf16.restype = dbl
         L.orc_sumsq_bf16.argtypes = [vp, i64]
+        L.orc_adamw_sensitivity_sumsq.restype = dbl
+        L.orc_adamw_sensitivity_sumsq.argtypes = [vp, vp, vp, i64, dbl, dbl, dbl]
         L.orc_num_threads.restype = i32
         L.orc_num_threads.argtypes = []
         _lib = L
@@ -329,3 +331,11 @@ def sf_atoms(q: Quantized, transposed: bool) -> np.ndarray:
                 atom[(r % 32) * 4 + r // 32, :] = b
     return out.reshape(-1)
 
+
+
+def adamw_sensitivity_sumsq(m, v, g, beta1: float, beta2: float, eps: float) -> float:
+    """Sum over all elements of T^2, T = (1-beta1)/(sqrt(v)+eps) - (1-beta2) m g / (sqrt(v) (sqrt(v)+eps)^2)
+    (Sec. 4.3); its square root is the norm Step 1 collects for the weight-divergence estimate."""
+    m64, v64, g64 = (np.ascontiguousarray(np.asarray(a, dtype=np.float64).reshape(-1)) for a in (m, v, g))
+    assert m64.size == v64.size == g64.size
+    return float(lib().orc_adamw_sensitivity_sumsq(_ptr(m64), _ptr(v64), _ptr(g64), m64.size, beta1, beta2, eps))
