@@ -381,6 +381,23 @@ def run_profile_case(name):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     parts = name.split("_")
+    if name.startswith("adamw"):
+        n = 12288 * 4096
+        ms_ = [torch.randn(n, device=device) * 1e-3 for _ in range(2)]
+        vs_ = [torch.rand(n, device=device) * 1e-6 + 1e-12 for _ in range(2)]
+        gs_ = [(torch.randn(n, device=device) * 1e-3).to(torch.bfloat16) for _ in range(2)]
+        out = torch.zeros(1, dtype=torch.float64, device=device)
+        ws = torch.empty(1 << 16, dtype=torch.uint8, device=device)
+        times = []
+        for i in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            api.snip_adamw_sensitivity(ms_[i % 2], vs_[i % 2], gs_[i % 2], 0.9, 0.95, 1e-8, out=out, ws=ws)
+            e1.record(); torch.cuda.synchronize()
+            if i >= 2: times.append(e0.elapsed_time(e1))
+        by = 10.0 * n
+        print(f"adamw_sensitivity 12288x4096 (m, v fp32, g bf16): {min(times) * 1e3:.1f} us, {by / (min(times) * 1e-3) / 1e9:.0f} GB/s")
+        return
     if name.startswith("layer_stats"):
         return run_layer_stats_case(api, torch, device, parts[2] if len(parts) > 2 else "x")
     mx = parts[1].startswith("mx")

@@ -355,6 +355,25 @@ int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY, void *Y, v
                         int out_dtype, int pow2_scale, int dy_rounding, uint64_t dy_seed,
                         snip_stats_t *stats6, void *ws, size_t ws_bytes, void *stream);
 
+/* ---- optimizer statistics (paper Sec. 4.3) ------------------------------------------------- */
+
+/*
+ * Sum over a parameter tensor of T^2 with
+ *     T = (1 - beta1) / (sqrt(v) + eps)  -  (1 - beta2) m g / ( sqrt(v) (sqrt(v) + eps)^2 ),
+ * elementwise over the AdamW moments m, v (binary32, after they absorbed g) and the gradient g
+ * (bf16 or binary32, g_dtype = SNIP_OUT_BF16 / SNIP_OUT_FP32).  T is the derivative of the AdamW
+ * direction m / (sqrt(v) + eps) with respect to g; Step 1 collects ||T||_F per layer, and the weight
+ * divergence of a quantization option is estimated as that norm times the option's gradient error
+ * norm (Sec. 4.3).  Where v == 0 the second term is taken as 0 (a reading: AdamW then has m = g = 0).
+ * n: number of elements, a multiple of 4; m, v 16-byte aligned, g 8-byte (bf16) or 16-byte aligned.
+ * *sumsq (device, binary64) receives the sum.  Arithmetic in binary32 (reciprocal square root and
+ * reciprocal to about 2 ulp), sums in binary64; agrees with the binary64 definition to about 1e-6.  One read of each input: 10 or 12 bytes per element.
+ */
+int snip_adamw_sensitivity_workspace(int64_t n, size_t *ws_bytes_host);
+int snip_adamw_sensitivity(const float *m, const float *v, const void *g, int g_dtype, int64_t n,
+                           float beta1, float beta2, float eps, double *sumsq, void *ws, size_t ws_bytes,
+                           void *stream);
+
 /* ---- device status ------------------------------------------------------------------------ */
 
 /*

@@ -25,7 +25,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
     "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
-    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace",
+    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace", "snip_adamw_sensitivity_workspace", "snip_adamw_sensitivity",
     "snip_poll_status",
 )
 
@@ -89,6 +89,8 @@ def _load():
     lib.snip_linear_fwd_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, i32, i32, ctypes.c_uint64, vp, vp, sz, vp]
     lib.snip_layer_stats.argtypes = [ctypes.POINTER(LayerTensors), u32, vp, vp, sz, vp]
     lib.snip_layer_stats_workspace.argtypes = [i64, i64, i64, psz]
+    lib.snip_adamw_sensitivity_workspace.argtypes = [i64, psz]
+    lib.snip_adamw_sensitivity.argtypes = [vp, vp, vp, i32, i64, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp, sz, vp]
     lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -394,6 +396,22 @@ def snip_layer_stats(X=None, W=None, Y=None, dY=None, dX=None, dW=None, *, M, N,
     if ws is None:
         ws = torch.empty(snip_layer_stats_workspace(M, N, K), dtype=torch.uint8, device=dev)
     _check("snip_layer_stats", _lib.snip_layer_stats(ctypes.byref(lt), fmt_mask, _p(out), _p(ws), ws.numel(), _stream()))
+    return out
+
+
+def snip_adamw_sensitivity(m: torch.Tensor, v: torch.Tensor, g: torch.Tensor, beta1: float, beta2: float, eps: float, *, out=None, ws=None):
+    """Sum of T^2 (AdamW sensitivity term) over a parameter tensor; returns a 1-element float64 CUDA tensor."""
+    assert m.dtype == torch.float32 and v.dtype == torch.float32 and g.dtype in (torch.bfloat16, torch.float32)
+    assert m.is_contiguous() and v.is_contiguous() and g.is_contiguous() and m.numel() == v.numel() == g.numel()
+    n = m.numel()
+    if out is None:
+        out = torch.zeros(1, dtype=torch.float64, device=m.device)
+    if ws is None:
+        w = ctypes.c_size_t()
+        _check("snip_adamw_sensitivity_workspace", _lib.snip_adamw_sensitivity_workspace(n, ctypes.byref(w)))
+        ws = torch.empty(w.value, dtype=torch.uint8, device=m.device)
+    _check("snip_adamw_sensitivity", _lib.snip_adamw_sensitivity(_p(m), _p(v), _p(g), OUT_BF16 if g.dtype == torch.bfloat16 else OUT_FP32, n, beta1, beta2,
+                                                                 eps, _p(out), _p(ws), ws.numel(), _stream()))
     return out
 
 
