@@ -317,29 +317,39 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
             }
+            // Reciprocal scale factors of chunk cn from its ring slot (the slot must have landed).  Block mode:
+            // one factor per 32-column group; vector mode: 1/S_a in fo[0], and the slot's column scales are
+            // turned into reciprocals in place (4 per lane).
+            auto prepare_factors = [&](int cn, float (&fo)[G]) {
+                float *sl = ring + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot;
+                const float sa = sl[lane];
+                if (SCALE == SCALE_BLOCK_B) {
+                    const float f0 = __fdividef(1.0f, sa * sl[32]), f1 = __fdividef(1.0f, sa * sl[33]);
+#pragma unroll
+                    for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
+                } else {
+                    fo[0] = __fdividef(1.0f, sa);
+                    if (4 * lane < HALF) {
+                        float4 *p4 = reinterpret_cast<float4 *>(sl + C::kRingB + 4 * lane);
+                        const float4 s4 = *p4;
+                        *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
+                    }
+                    __syncwarp();
+                }
+            };
+            float f_next[G];
+            if (SCALE != SCALE_NONE) {
+                cp_async_wait<C::kScaleDepth - 1>();   // chunk 0's scales
+                __syncwarp();
+                prepare_factors(0, f_next);
+                __syncwarp();
+            }
             for (int c = 0; c < nacc; ++c, ++cc) {
                 const uint32_t a = cc & 1u;
                 float f[G];
                 const float *slot = ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;
-                if (SCALE != SCALE_NONE) {
-                    cp_async_wait<C::kScaleDepth - 1>();
-                    __syncwarp();
-                    const float sa = slot[lane];
-                    if (SCALE == SCALE_BLOCK_B) {
-                        const float f0 = __fdividef(1.0f, sa * slot[32]), f1 = __fdividef(1.0f, sa * slot[33]);
 #pragma unroll
-                        for (int gi = 0; gi < G; ++gi) f[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
-                    } else {
-                        f[0] = __fdividef(1.0f, sa);
-                        // turn this chunk's column scales into reciprocals once (4 per lane), in place
-                        if (4 * lane < HALF) {
-                            float4 *p4 = reinterpret_cast<float4 *>(ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot + C::kRingB + 4 * lane);
-                            const float4 s4 = *p4;
-                            *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
-                        }
-                        __syncwarp();
-                    }
-                }
+                for (int gi = 0; gi < G; ++gi) f[gi] = f_next[gi];
                 if (!ready) {
                     const bool got = mbar_wait(tfull_bar(a), (cc >> 1) & 1u, abort_flag);
                     if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
@@ -349,6 +359,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
                 uint32_t v[2][32];
                 tmem_ld32(taddr, v[0]);
+                if (SCALE != SCALE_NONE) {
+                    // In the shadow of the first load: next chunk's factors, so that no shared-memory or
+                    // special-function latency opens the next iteration.  Block mode has consumed this chunk's
+                    // slot into registers already and refills it now; vector mode still reads its column
+                    // reciprocals from the slot below and refills it at the end of the iteration.
+                    if (SCALE == SCALE_BLOCK_B) {
+                        prefetch_scales(c + C::kScaleDepth);
+                        cp_async_wait<C::kScaleDepth - 1>();
+                    } else {
+                        cp_async_wait<C::kScaleDepth - 2>();
+                    }
+                    __syncwarp();
+                    prepare_factors(c + 1, f_next);
+                    __syncwarp();   // every lane has read slot c+1 before a later refill may overwrite it
+                }
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) {
                     uint32_t (&cur)[32] = v[gi & 1];
@@ -392,7 +417,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 }
                 ready = __shfl_sync(0xFFFFFFFFu, early, 0) != 0;
-                if (SCALE != SCALE_NONE) {
+                if (SCALE == SCALE_VEC_B) {
                     __syncwarp();                       // every lane has read this slot
                     prefetch_scales(c + C::kScaleDepth); // refill it for a later chunk
                 }
