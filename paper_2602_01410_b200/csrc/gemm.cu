@@ -357,6 +357,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 tc_fence_after_sync();
                 uint32_t early = 0;
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
+                // two 32-column groups in registers next to the accumulators: one in flight, one being consumed
                 uint32_t v[2][32];
                 tmem_ld32(taddr, v[0]);
                 if (SCALE != SCALE_NONE) {
@@ -374,23 +375,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     prepare_factors(c + 1, f_next);
                     __syncwarp();   // every lane has read slot c+1 before a later refill may overwrite it
                 }
-#pragma unroll
-                for (int gi = 0; gi < G; ++gi) {
-                    uint32_t (&cur)[32] = v[gi & 1];
-                    tmem_ld_wait();
-                    if (gi + 1 < G) {
-                        tmem_ld32(taddr + 32 * (gi + 1), v[(gi + 1) & 1]);   // in flight during the FMAs below
-                    } else {
-                        // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) {
-                            mbar_arrive(tempty_bar(a));
-                            // non-blocking look at the next chunk's barrier: its shared-memory latency hides
-                            // behind the FMAs below instead of opening the next iteration
-                            early = mbar_test_wait(tfull_bar(a ^ 1u), ((cc + 1) >> 1) & 1u) ? 1u : 0u;
-                        }
+                // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
+                auto release_buffer = [&]() {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(tempty_bar(a));
+                        // non-blocking look at the next chunk's barrier: its shared-memory latency hides
+                        // behind the FMAs below instead of opening the next iteration
+                        early = mbar_test_wait(tfull_bar(a ^ 1u), ((cc + 1) >> 1) & 1u) ? 1u : 0u;
                     }
+                };
+                auto consume_group = [&](int gi, const uint32_t (&cur)[32]) {
                     if (SCALE == SCALE_NONE) {
                         float o[32];
 #pragma unroll
@@ -415,6 +411,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             acc[16 * gi + 2 * i + 1] = __ffma2_rn(p1, ff, acc[16 * gi + 2 * i + 1]);
                         }
                     }
+                };
+#pragma unroll
+                for (int gi = 0; gi < G; ++gi) {
+                    tmem_ld_wait();
+                    if (gi + 1 < G) tmem_ld32(taddr + 32 * (gi + 1), v[(gi + 1) & 1]);   // in flight during the FMAs below
+                    else release_buffer();
+                    consume_group(gi, v[gi & 1]);
                 }
                 ready = __shfl_sync(0xFFFFFFFFu, early, 0) != 0;
                 if (SCALE == SCALE_VEC_B) {
