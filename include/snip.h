@@ -374,6 +374,41 @@ int snip_adamw_sensitivity(const float *m, const float *v, const void *g, int g_
                            float beta1, float beta2, float eps, double *sumsq, void *ws, size_t ws_bytes,
                            void *stream);
 
+/* ---- scheme generation, host side (paper Sec. 4.2, 4.3, 5) --------------------------------- */
+
+/*
+ * Normalised loss divergence of one layer under one quantization option (Sec. 4.2):
+ *     sqrt( (|dL/dX|_F |X - q(X)|_F / sqrt(M K))^2 + (|dL/dW|_F |W - q(W)|_F / sqrt(N K))^2 ) / |L| .
+ * The gradient norms are the plain norms of dX and dW, the error norms come from snip_layer_stats /
+ * snip_quantize for that option.  Host arithmetic only.
+ */
+double snip_loss_divergence(double grad_x_norm, double err_x_norm, int64_t M, int64_t K,
+                            double grad_w_norm, double err_w_norm, int64_t N, double loss);
+
+/*
+ * Normalised weight divergence of one layer (Sec. 4.3):
+ *     (1/num_layers) * lr * sqrt(1 - beta2^step) / (1 - beta1^step) * |T|_F |g_err|_F / sqrt(N K) / |W|_F
+ * with |T|_F^2 from snip_adamw_sensitivity and |g_err|_F the error norm of the weight gradient under
+ * the option (how it is obtained - the paper adds noise-injection passes - is the caller's business).
+ */
+double snip_weight_divergence(double sens_norm, double grad_err_norm, int64_t N, int64_t K, double lr,
+                              double beta1, double beta2, int64_t step, double weight_norm,
+                              int64_t num_layers);
+
+/*
+ * One option per layer (Sec. 5.2): minimise sum_i q[i][choice[i]] subject to
+ * sum_i w[i][choice[i]] >= target, where q (m x n, row-major, finite, >= 0) is the quality loss and w
+ * (m x n, >= 0) the work that option moves to the cheaper format, as an integer (FLOPs run in FP4; the
+ * paper's e[i][j] is w[i][j] / total FLOPs and E_t = target / total FLOPs).  num_groups > 1 is the
+ * pipeline form (Sec. 5.3): m must be a multiple of it and every group of m / num_groups consecutive
+ * layers must reach ceil(target / num_groups) by itself.  Exact (Pareto-frontier dynamic programme
+ * over integer work); returns SNIP_ERR_UNSUPPORTED if the target cannot be reached or the frontier
+ * outgrows the solver's cap, SNIP_ERR_ARG / SNIP_ERR_SHAPE for malformed input.  Among assignments of
+ * equal loss any one may be returned.  choice: m ints; q_total / w_total may be NULL.  Host only.
+ */
+int snip_select_scheme(int m, int n, const double *q, const int64_t *w, int64_t target, int num_groups,
+                       int *choice, double *q_total, int64_t *w_total);
+
 /* ---- device status ------------------------------------------------------------------------ */
 
 /*

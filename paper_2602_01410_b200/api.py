@@ -25,7 +25,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
     "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
-    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace", "snip_adamw_sensitivity_workspace", "snip_adamw_sensitivity",
+    "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace", "snip_adamw_sensitivity_workspace", "snip_adamw_sensitivity", "snip_loss_divergence", "snip_weight_divergence", "snip_select_scheme",
     "snip_poll_status",
 )
 
@@ -91,6 +91,12 @@ def _load():
     lib.snip_layer_stats_workspace.argtypes = [i64, i64, i64, psz]
     lib.snip_adamw_sensitivity_workspace.argtypes = [i64, psz]
     lib.snip_adamw_sensitivity.argtypes = [vp, vp, vp, i32, i64, ctypes.c_float, ctypes.c_float, ctypes.c_float, vp, vp, sz, vp]
+    dbl = ctypes.c_double
+    lib.snip_loss_divergence.restype = dbl
+    lib.snip_loss_divergence.argtypes = [dbl, dbl, i64, i64, dbl, dbl, i64, dbl]
+    lib.snip_weight_divergence.restype = dbl
+    lib.snip_weight_divergence.argtypes = [dbl, dbl, i64, i64, dbl, dbl, dbl, i64, dbl, i64]
+    lib.snip_select_scheme.argtypes = [i32, i32, vp, vp, i64, i32, vp, vp, vp]
     lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -413,6 +419,28 @@ def snip_adamw_sensitivity(m: torch.Tensor, v: torch.Tensor, g: torch.Tensor, be
     _check("snip_adamw_sensitivity", _lib.snip_adamw_sensitivity(_p(m), _p(v), _p(g), OUT_BF16 if g.dtype == torch.bfloat16 else OUT_FP32, n, beta1, beta2,
                                                                  eps, _p(out), _p(ws), ws.numel(), _stream()))
     return out
+
+
+def snip_loss_divergence(grad_x_norm, err_x_norm, M, K, grad_w_norm, err_w_norm, N, loss) -> float:
+    return float(_lib.snip_loss_divergence(grad_x_norm, err_x_norm, M, K, grad_w_norm, err_w_norm, N, loss))
+
+
+def snip_weight_divergence(sens_norm, grad_err_norm, N, K, lr, beta1, beta2, step, weight_norm, num_layers) -> float:
+    return float(_lib.snip_weight_divergence(sens_norm, grad_err_norm, N, K, lr, beta1, beta2, step, weight_norm, num_layers))
+
+
+def snip_select_scheme(q, w, target: int, num_groups: int = 1):
+    """q: m x n floats, w: m x n ints.  Returns (choice list, total loss, total work)."""
+    import numpy as np
+    qa = np.ascontiguousarray(np.asarray(q, dtype=np.float64))
+    wa = np.ascontiguousarray(np.asarray(w, dtype=np.int64))
+    m, n = qa.shape
+    assert wa.shape == (m, n)
+    choice = np.zeros(m, dtype=np.int32)
+    qt, wt = ctypes.c_double(), ctypes.c_int64()
+    _check("snip_select_scheme", _lib.snip_select_scheme(m, n, qa.ctypes.data_as(ctypes.c_void_p), wa.ctypes.data_as(ctypes.c_void_p), int(target),
+                                                         num_groups, choice.ctypes.data_as(ctypes.c_void_p), ctypes.byref(qt), ctypes.byref(wt)))
+    return [int(c) for c in choice], qt.value, wt.value
 
 
 def snip_poll_status(ws: torch.Tensor) -> int:
