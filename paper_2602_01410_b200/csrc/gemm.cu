@@ -641,8 +641,13 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
         return f32 ? launch_gemm<MmaKind::F16, 256, SCALE_NONE, true>(tmA, tmB, tmO, g, idesc, st)
                    : launch_gemm<MmaKind::F16, 256, SCALE_NONE, false>(tmA, tmB, tmO, g, idesc, st);
     }
-    if (fmt_a == SNIP_FMT_FP4_E2M1 && fmt_b == SNIP_FMT_FP4_E2M1) {
-        // packed FP4 on both sides: kind::mxf4 at twice the FP8 rate; the bytes are fetched as plain u8
+    if (fmt_a == SNIP_FMT_FP4_E2M1 && fmt_b == SNIP_FMT_FP4_E2M1 && (Kc % 128) != 0) {
+        // Packed FP4 on both sides, contraction length ending in a 64-wide tile: kind::mxf4 on the packed bytes
+        // (fetched as plain u8, exact extents).  Whole chunks take the path below instead: the per-chunk
+        // promotion, not the tensor pipe, sets the pace of these kernels, and there a 128x256 tile of
+        // kind::f8f6f4 (FP4 codes expanded by the TMA unit, still fetched packed from L2) does a third more
+        // columns per hand-off than the 128x192 tile that tensor memory allows next to kind::mxf4's scale
+        // factors: measured 10-20 % faster on the 7B shapes.
         constexpr int BN = 192;
         rc = make_operand_map(&tmA, a_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, Kc / 2, Kc / 2, 128, BM);
         if (rc) return rc;
@@ -652,15 +657,16 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
         g.stage_tx_bytes = (BM + BN) * 128;
         return launch_gemm_scale<MmaKind::MXF4, BN>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
     }
-    // FP8 x FP8 and the mixed pairs: kind::f8f6f4; FP4 operands are expanded by the TMA unit to one
-    // 16-byte-aligned group per 16 elements, which is the layout this MMA kind reads
+    // FP8 x FP8, the mixed pairs and FP4 x FP4 over whole chunks: kind::f8f6f4; FP4 operands are expanded by
+    // the TMA unit to one 16-byte-aligned group per 16 elements, which is the layout this MMA kind reads
     constexpr int BN = 256;
     const bool a4 = fmt_a == SNIP_FMT_FP4_E2M1, b4 = fmt_b == SNIP_FMT_FP4_E2M1;
     // The expanding 4-bit tensor-map type only accepts an inner extent that is a multiple of 128
     // elements.  A contraction length ending in a 64-wide tile is therefore declared rounded up: the
     // extra 64 codes of each row are the first codes of the next row (for the last row, 32 bytes of
     // the slack that snip_quantize_sizes reserves); they meet zero-filled FP8 codes of the other
-    // operand, whose map has the exact extent, so they contribute nothing.
+    // operand, whose map has the exact extent, so they contribute nothing.  (Two FP4 operands with such a
+    // length never get here: both maps would be padded.)
     const int64_t kpad = ceil_div(Kc, 128) * 128;
     rc = make_operand_map(&tmA, a_codes, a4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, a4 ? kpad : Kc,
                           a4 ? Kc / 2 : Kc, 128, BM);
