@@ -279,6 +279,7 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 // Copy a 512-byte scale-factor atom (32 rows x 16 bytes, rows contiguous) from shared memory into
 // four tensor-memory columns, replicated into the four 32-lane quarters.  Runs in the tensor core's
 // queue, in issue order with the MMAs of the same thread.
+template <bool PAIR = false>
 __device__ __forceinline__ void tmem_cp_sf_atom(uint32_t taddr, uint32_t smem_addr)
 {
     // shared-memory matrix descriptor without swizzle: 8-row groups 128 bytes apart, one 16-byte column
@@ -287,7 +288,9 @@ __device__ __forceinline__ void tmem_cp_sf_atom(uint32_t taddr, uint32_t smem_ad
     d |= (uint64_t)(16 >> 4) << 16;     // leading byte offset (a single 16-byte column: unused)
     d |= (uint64_t)(128 >> 4) << 32;    // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;             // descriptor version for sm_100
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+    // PAIR: one instruction copies in both CTAs of the pair, each from its own shared memory (same offset)
+    if constexpr (PAIR) asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+    else asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
 }
 
 // ---- descriptors -----------------------------------------------------------------------
