@@ -555,11 +555,8 @@ int launch_gemm(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMa
 {
     using C = Cfg<KIND, BN, SCALE>;
     auto kern = gemm_kernel<KIND, BN, SCALE, OUT_F32>;
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-        attr_set = true;
-    }
+    // a per-function, per-device attribute; setting it on every launch is cheap and correct on any device
+    SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
     const int num_tiles = (int)(ceil_div(g.Mo, BM) * ceil_div(g.No, BN));
     const int grid = num_tiles < sm_count() ? num_tiles : sm_count();
     kern<<<grid, kGemmThreads, C::kSmemBytes, st>>>(tmA, tmB, tmO, g, idesc);

@@ -255,11 +255,8 @@ int launch_mx(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap 
 {
     using C = MxCfg<KIND>;
     auto kern = gemm_mx_kernel<KIND, OUT_F32>;
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-        attr_set = true;
-    }
+    // a per-function, per-device attribute; setting it on every launch is cheap and correct on any device
+    SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
     const int num_tiles = (int)(ceil_div(g.Mo, BM) * ceil_div(g.No, BN));
     const int grid = num_tiles < sms ? num_tiles : sms;
     kern<<<grid, kThreads, C::kSmemBytes, st>>>(tmA, tmB, tmO, g, idesc);
