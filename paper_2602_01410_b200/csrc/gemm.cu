@@ -294,7 +294,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const uint32_t slot = ring_u32 + d * C::kRingFloatsPerSlot * 4;
                     if (row_ok) cp_async_4(slot + lane * 4, g.sa + (int64_t)cn * g.sa_chunk_stride + row);
                     if (SCALE == SCALE_BLOCK_B) {
-                        if (lane < 2) {
+                        // a warp's HALF columns lie in one 128-wide block when HALF is a multiple of 128, else in two
+                        if (lane < ((HALF % 128) == 0 ? 1 : 2)) {
                             const int blk = min(blk0 + lane, blk_last);
                             cp_async_4(slot + (32 + lane) * 4, g.sb + (int64_t)blk * g.sb_blk_stride + (int64_t)cn * g.sb_chunk_stride);
                         }
@@ -324,9 +325,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 float *sl = ring + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot;
                 const float sa = sl[lane];
                 if (SCALE == SCALE_BLOCK_B) {
-                    const float f0 = __fdividef(1.0f, sa * sl[32]), f1 = __fdividef(1.0f, sa * sl[33]);
+                    const float f0 = __fdividef(1.0f, sa * sl[32]);
+                    if ((HALF % 128) == 0) {
 #pragma unroll
-                    for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
+                        for (int gi = 0; gi < G; ++gi) fo[gi] = f0;
+                    } else {
+                        const float f1 = __fdividef(1.0f, sa * sl[33]);
+#pragma unroll
+                        for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
+                    }
                 } else {
                     fo[0] = __fdividef(1.0f, sa);
                     if (4 * lane < HALF) {
