@@ -59,7 +59,10 @@ struct Cfg {
     static constexpr int kRingB = 36;                            // float offset of the per-column B scales in a slot
     // a slot holds 32 A scales, 4 block scales and, in vector mode, BN/2 column scales
     static constexpr int kRingFloatsPerSlot = (SCALE == 2) ? 36 + BN / 2 + 28 : 64;
-    static constexpr int kRingFloatsPerWarp = kScaleDepth * kRingFloatsPerSlot;
+    // block mode (fwd / dgrad) fetches four chunks of scale factors per instruction into two alternating group slots:
+    // [4 chunks][32 rows] S_a, then [2 blocks][4 chunks] S_b
+    static constexpr int kGroupFloats = 144;
+    static constexpr int kRingFloatsPerWarp = (SCALE == 1) ? 2 * kGroupFloats : kScaleDepth * kRingFloatsPerSlot;
     static constexpr int kSbInvBytes = kNumEpiWarps * kRingFloatsPerWarp * 4;
     // block mode (fwd / dgrad) writes its output through per-warp 2 KB staging tiles and TMA stores
     static constexpr bool kTmaOut = (SCALE == 1);
@@ -308,33 +311,59 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 cp_async_commit();
             };
 
+            // Block mode: the scale factors of four consecutive chunks with two instructions per warp.  Lane L
+            // fetches 16 bytes = S_a of rows 4*(L%8) .. +3 of chunk 4*gn + L/8 (the warp's 32 rows lie inside or
+            // outside the matrix together: row counts are multiples of 64); lanes 0..3 (0..7 with two blocks)
+            // fetch S_b of one chunk each.  Group gn lands in slot gn % 2.
+            constexpr int kBlocksPerWarp = ((HALF % 128) == 0) ? 1 : 2;
+            auto prefetch_group = [&](int gn) {
+                if (4 * gn < nacc) {
+                    const uint32_t slot = ring_u32 + (gn & 1) * C::kGroupFloats * 4;
+                    const int ci = lane >> 3, r4 = (lane & 7) * 4, chunk = 4 * gn + ci;
+                    if (row0 < g.Mo && chunk < nacc)
+                        cp_async_16(slot + (ci * 32 + r4) * 4, g.sa + (int64_t)chunk * g.sa_chunk_stride + row0 + r4);
+                    if (lane < 4 * kBlocksPerWarp) {
+                        const int blk = min(blk0 + (lane >> 2), blk_last), cb = 4 * gn + (lane & 3);
+                        if (cb < nacc) cp_async_4(slot + (128 + lane) * 4, g.sb + (int64_t)blk * g.sb_blk_stride + (int64_t)cb * g.sb_chunk_stride);
+                    }
+                }
+                cp_async_commit();
+            };
+
             float2 acc[SCALE == SCALE_NONE ? 1 : HALF / 2];
             if (SCALE != SCALE_NONE) {
 #pragma unroll
                 for (int i = 0; i < HALF / 2; ++i) acc[i] = make_float2(0.0f, 0.0f);
                 // out-of-range rows / columns read 1.0 (their products are zero anyway)
-                for (int i = lane; i < C::kScaleDepth * C::kRingFloatsPerSlot; i += 32) ring[i] = 1.0f;
+                for (int i = lane; i < C::kRingFloatsPerWarp; i += 32) ring[i] = 1.0f;
                 __syncwarp();
+                if (SCALE == SCALE_BLOCK_B) {
+                    prefetch_group(0);
+                    prefetch_group(1);
+                } else {
 #pragma unroll
-                for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
+                    for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
+                }
             }
             // Reciprocal scale factors of chunk cn from its ring slot (the slot must have landed).  Block mode:
             // one factor per 32-column group; vector mode: 1/S_a in fo[0], and the slot's column scales are
             // turned into reciprocals in place (4 per lane).
             auto prepare_factors = [&](int cn, float (&fo)[G]) {
-                float *sl = ring + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot;
-                const float sa = sl[lane];
                 if (SCALE == SCALE_BLOCK_B) {
-                    const float f0 = __fdividef(1.0f, sa * sl[32]);
-                    if ((HALF % 128) == 0) {
+                    const float *sl = ring + ((cn >> 2) & 1) * C::kGroupFloats;
+                    const float sa = sl[(cn & 3) * 32 + lane];
+                    const float f0 = __fdividef(1.0f, sa * sl[128 + (cn & 3)]);
+                    if (kBlocksPerWarp == 1) {
 #pragma unroll
                         for (int gi = 0; gi < G; ++gi) fo[gi] = f0;
                     } else {
-                        const float f1 = __fdividef(1.0f, sa * sl[33]);
+                        const float f1 = __fdividef(1.0f, sa * sl[132 + (cn & 3)]);
 #pragma unroll
                         for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
                     }
                 } else {
+                    float *sl = ring + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot;
+                    const float sa = sl[lane];
                     fo[0] = __fdividef(1.0f, sa);
                     if (4 * lane < HALF) {
                         float4 *p4 = reinterpret_cast<float4 *>(sl + C::kRingB + 4 * lane);
@@ -346,7 +375,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             };
             float f_next[G];
             if (SCALE != SCALE_NONE) {
-                cp_async_wait<C::kScaleDepth - 1>();   // chunk 0's scales
+                if (SCALE == SCALE_BLOCK_B) cp_async_wait<1>();   // group 0
+                else cp_async_wait<C::kScaleDepth - 1>();          // chunk 0
                 __syncwarp();
                 prepare_factors(0, f_next);
                 __syncwarp();
@@ -373,8 +403,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     // slot into registers already and refills it now; vector mode still reads its column
                     // reciprocals from the slot below and refills it at the end of the iteration.
                     if (SCALE == SCALE_BLOCK_B) {
-                        prefetch_scales(c + C::kScaleDepth);
-                        cp_async_wait<C::kScaleDepth - 1>();
+                        // chunk c is the last of its group: every lane took its factors in the previous iteration,
+                        // so the group's slot is refilled (two groups ahead) and the next group must have landed
+                        if ((c & 3) == 3) {
+                            prefetch_group((c >> 2) + 2);
+                            cp_async_wait<1>();
+                        }
                     } else {
                         cp_async_wait<C::kScaleDepth - 2>();
                     }
@@ -618,6 +652,7 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     const bool a16 = fmt_a == SNIP_FMT_BF16, b16 = fmt_b == SNIP_FMT_BF16;
     if (a16 != b16) return SNIP_ERR_UNSUPPORTED;
     if (!a16 && (!sa || !sb)) return SNIP_ERR_ARG;
+    if (!a16 && (!aligned16(sa) || !aligned16(sb))) return SNIP_ERR_ALIGN;   // scale factors are fetched 16 bytes at a time
     int rc = require_sm100();
     if (rc != SNIP_OK) return rc;
 
