@@ -56,13 +56,13 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = (BN >= 256) ? 4 : 5;
     static constexpr int kScaleDepth = 4;                        // chunks of scale factors in flight per warp
-    static constexpr int kRingB = 36;                            // float offset of the per-column B scales in a slot
+    static constexpr int kRingB = 256;                           // vector mode: float offset of the per-column B scale slots (after two S_a groups)
     // a slot holds 32 A scales, 4 block scales and, in vector mode, BN/2 column scales
-    static constexpr int kRingFloatsPerSlot = (SCALE == 2) ? 36 + BN / 2 + 28 : 64;
+    static constexpr int kRingFloatsPerSlot = (SCALE == 2) ? BN / 2 : 64;   // vector mode: one chunk's column scales of a warp
     // block mode (fwd / dgrad) fetches four chunks of scale factors per instruction into two alternating group slots:
     // [4 chunks][32 rows] S_a, then [2 blocks][4 chunks] S_b
     static constexpr int kGroupFloats = 144;
-    static constexpr int kRingFloatsPerWarp = (SCALE == 1) ? 2 * kGroupFloats : kScaleDepth * kRingFloatsPerSlot;
+    static constexpr int kRingFloatsPerWarp = (SCALE == 1) ? 2 * kGroupFloats : kRingB + kScaleDepth * kRingFloatsPerSlot;
     static constexpr int kSbInvBytes = kNumEpiWarps * kRingFloatsPerWarp * 4;
     // block mode (fwd / dgrad) writes its output through per-warp 2 KB staging tiles and TMA stores
     static constexpr bool kTmaOut = (SCALE == 1);
@@ -269,11 +269,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int e = warp - 4;          // 0..7
         const int q = warp & 3;          // tensor-memory lane quarter this warp may access
         const int h = e >> 2;            // column half
-        // Per-warp ring of scale factors, filled kScaleDepth chunks ahead with cp.async so that no
-        // global-memory latency sits between two chunks:
-        //   [d][0..31]               S_a of this warp's 32 rows
-        //   [d][32..35]              S_b of the (at most two) 128-column blocks this warp covers (block mode)
-        //   [d][kRingB..kRingB+HALF) S_b of this warp's HALF output columns (vector mode)
+        // Per-warp scale-factor buffers, filled ahead with cp.async so that no global-memory latency sits
+        // between two chunks.  S_a of this warp's 32 rows comes four chunks at a time into two alternating
+        // group slots [4 chunks][32 rows]; block mode keeps the S_b of its one or two 128-column blocks next
+        // to them ([2 blocks][4 chunks] at float 128 of the group), vector mode keeps kScaleDepth per-chunk
+        // slots of HALF column scales from float kRingB on.
         float *ring = scale_ring + e * C::kRingFloatsPerWarp;
         const uint32_t ring_u32 = smem_u32(ring);
         const uint32_t stage_u32 = out_stage0 + e * 2048;   // this warp's staging tile: 32 rows x 64 bytes
@@ -291,21 +291,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int blk0 = col0 >> 7;
             const int blk_last = (g.No - 1) >> 7;
 
+            // Vector mode (wgrad): chunk cn's column scales (one 16-byte copy per lane) and, with every fourth chunk,
+            // the S_a of four chunks (as in block mode, see below) travel in one commit group.
             auto prefetch_scales = [&](int cn) {
-                if (SCALE != SCALE_NONE && cn < nacc) {
-                    const int d = cn % C::kScaleDepth;
-                    const uint32_t slot = ring_u32 + d * C::kRingFloatsPerSlot * 4;
-                    if (row_ok) cp_async_4(slot + lane * 4, g.sa + (int64_t)cn * g.sa_chunk_stride + row);
-                    if (SCALE == SCALE_BLOCK_B) {
-                        // a warp's HALF columns lie in one 128-wide block when HALF is a multiple of 128, else in two
-                        if (lane < ((HALF % 128) == 0 ? 1 : 2)) {
-                            const int blk = min(blk0 + lane, blk_last);
-                            cp_async_4(slot + (32 + lane) * 4, g.sb + (int64_t)blk * g.sb_blk_stride + (int64_t)cn * g.sb_chunk_stride);
-                        }
-                    } else if (SCALE == SCALE_VEC_B) {
-                        const int n = col0 + 4 * lane;
-                        if (4 * lane < HALF && n < g.No)
-                            cp_async_16(slot + (C::kRingB + 4 * lane) * 4, g.sb + (int64_t)cn * g.sb_chunk_stride + n);
+                if (SCALE == SCALE_VEC_B && cn < nacc) {
+                    const uint32_t slot = ring_u32 + (C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot) * 4;
+                    const int n = col0 + 4 * lane;
+                    if (4 * lane < HALF && n < g.No) cp_async_16(slot + 4 * lane * 4, g.sb + (int64_t)cn * g.sb_chunk_stride + n);
+                    if ((cn & 3) == 0) {
+                        const uint32_t grp = ring_u32 + ((cn >> 2) & 1) * 128 * 4;
+                        const int ci = lane >> 3, r4 = (lane & 7) * 4, chunk = cn + ci;
+                        if (row0 < g.Mo && chunk < nacc) cp_async_16(grp + (ci * 32 + r4) * 4, g.sa + (int64_t)chunk * g.sa_chunk_stride + row0 + r4);
                     }
                 }
                 cp_async_commit();
@@ -362,11 +358,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
                     }
                 } else {
-                    float *sl = ring + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot;
-                    const float sa = sl[lane];
+                    const float sa = ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane];
                     fo[0] = __fdividef(1.0f, sa);
                     if (4 * lane < HALF) {
-                        float4 *p4 = reinterpret_cast<float4 *>(sl + C::kRingB + 4 * lane);
+                        float4 *p4 = reinterpret_cast<float4 *>(ring + C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot + 4 * lane);
                         const float4 s4 = *p4;
                         *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
                     }
@@ -384,7 +379,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int c = 0; c < nacc; ++c, ++cc) {
                 const uint32_t a = cc & 1u;
                 float f[G];
-                const float *slot = ring + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;
+                const float *slot = ring + C::kRingB + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;   // vector mode: this chunk's column reciprocals
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) f[gi] = f_next[gi];
                 if (!ready) {
@@ -440,7 +435,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             acc[16 * gi + i] = __ffma2_rn(make_float2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), ff, acc[16 * gi + i]);
                     } else {
                         const float2 ff = make_float2(f[0], f[0]);
-                        const float4 *sbv = reinterpret_cast<const float4 *>(slot + C::kRingB + 32 * gi);
+                        const float4 *sbv = reinterpret_cast<const float4 *>(slot + 32 * gi);
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const float4 s4 = sbv[i];   // reciprocal column scales, broadcast read
