@@ -239,8 +239,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
                             mma_ss<KIND, false>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, k > 0 ? 1u : 0u, 0, 0);
+                        // one commit serves both hand-offs (a stage is one chunk here): the producer takes it as
+                        // "stage s is free", the epilogue warps as "the chunk's partial sums are complete"
                         tc_commit<false>(empty_bar(s));
-                        tc_commit<false>(tfull_bar(a));
                         ++cc;
                     } else {
 #pragma unroll
@@ -382,8 +383,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const float *slot = ring + C::kRingB + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;   // vector mode: this chunk's column reciprocals
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) f[gi] = f_next[gi];
+                // barrier that announces this chunk's partial sums (see the MMA issuer) and the one of the next chunk
+                const uint32_t done_bar = (KIND == MmaKind::F8F6F4) ? empty_bar(cc % S) : tfull_bar(a);
+                const uint32_t done_par = (KIND == MmaKind::F8F6F4) ? ((cc / S) & 1u) : ((cc >> 1) & 1u);
+                const uint32_t next_bar = (KIND == MmaKind::F8F6F4) ? empty_bar((cc + 1) % S) : tfull_bar(a ^ 1u);
+                const uint32_t next_par = (KIND == MmaKind::F8F6F4) ? (((cc + 1) / S) & 1u) : (((cc + 1) >> 1) & 1u);
                 if (!ready) {
-                    const bool got = mbar_wait(tfull_bar(a), (cc >> 1) & 1u, abort_flag);
+                    const bool got = mbar_wait(done_bar, done_par, abort_flag);
                     if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
                 }
                 tc_fence_after_sync();
@@ -419,7 +425,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         mbar_arrive(tempty_bar(a));
                         // non-blocking look at the next chunk's barrier: its shared-memory latency hides
                         // behind the FMAs below instead of opening the next iteration
-                        early = mbar_test_wait(tfull_bar(a ^ 1u), ((cc + 1) >> 1) & 1u) ? 1u : 0u;
+                        early = mbar_test_wait(next_bar, next_par) ? 1u : 0u;
                     }
                 };
                 auto consume_group = [&](int gi, const uint32_t (&cur)[32]) {
