@@ -359,23 +359,32 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
                     }
                 } else {
-                    const float sa = ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane];
-                    fo[0] = __fdividef(1.0f, sa);
-                    if (4 * lane < HALF) {
-                        float4 *p4 = reinterpret_cast<float4 *>(ring + C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot + 4 * lane);
-                        const float4 s4 = *p4;
-                        *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
-                    }
-                    __syncwarp();
+                    fo[0] = __fdividef(1.0f, ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane]);
                 }
             };
+            // Vector mode: turns chunk cn's column scales into reciprocals in place (4 per lane).  Done two chunks
+            // ahead of their use, at the end of an iteration, so that the load - reciprocal - store chain never
+            // sits in front of FMAs.
+            auto convert_columns = [&](int cn) {
+                if (4 * lane < HALF) {
+                    float4 *p4 = reinterpret_cast<float4 *>(ring + C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot + 4 * lane);
+                    const float4 s4 = *p4;
+                    *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
+                }
+                __syncwarp();
+            };
             float f_next[G];
-            if (SCALE != SCALE_NONE) {
-                if (SCALE == SCALE_BLOCK_B) cp_async_wait<1>();   // group 0
-                else cp_async_wait<C::kScaleDepth - 1>();          // chunk 0
+            if (SCALE == SCALE_BLOCK_B) {
+                cp_async_wait<1>();   // group 0
                 __syncwarp();
                 prepare_factors(0, f_next);
                 __syncwarp();
+            } else if (SCALE == SCALE_VEC_B) {
+                cp_async_wait<C::kScaleDepth - 2>();   // chunks 0 and 1
+                __syncwarp();
+                convert_columns(0);
+                convert_columns(1);
+                prepare_factors(0, f_next);
             }
             for (int c = 0; c < nacc; ++c, ++cc) {
                 const uint32_t a = cc & 1u;
@@ -410,12 +419,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             prefetch_group((c >> 2) + 2);
                             cp_async_wait<1>();
                         }
+                        __syncwarp();
+                        prepare_factors(c + 1, f_next);
+                        __syncwarp();   // every lane has read its factors before a later refill may overwrite the slot
                     } else {
-                        cp_async_wait<C::kScaleDepth - 2>();
+                        prepare_factors(c + 1, f_next);   // 1/S_a only; its group landed with an earlier chunk
                     }
-                    __syncwarp();
-                    prepare_factors(c + 1, f_next);
-                    __syncwarp();   // every lane has read slot c+1 before a later refill may overwrite it
                 }
                 // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
                 auto release_buffer = [&]() {
@@ -463,8 +472,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 ready = __shfl_sync(0xFFFFFFFFu, early, 0) != 0;
                 if (SCALE == SCALE_VEC_B) {
-                    __syncwarp();                       // every lane has read this slot
-                    prefetch_scales(c + C::kScaleDepth); // refill it for a later chunk
+                    cp_async_wait<1>();                  // chunk c+2 has landed (c+3 may be in flight)
+                    __syncwarp();                        // ... for every lane, and every lane has read slot c
+                    convert_columns(c + 2);
+                    prefetch_scales(c + C::kScaleDepth); // refill slot c for a later chunk
                 }
             }
             if (SCALE != SCALE_NONE) {
