@@ -89,6 +89,15 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int &m_
     n_idx = r / gm;
 }
 
+// Reciprocal from the special-function unit (one instruction, ~1 ulp; a subnormal result is flushed to zero,
+// which only affects products of scales beyond FP32's range).
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -349,17 +358,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (SCALE == SCALE_BLOCK_B) {
                     const float *sl = ring + ((cn >> 2) & 1) * C::kGroupFloats;
                     const float sa = sl[(cn & 3) * 32 + lane];
-                    const float f0 = __fdividef(1.0f, sa * sl[128 + (cn & 3)]);
+                    const float f0 = rcp_approx(sa * sl[128 + (cn & 3)]);
                     if (kBlocksPerWarp == 1) {
 #pragma unroll
                         for (int gi = 0; gi < G; ++gi) fo[gi] = f0;
                     } else {
-                        const float f1 = __fdividef(1.0f, sa * sl[132 + (cn & 3)]);
+                        const float f1 = rcp_approx(sa * sl[132 + (cn & 3)]);
 #pragma unroll
                         for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
                     }
                 } else {
-                    fo[0] = __fdividef(1.0f, ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane]);
+                    fo[0] = rcp_approx(ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane]);
                 }
             };
             // Vector mode: turns chunk cn's column scales into reciprocals in place (4 per lane).  Done two chunks
@@ -369,7 +378,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (4 * lane < HALF) {
                     float4 *p4 = reinterpret_cast<float4 *>(ring + C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot + 4 * lane);
                     const float4 s4 = *p4;
-                    *p4 = make_float4(__fdividef(1.0f, s4.x), __fdividef(1.0f, s4.y), __fdividef(1.0f, s4.z), __fdividef(1.0f, s4.w));
+                    *p4 = make_float4(rcp_approx(s4.x), rcp_approx(s4.y), rcp_approx(s4.z), rcp_approx(s4.w));
                 }
                 __syncwarp();
             };
