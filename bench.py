@@ -670,6 +670,12 @@ def main():
     if not args.no_cpu_baseline:
         v, cores, sample = cpu_baseline_sample(cfg)
         cpu = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+        # the same oracle on one core, on an eighth of the sample
+        from oracle import snip_oracle as orc
+        orc.set_num_threads(1)
+        v1, _, sample1 = cpu_baseline_sample(cfg, tokens=512)
+        orc.set_num_threads(cores)
+        cpu["one_core"] = {"value": v1, "unit": "TFLOP/s", "cores": 1, "sample": sample1}
 
     line = {"metric": "mixed-precision linear fwd+dgrad+wgrad TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

@@ -539,6 +539,17 @@ double orc_adamw_sensitivity_sumsq(const double *m, const double *v, const doubl
     return acc;
 }
 
+/* Number of threads the parallel loops use from now on (timing aid: the benchmark also reports a
+ * one-core figure).  No effect without OpenMP. */
+void orc_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

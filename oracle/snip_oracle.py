@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.orc_sumsq_bf16.argtypes = [vp, i64]
         L.orc_adamw_sensitivity_sumsq.restype = dbl
         L.orc_adamw_sensitivity_sumsq.argtypes = [vp, vp, vp, i64, dbl, dbl, dbl]
+        L.orc_set_num_threads.restype = None
+        L.orc_set_num_threads.argtypes = [i32]
         L.orc_num_threads.restype = i32
         L.orc_num_threads.argtypes = []
         _lib = L
@@ -93,6 +95,10 @@ def lib() -> ctypes.CDLL:
 
 def _ptr(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def set_num_threads(n: int) -> None:
+    lib().orc_set_num_threads(n)
 
 
 def num_threads() -> int:
