@@ -308,11 +308,11 @@ class KernelTimer:
         assert api.snip_poll_status(ws) == 0
         return 2.0 * M * N * K, times
 
-    def quantizer(self, fmt, block, transposed, rows, cols, iters=20, warmup=3):
+    def quantizer(self, fmt, block, transposed, rows, cols, iters=20, warmup=3, stats=True):
         api, torch = self.api, self.torch
         g = torch.Generator(device=self.device); g.manual_seed(2)
         xs = [torch.randn(rows, cols, generator=g, device=self.device, dtype=torch.float32).to(torch.bfloat16) for _ in range(3)]
-        flags = api.Q_STATS | (api.Q_TRANSPOSED if transposed else 0)
+        flags = (api.Q_STATS if stats else 0) | (api.Q_TRANSPOSED if transposed else 0)
         codes, scales, stats, _ = api.snip_quantize(xs[0], fmt, block, flags)
         _, _, wb = api.snip_quantize_sizes(rows, cols, fmt, block, flags)
         ws = torch.empty(wb, dtype=torch.uint8, device=self.device)
@@ -333,12 +333,12 @@ class KernelTimer:
         return bytes_per_elt * rows * cols, times
 
 
-    def quantizer_dual(self, fmt, kind, rows, cols, iters=20, warmup=3):
-        """snip_quantize_dual with statistics, timed like quantizer(); bytes = one read + two outputs."""
+    def quantizer_dual(self, fmt, kind, rows, cols, iters=20, warmup=3, stats=True):
+        """snip_quantize_dual (with statistics unless stats=False), timed like quantizer(); bytes = one read + two outputs."""
         api, torch = self.api, self.torch
         g = torch.Generator(device=self.device); g.manual_seed(2)
         xs = [torch.randn(rows, cols, generator=g, device=self.device, dtype=torch.float32).to(torch.bfloat16) for _ in range(3)]
-        bufs = api.snip_quantize_dual(xs[0], kind, fmt, fmt)
+        bufs = api.snip_quantize_dual(xs[0], kind, fmt, fmt, want_stats=stats)
         ws = torch.empty(api.snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=self.device)
         times = []
         batch = 6
@@ -402,10 +402,13 @@ def run_profile_case(name):
         return run_layer_stats_case(api, torch, device, parts[2] if len(parts) > 2 else "x")
     mx = parts[1].startswith("mx")
     fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4, "mxfp8": FMT_FP8, "mxfp4": FMT_FP4}[parts[1]]
+    nostats = parts[-1] == "nostats"
+    if nostats:
+        parts = parts[:-1]
     if parts[0] == "quantize" and parts[2] == "dual":
         kt = KernelTimer(api, torch, wl.CONFIGS[3], device)
         kind = api.DUAL_BLK_BLKT if parts[-1] == "blk" else api.DUAL_ROW_COLT
-        by, times = kt.quantizer_dual(fmt, kind, 16384, 4096, iters=3, warmup=1)
+        by, times = kt.quantizer_dual(fmt, kind, 16384, 4096, iters=3, warmup=1, stats=not nostats)
         print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
     elif parts[0] == "quantize" and parts[2] == "sr":
         # stochastic rounding (FP4): quantize_fp4_sr_row | quantize_fp4_sr_col_t
@@ -431,7 +434,7 @@ def run_profile_case(name):
         block, tr = {"row": (api.BLOCK_ROW, False), "col_t": (api.BLOCK_COL, True), "blk_t": (api.BLOCK_BLK, True),
                      "blk": (api.BLOCK_BLK, False), "col": (api.BLOCK_COL, False)}[kind]
         kt = KernelTimer(api, torch, wl.CONFIGS[3], device)
-        by, times = kt.quantizer(fmt, block, tr, 16384, 4096, iters=3, warmup=1)
+        by, times = kt.quantizer(fmt, block, tr, 16384, 4096, iters=3, warmup=1, stats=not nostats)
         print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
     else:
         op = {"fwd": api.OP_FWD, "dgrad": api.OP_DGRAD, "wgrad": api.OP_WGRAD}[parts[2]]
@@ -665,6 +668,13 @@ def main():
                 by, times = kt.quantizer_dual(f, kind, cfg.M, 4096)
                 avg = sum(times) / len(times)
                 kernels[f"quantize_dual_{FMT_NAME[f]}_{name}"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
+            # the same quantizers without the fused statistics (the paper collects them at intervals, Sec. 3.1)
+            by, times = kt.quantizer(f, api.BLOCK_ROW, False, cfg.M, 4096, stats=False)
+            avg = sum(times) / len(times)
+            kernels[f"quantize_{FMT_NAME[f]}_row_nostats"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
+            by, times = kt.quantizer_dual(f, api.DUAL_ROW_COLT, cfg.M, 4096, stats=False)
+            avg = sum(times) / len(times)
+            kernels[f"quantize_dual_{FMT_NAME[f]}_row+col_t_nostats"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
 
     cpu = None
     if not args.no_cpu_baseline:
