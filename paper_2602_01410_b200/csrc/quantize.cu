@@ -34,12 +34,13 @@ struct CtaPartial {  // one per CTA, reduced in fixed order by stats_reduce_kern
 
 struct QuantArgs {
     const uint16_t *x;
-    int64_t rows, cols, ld;
+    int32_t rows, cols, ld;   // 32-bit (checked on the host): index products are 32 x 32 -> 64-bit multiplies
     uint8_t *codes;       // may be null (NO_CODES)
     float *scales;        // may be null (NO_CODES)
     CtaPartial *partials; // may be null (no stats)
     float2 *row_partials; // [col tiles][rows] {sum x^2, sum err^2}; may be null
-    int64_t tiles_r, tiles_c, ntiles;
+    int32_t tiles_r, tiles_c;
+    int64_t ntiles;
     uint64_t seed;        // stochastic rounding: key of the generator
     int pow2;             // 1: power-of-two scale rule (largest 2^e with amax * 2^e <= FPX_MAX)
     uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
@@ -73,7 +74,7 @@ __device__ __forceinline__ void prefetch_tile(const QuantArgs &a, int tr, int tc
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     const int64_t rbase = (int64_t)tr * kTile + 8 * ty, cbase = (int64_t)tc * kTile + 8 * tx;
     const bool ok = cbase < a.cols && rbase < a.rows;       // dims are multiples of 64: all 64 elements or none
-    const uint16_t *xb = a.x + (ok ? rbase * a.ld + cbase : 0);
+    const uint16_t *xb = a.x + (ok ? (int64_t)(int32_t)rbase * a.ld + cbase : 0);
     const uint32_t ld32 = (uint32_t)a.ld;
     const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage_base) + tid * 16;
     const int nbytes = ok ? 16 : 0;                          // 0: the slot is zero-filled, nothing is read
@@ -156,13 +157,18 @@ __device__ __forceinline__ void pack8(const uint32_t (&c)[4], uint32_t (&out)[2]
     }
 }
 
-// Stores this thread's 8x8 codes as stored (row-major): one 8-byte (FP8) or 4-byte (FP4) store per row.
+// Address of this thread's codes of row rbase in the as-stored (row-major) output; row p follows p * out_ld bytes later.
 template <int FMT>
-__device__ __forceinline__ void store_row(const QuantArgs &a, int64_t rbase, int64_t cbase, int p, const uint32_t (&code)[2])
+__device__ __forceinline__ uint8_t *row_store_base(const QuantArgs &a, int64_t rbase, int64_t cbase, uint32_t &out_ld)
 {
     constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;
-    const int64_t out_ld = a.cols * kCodeBytes8 / 8;
-    uint8_t *dst = a.codes + (rbase + p) * out_ld + cbase * kCodeBytes8 / 8;
+    out_ld = (uint32_t)(a.cols * kCodeBytes8 / 8);
+    return a.codes + (uint64_t)(uint32_t)rbase * out_ld + (uint32_t)cbase * kCodeBytes8 / 8;
+}
+// One 8-byte (FP8) or 4-byte (FP4) store per row.
+template <int FMT>
+__device__ __forceinline__ void store_row(uint8_t *dst, const uint32_t (&code)[2])
+{
     if (FMT == SNIP_FMT_FP8_E4M3) *reinterpret_cast<uint2 *>(dst) = make_uint2(code[0], code[1]);
     else *reinterpret_cast<uint32_t *>(dst) = code[0];
 }
@@ -225,10 +231,10 @@ __device__ __forceinline__ void write_transposed(const QuantArgs &a, const uint8
     constexpr int kCodeBytes8 = (FMT == SNIP_FMT_FP8_E4M3) ? 8 : 4;
     constexpr int kRowBytes = kTile * kCodeBytes8 / 8;
     constexpr int kChunks = kRowBytes / 16;
-    const int64_t out_ld = a.rows * kCodeBytes8 / 8;
+    const uint32_t out_ld = (uint32_t)a.rows * kCodeBytes8 / 8;
     const int valid_rows = (int)min((int64_t)kTile, a.rows - r0);   // rows is a multiple of 64
     const int valid_cols = (int)min((int64_t)kTile, a.cols - c0);
-    uint8_t *base = a.codes + c0 * out_ld + r0 * kCodeBytes8 / 8;
+    uint8_t *base = a.codes + (uint64_t)(uint32_t)c0 * out_ld + (uint32_t)r0 * kCodeBytes8 / 8;
 #pragma unroll
     for (int idx = threadIdx.x; idx < kTile * kChunks; idx += kThreads) {
         const int c = idx / kChunks, q = idx % kChunks;
@@ -245,7 +251,7 @@ __device__ __forceinline__ void write_transposed(const QuantArgs &a, const uint8
             o = make_uint4(src[(4 * q) ^ key], src[(4 * q + 1) ^ key], src[(4 * q + 2) ^ key], src[(4 * q + 3) ^ key]);
             ok = ok && 32 * q < valid_rows;
         }
-        if (ok) *reinterpret_cast<uint4 *>(base + (int64_t)c * out_ld + 16 * q) = o;
+        if (ok) *reinterpret_cast<uint4 *>(base + (uint64_t)(uint32_t)c * out_ld + 16 * q) = o;
     }
 }
 
@@ -429,6 +435,10 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
     // ---- encode, statistics, as-stored codes ------------------------------------------------------
     uint32_t keep[8][2];   // codes of the transposed output, held until the sub-block is complete
     (void)keep;
+    uint32_t ld_a = 0, ld_b = 0;
+    uint8_t *dst_a = (A::kQuant && A::CODES && !A::TRANSPOSED) ? row_store_base<A::FMT>(qa, rbase, cbase, ld_a) : nullptr;
+    uint8_t *dst_b = (B::kQuant && B::CODES && !B::TRANSPOSED) ? row_store_base<B::FMT>(qb, rbase, cbase, ld_b) : nullptr;
+    (void)dst_a; (void)dst_b;
     float2 sx2 = make_float2(0.0f, 0.0f), sea2 = make_float2(0.0f, 0.0f), seb2 = make_float2(0.0f, 0.0f);
     float rsx[8], rse[8];
     (void)rsx; (void)rse;
@@ -467,13 +477,13 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
             uint32_t code[2];
             pack8<A::FMT>(ca, code);
             if (A::TRANSPOSED) { keep[p][0] = code[0]; keep[p][1] = code[1]; }
-            else if (in_range) store_row<A::FMT>(qa, rbase, cbase, p, code);
+            else if (in_range) store_row<A::FMT>(dst_a + p * ld_a, code);
         }
         if (B::kQuant && B::CODES) {
             uint32_t code[2];
             pack8<B::FMT>(cb, code);
             if (B::TRANSPOSED) { keep[p][0] = code[0]; keep[p][1] = code[1]; }
-            else if (in_range) store_row<B::FMT>(qb, rbase, cbase, p, code);
+            else if (in_range) store_row<B::FMT>(dst_b + p * ld_b, code);
         }
     }
     after_reads();
@@ -768,7 +778,7 @@ int quantize_impl_full(const void *x, int64_t rows, int64_t cols, int64_t ld, in
         if (!pow2 || !aligned16(sf) || (block == SNIP_BLOCK_ROW_1x128 && tr) || (block == SNIP_BLOCK_COL_128x1 && !tr)) return SNIP_ERR_UNSUPPORTED;
     }
     if (!x || !valid_fmt(fmt) || !valid_block(block)) return SNIP_ERR_ARG;
-    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0) return SNIP_ERR_SHAPE;
+    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
     const bool want_stats = (flags & SNIP_Q_STATS) != 0;
     const bool want_rows = row_stats != nullptr;
     const bool want_codes = fmt != SNIP_FMT_BF16 && !(flags & SNIP_Q_NO_CODES);
@@ -789,14 +799,14 @@ int quantize_impl_full(const void *x, int64_t rows, int64_t cols, int64_t ld, in
     const int64_t tr = ceil_div(rows, kTile), tc = ceil_div(cols, kTile);
     QuantArgs a;
     a.x = static_cast<const uint16_t *>(x);
-    a.rows = rows; a.cols = cols; a.ld = ld;
+    a.rows = (int32_t)rows; a.cols = (int32_t)cols; a.ld = (int32_t)ld;
     a.pow2 = pow2; a.sf = static_cast<uint32_t *>(sf);
     a.seed = seed;
     a.codes = want_codes ? static_cast<uint8_t *>(codes) : nullptr;
     a.scales = want_codes ? scales : nullptr;
     a.partials = any_stats ? static_cast<CtaPartial *>(ws) : nullptr;
     a.row_partials = want_rows ? reinterpret_cast<float2 *>(static_cast<uint8_t *>(ws) + align_up((size_t)(tr * tc) * sizeof(CtaPartial), 256)) : nullptr;
-    a.tiles_r = tr; a.tiles_c = tc; a.ntiles = tr * tc;
+    a.tiles_r = (int32_t)tr; a.tiles_c = (int32_t)tc; a.ntiles = tr * tc;
     const int64_t nparts = persistent_ctas(tr * tc);
     dim3 grid((unsigned)nparts);
     if (sr) {
@@ -855,7 +865,7 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bo
                        void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (!x) return SNIP_ERR_ARG;
-    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0) return SNIP_ERR_SHAPE;
+    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
     const DualOut *o[2] = {&oa, &ob};
     for (int i = 0; i < 2; ++i) {
         if (o[i]->fmt != SNIP_FMT_FP8_E4M3 && o[i]->fmt != SNIP_FMT_FP4_E2M1) return SNIP_ERR_UNSUPPORTED;
@@ -878,7 +888,7 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bo
     for (int i = 0; i < 2; ++i) {
         QuantArgs &q = i ? d.b : d.a;
         q.x = static_cast<const uint16_t *>(x);
-        q.rows = rows; q.cols = cols; q.ld = ld;
+        q.rows = (int32_t)rows; q.cols = (int32_t)cols; q.ld = (int32_t)ld;
         q.codes = static_cast<uint8_t *>(o[i]->codes);
         q.scales = o[i]->scales;
         q.partials = stats ? reinterpret_cast<CtaPartial *>(static_cast<uint8_t *>(ws) + i * one) : nullptr;
@@ -886,7 +896,7 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bo
         q.pow2 = pow2;
         q.seed = o[i]->seed;
         q.sf = static_cast<uint32_t *>(o[i]->sf);
-        q.tiles_r = tr; q.tiles_c = tc; q.ntiles = tr * tc;
+        q.tiles_r = (int32_t)tr; q.tiles_c = (int32_t)tc; q.ntiles = tr * tc;
     }
     const int64_t nparts = persistent_ctas(tr * tc, kDualCtasPerSm);
     dim3 grid((unsigned)nparts);
