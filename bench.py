@@ -12,7 +12,9 @@ Prints ONE JSON line (rank 0).  `value` is GEMM TFLOP/s (2*M*N*K per GEMM) over 
 quantizers and statistics included, with inputs resident in HBM.  `roofline` describes the
 dominant kernel family (the GEMM kernels of the slower format), timed with CUDA events around
 each launch inside the timed region.  `e2e` repeats the step through the snip_linear_* calls with
-the inputs starting in pinned host memory.  `cpu_baseline` times the CPU oracle on a bounded
+the inputs starting in pinned host memory: every step copies all of them to the device (on a copy
+stream, into one of two input sets, so that the copy of one step overlaps the kernels of the
+previous one) and reads the statistics back.  `cpu_baseline` times the CPU oracle on a bounded
 sample on this machine's host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 7b|1b|small]
@@ -158,21 +160,28 @@ class Step:
         self.launches_per_step = n_gemm * (3 if dual else 5)
 
     # -- the step through the snip_linear_* entry points (what a user calls) -------------
-    def run_linear_calls(self, mx=False):
+    def run_linear_calls(self, mx=False, inputs=None, before=None):
+        """One step through the per-layer entry points.  `inputs` replaces the resident input tensors;
+        `before(j)` runs ahead of the first call that reads linear j's inputs (end-to-end leg: wait for their copy)."""
         api = self.api
         i = 0
+        inputs = self.inputs if inputs is None else inputs
         if self.dual:
             lib, p, st = api._lib, api._p, api._stream()
-            for f in self.formats:
-                for (x, w, dy), (y, dx, dw) in zip(self.inputs, self.out):
+            for fi, f in enumerate(self.formats):
+                for j, ((x, w, dy), (y, dx, dw)) in enumerate(zip(inputs, self.out)):
+                    if before is not None and fi == 0:
+                        before(j)
                     M, K = x.shape
                     N = w.shape[0]
                     api._check("snip_linear_fwd_bwd", lib.snip_linear_fwd_bwd(p(x), p(w), p(dy), p(y), p(dx), p(dw), M, N, K, f, f, f, api.OUT_BF16,
                                                                               int(mx), 0, 0, p(self.stats6[i]), p(self.ws), self.ws.numel(), st))
                     i += 1
             return
-        for f in self.formats:
-            for (x, w, dy), (y, dx, dw) in zip(self.inputs, self.out):
+        for fi, f in enumerate(self.formats):
+            for j, ((x, w, dy), (y, dx, dw)) in enumerate(zip(inputs, self.out)):
+                if before is not None and fi == 0:
+                    before(j)
                 M, K = x.shape
                 N = w.shape[0]
                 lib, p, st = api._lib, api._p, api._stream()
@@ -601,25 +610,44 @@ def main():
         h2d = sum(t.numel() * 2 for trip in host for t in trip)
         stats_dev = step.stats6 if step.dual else step.stats
         stats_host = torch.empty_like(stats_dev, device="cpu").pin_memory()
-        def e2e_step():
-            for trip_d, trip_h in zip(step.inputs, host):
-                for d, h in zip(trip_d, trip_h):
-                    d.copy_(h, non_blocking=True)
-            step.run_linear_calls()
+        # Two device copies of the inputs: while one step computes from one set, the copy engine fills the other
+        # from pinned host memory on its own stream.  Every linear waits only for its own three tensors, and a set
+        # is overwritten only after the last kernel that reads it has finished.
+        sets = [step.inputs, [tuple(torch.empty_like(t) for t in trip) for trip in step.inputs]]
+        copy_stream = torch.cuda.Stream(device=device)
+        main_stream = torch.cuda.current_stream(device)
+        set_free = [None, None]
+        def e2e_step(k):
+            dev_in = sets[k % 2]
+            ready = []
+            with torch.cuda.stream(copy_stream):
+                if set_free[k % 2] is not None:
+                    copy_stream.wait_event(set_free[k % 2])
+                for trip_d, trip_h in zip(dev_in, host):
+                    for d, h in zip(trip_d, trip_h):
+                        d.copy_(h, non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(copy_stream)
+                    ready.append(ev)
+            step.run_linear_calls(inputs=dev_in, before=lambda i: main_stream.wait_event(ready[i]))
             stats_host.copy_(stats_dev, non_blocking=True)
-        e2e_step(); barrier()
-        n_e2e = max(1, min(args.steps, 3))
+            set_free[k % 2] = torch.cuda.Event()
+            set_free[k % 2].record(main_stream)
+        e2e_step(0); e2e_step(1); barrier()
+        n_e2e = max(2, min(args.steps, 10))
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s0.record()
-        for _ in range(n_e2e):
-            e2e_step()
+        copy_stream.wait_event(s0)   # no copy of a timed step starts before the clock does
+        for k in range(n_e2e):
+            e2e_step(k)
         s1.record()
         barrier()
         ms_e2e = s0.elapsed_time(s1) / n_e2e
         ms_e2e, flops_e2e = combine_replicas(ms_e2e, step.flops, dist if world > 1 else None, device)
         e2e = {"value": flops_e2e / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": stats_host.numel()}
-        del host
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": stats_host.numel(), "steps": n_e2e,
+               "overlap": "copies on a second stream into alternating input sets"}
+        del host, sets
 
     if rank != 0:
         if world > 1:
