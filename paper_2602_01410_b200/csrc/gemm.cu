@@ -197,7 +197,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
 
     if (warp < 4) {
-      reg_dealloc<48>();  // frees (168-48)*128 = 15360 registers
+      reg_dealloc<40>();  // frees (168-40)*128 = 16384 registers
       if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
@@ -274,7 +274,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
     } else {
-        reg_alloc<224>();    // needs (224-168)*256 = 14336 <= 15360 (an unsatisfiable request would block forever)
+        reg_alloc<232>();    // needs (232-168)*256 = 16384 <= 16384 (an unsatisfiable request would block forever)
         // ================= promotion / epilogue warps =================
         const int e = warp - 4;          // 0..7
         const int q = warp & 3;          // tensor-memory lane quarter this warp may access
@@ -289,7 +289,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const uint32_t stage_u32 = out_stage0 + e * 2048;   // this warp's staging tile: 32 rows x 64 bytes
         uint32_t cc = 0;
         bool ok = true;
-        bool ready = false;   // the next chunk's partial sums were already seen complete by an early test
         for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
             int m_idx, n_idx;
             tile_coords(t, num_m, num_n, m_idx, n_idx);
@@ -351,25 +350,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
                 }
             }
-            // Reciprocal scale factors of chunk cn from its ring slot (the slot must have landed).  Block mode:
-            // one factor per 32-column group; vector mode: 1/S_a in fo[0], and the slot's column scales are
-            // turned into reciprocals in place (4 per lane).
-            auto prepare_factors = [&](int cn, float (&fo)[G]) {
-                if (SCALE == SCALE_BLOCK_B) {
-                    const float *sl = ring + ((cn >> 2) & 1) * C::kGroupFloats;
-                    const float sa = sl[(cn & 3) * 32 + lane];
-                    const float f0 = rcp_approx(sa * sl[128 + (cn & 3)]);
-                    if (kBlocksPerWarp == 1) {
+            // Block mode: the reciprocal factors 1/(S_a*S_b) of the four chunks of group gn, from its slot (which must
+            // have landed and been made visible to the warp), into a register queue that the chunk loop shifts.
+            float fq[kBlocksPerWarp][4];
+            auto load_factors = [&](int gn) {
+                const float *sl = ring + (gn & 1) * C::kGroupFloats;
+                const float4 b0 = *reinterpret_cast<const float4 *>(sl + 128);
+                const float sb0[4] = {b0.x, b0.y, b0.z, b0.w};
 #pragma unroll
-                        for (int gi = 0; gi < G; ++gi) fo[gi] = f0;
-                    } else {
-                        const float f1 = rcp_approx(sa * sl[132 + (cn & 3)]);
-#pragma unroll
-                        for (int gi = 0; gi < G; ++gi) fo[gi] = (((col0 + 32 * gi) >> 7) == blk0) ? f0 : f1;
-                    }
-                } else {
-                    fo[0] = rcp_approx(ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane]);
+                for (int j = 0; j < 4; ++j) {
+                    const float sa = sl[j * 32 + lane];
+                    fq[0][j] = rcp_approx(sa * sb0[j]);
+                    if (kBlocksPerWarp == 2) fq[1][j] = rcp_approx(sa * sl[132 + j]);
                 }
+            };
+            // Vector mode: 1/S_a of chunk cn from its group slot (the group landed with an earlier chunk).
+            auto prepare_factors = [&](int cn, float (&fo)[G]) {
+                fo[0] = rcp_approx(ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane]);
             };
             // Vector mode: turns chunk cn's column scales into reciprocals in place (4 per lane).  Done two chunks
             // ahead of their use, at the end of an iteration, so that the load - reciprocal - store chain never
@@ -386,8 +383,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (SCALE == SCALE_BLOCK_B) {
                 cp_async_wait<1>();   // group 0
                 __syncwarp();
-                prepare_factors(0, f_next);
-                __syncwarp();
+                load_factors(0);
             } else if (SCALE == SCALE_VEC_B) {
                 cp_async_wait<C::kScaleDepth - 2>();   // chunks 0 and 1
                 __syncwarp();
@@ -400,51 +396,47 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 float f[G];
                 const float *slot = ring + C::kRingB + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;   // vector mode: this chunk's column reciprocals
 #pragma unroll
-                for (int gi = 0; gi < G; ++gi) f[gi] = f_next[gi];
-                // barrier that announces this chunk's partial sums (see the MMA issuer) and the one of the next chunk
+                for (int gi = 0; gi < G; ++gi) {
+                    if (SCALE == SCALE_BLOCK_B) f[gi] = (kBlocksPerWarp == 1 || ((col0 + 32 * gi) >> 7) == blk0) ? fq[0][0] : fq[kBlocksPerWarp - 1][0];
+                    else f[gi] = f_next[gi];
+                }
+                if (SCALE == SCALE_BLOCK_B) {
+#pragma unroll
+                    for (int b = 0; b < kBlocksPerWarp; ++b) { fq[b][0] = fq[b][1]; fq[b][1] = fq[b][2]; fq[b][2] = fq[b][3]; }
+                }
+                // barrier that announces this chunk's partial sums (see the MMA issuer)
                 const uint32_t done_bar = (KIND == MmaKind::F8F6F4) ? empty_bar(cc % S) : tfull_bar(a);
                 const uint32_t done_par = (KIND == MmaKind::F8F6F4) ? ((cc / S) & 1u) : ((cc >> 1) & 1u);
-                const uint32_t next_bar = (KIND == MmaKind::F8F6F4) ? empty_bar((cc + 1) % S) : tfull_bar(a ^ 1u);
-                const uint32_t next_par = (KIND == MmaKind::F8F6F4) ? (((cc + 1) / S) & 1u) : (((cc + 1) >> 1) & 1u);
-                if (!ready) {
+                {
                     const bool got = mbar_wait(done_bar, done_par, abort_flag);
                     if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
                 }
                 tc_fence_after_sync();
-                uint32_t early = 0;
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
                 // two 32-column groups in registers next to the accumulators: one in flight, one being consumed
                 uint32_t v[2][32];
                 tmem_ld32(taddr, v[0]);
                 if (SCALE != SCALE_NONE) {
-                    // In the shadow of the first load: next chunk's factors, so that no shared-memory or
-                    // special-function latency opens the next iteration.  Block mode has consumed this chunk's
-                    // slot into registers already and refills it now; vector mode still reads its column
-                    // reciprocals from the slot below and refills it at the end of the iteration.
+                    // In the shadow of the first load.  Block mode: with the last chunk of a group of four the register
+                    // queue is empty; the next group's slot (requested four chunks ago) is turned into the next four
+                    // factors and the slot of the group just finished is refilled two groups ahead.  One warp barrier
+                    // per four chunks: between the copies of all lanes and the reads of all lanes.
                     if (SCALE == SCALE_BLOCK_B) {
-                        // chunk c is the last of its group: every lane took its factors in the previous iteration,
-                        // so the group's slot is refilled (two groups ahead) and the next group must have landed
                         if ((c & 3) == 3) {
+                            cp_async_wait<0>();
+                            __syncwarp();
+                            load_factors((c >> 2) + 1);
                             prefetch_group((c >> 2) + 2);
-                            cp_async_wait<1>();
                         }
-                        __syncwarp();
-                        prepare_factors(c + 1, f_next);
-                        __syncwarp();   // every lane has read its factors before a later refill may overwrite the slot
                     } else {
-                        prepare_factors(c + 1, f_next);   // 1/S_a only; its group landed with an earlier chunk
+                        prepare_factors(c + 1, f_next);   // vector mode: 1/S_a only
                     }
                 }
                 // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
                 auto release_buffer = [&]() {
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(tempty_bar(a));
-                        // non-blocking look at the next chunk's barrier: its shared-memory latency hides
-                        // behind the FMAs below instead of opening the next iteration
-                        early = mbar_test_wait(next_bar, next_par) ? 1u : 0u;
-                    }
+                    if (lane == 0) mbar_arrive(tempty_bar(a));
                 };
                 auto consume_group = [&](int gi, const uint32_t (&cur)[32]) {
                     if (SCALE == SCALE_NONE) {
@@ -479,7 +471,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     else release_buffer();
                     consume_group(gi, v[gi & 1]);
                 }
-                ready = __shfl_sync(0xFFFFFFFFu, early, 0) != 0;
                 if (SCALE == SCALE_VEC_B) {
                     cp_async_wait<1>();                  // chunk c+2 has landed (c+3 may be in flight)
                     __syncwarp();                        // ... for every lane, and every lane has read slot c
