@@ -141,8 +141,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 {
     using C = Cfg<KIND, BN, SCALE>;
     constexpr int S = C::kStages;
-    constexpr int G = BN / 64;       // 32-column groups handled by one epilogue warp
     constexpr int HALF = BN / 2;     // columns handled by one epilogue warp
+    constexpr int GC = 32;           // columns per tensor-memory load
+    constexpr int G = HALF / GC;     // groups handled by one epilogue warp per chunk
 
     extern __shared__ uint8_t smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle
@@ -413,9 +414,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * BN + h * HALF;
-                // two 32-column groups in registers next to the accumulators: one in flight, one being consumed
-                uint32_t v[2][32];
-                tmem_ld32(taddr, v[0]);
+                // two 32-column groups in registers next to the accumulators
+                uint32_t v[2][GC];
+                tmem_ld_cols(taddr, v[0]);
+                if (G > 1) tmem_ld_cols(taddr + GC, v[1]);
                 if (SCALE != SCALE_NONE) {
                     // In the shadow of the first load.  Block mode: with the last chunk of a group of four the register
                     // queue is empty; the next group's slot (requested four chunks ago) is turned into the next four
@@ -438,7 +440,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(a));
                 };
-                auto consume_group = [&](int gi, const uint32_t (&cur)[32]) {
+                auto consume_group = [&](int gi, const uint32_t (&cur)[GC]) {
                     if (SCALE == SCALE_NONE) {
                         float o[32];
 #pragma unroll
@@ -447,29 +449,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     } else if (SCALE == SCALE_BLOCK_B) {
                         const float2 ff = make_float2(f[gi], f[gi]);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            acc[16 * gi + i] = __ffma2_rn(make_float2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), ff, acc[16 * gi + i]);
+                        for (int i = 0; i < GC / 2; ++i)
+                            acc[(GC / 2) * gi + i] = __ffma2_rn(make_float2(__uint_as_float(cur[2 * i]), __uint_as_float(cur[2 * i + 1])), ff, acc[(GC / 2) * gi + i]);
                     } else {
                         const float2 ff = make_float2(f[0], f[0]);
-                        const float4 *sbv = reinterpret_cast<const float4 *>(slot + 32 * gi);
+                        const float4 *sbv = reinterpret_cast<const float4 *>(slot + GC * gi);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
+                        for (int i = 0; i < GC / 4; ++i) {
                             const float4 s4 = sbv[i];   // reciprocal column scales, broadcast read
                             const float2 r0 = make_float2(s4.x, s4.y);
                             const float2 r1 = make_float2(s4.z, s4.w);
                             const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i]), __uint_as_float(cur[4 * i + 1])), r0);
                             const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(cur[4 * i + 2]), __uint_as_float(cur[4 * i + 3])), r1);
-                            acc[16 * gi + 2 * i] = __ffma2_rn(p0, ff, acc[16 * gi + 2 * i]);
-                            acc[16 * gi + 2 * i + 1] = __ffma2_rn(p1, ff, acc[16 * gi + 2 * i + 1]);
+                            acc[(GC / 2) * gi + 2 * i] = __ffma2_rn(p0, ff, acc[(GC / 2) * gi + 2 * i]);
+                            acc[(GC / 2) * gi + 2 * i + 1] = __ffma2_rn(p1, ff, acc[(GC / 2) * gi + 2 * i + 1]);
                         }
                     }
                 };
+                // Two loads are in flight from the start; each group's FMAs free its registers for the load two groups
+                // on.  The buffer goes back to the MMA warp as soon as the last load has landed, so that the stretch in
+                // which that warp may be waiting holds the FMAs of only G-2 groups; the last two groups follow the release.
+                tmem_ld_wait();
+                if (G <= 2) release_buffer();
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) {
-                    tmem_ld_wait();
-                    if (gi + 1 < G) tmem_ld32(taddr + 32 * (gi + 1), v[(gi + 1) & 1]);   // in flight during the FMAs below
-                    else release_buffer();
                     consume_group(gi, v[gi & 1]);
+                    if (gi + 2 < G) {
+                        tmem_ld_cols(taddr + GC * (gi + 2), v[gi & 1]);
+                        if (gi + 3 >= G) {   // that was the chunk's last load
+                            tmem_ld_wait();
+                            release_buffer();
+                        }
+                    }
                 }
                 if (SCALE == SCALE_VEC_B) {
                     cp_async_wait<1>();                  // chunk c+2 has landed (c+3 may be in flight)
@@ -506,7 +517,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         }
                     } else if (row_ok) {
 #pragma unroll
-                        for (int gi = 0; gi < G; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, reinterpret_cast<const float *>(acc) + 32 * gi);
+                        for (int gi = 0; gi < HALF / 32; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, reinterpret_cast<const float *>(acc) + 32 * gi);
                     }
                 }
                 __syncwarp();
