@@ -39,7 +39,7 @@ NOMINAL_RATIO = {0: 1.0, 1: 2.0, 2: 4.0}   # dense tensor peak relative to bf16
 # DRAM bytes (read + write) of one GEMM launch on the fused-QKV forward shape 16384 x 12288 x 4096, from the
 # ncu captures summarised in profiles/gemm_kernel_gemm_<fmt>_fwd_16384x12288x4096.md (algorithmic: 519 MB FP8,
 # 461 MB FP4).  Reported as `traffic` of the roofline object together with the shape it belongs to.
-NCU_TRAFFIC = {1: 824.7e6, 2: 498.3e6}
+NCU_TRAFFIC = {1: 823.5e6, 2: 493.9e6}
 
 
 def load_peaks():
