@@ -583,6 +583,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
     extern __shared__ __align__(128) uint8_t smem[];
     QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
     const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
+    // this grid may have been scheduled before the kernel ahead of it on the stream has finished (see
+    // launch_persistent): nothing is read or written before that kernel is complete
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // the statistics reduction that follows on the stream may be scheduled now; it waits for this
     // grid to finish before it reads anything (programmatic dependent launch)
     if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -615,6 +618,7 @@ __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel
     extern __shared__ __align__(128) uint8_t smem[];
     QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
     const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     ThreadStats ts;
     TileWalk w((int)d.a.tiles_r, (int)d.a.tiles_c);
@@ -649,6 +653,9 @@ __global__ void __launch_bounds__(1024) stats_reduce_kernel(const ReduceSets set
     __shared__ float sh_m[32];
     const CtaPartial *partials = sets.partials[blockIdx.x];
     snip_stats_t *out = sets.out[blockIdx.x];
+    // a quantizer launched behind this reduction may take the SMs the previous quantizer is leaving; it waits
+    // for this grid before it reads or writes anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     double dx = 0.0, de = 0.0;
     float am = 0.0f;
@@ -699,7 +706,20 @@ template <typename Kernel, typename Args>
 void launch_persistent(Kernel kernel, const Args &args, dim3 grid, cudaStream_t st)
 {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) return;  // left in cudaGetLastError
-    kernel<<<grid, kThreads, kSmemBytes, st>>>(args);
+    // Programmatic stream serialization: when the kernel before it on the stream signals its dependents early (the
+    // statistics reduction of the previous call does), this grid's CTAs may take their places while that kernel
+    // drains; they block in griddepcontrol.wait until it has completed, before they touch global memory.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, args);   // an error stays in cudaGetLastError for the caller
 }
 
 template <int FMT, int BLOCK, bool TRANSPOSED>
