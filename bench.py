@@ -715,12 +715,15 @@ def main():
         orc.set_num_threads(cores)
         cpu["one_core"] = {"value": v1, "unit": "TFLOP/s", "cores": 1, "sample": sample1}
 
+    input_bytes = sum(2 * (cfg.M * L.K + L.N * L.K + cfg.M * L.N) for L in cfg.linears)   # bf16 X, W, dY of every linear
     line = {"metric": "mixed-precision linear fwd+dgrad+wgrad TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4_e2m1+fp8_e4m3 (fp32 accumulate)", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: one block (qkv,o,gate,up,down) x (fwd,dgrad,wgrad) all-FP4 then all-FP8, tokens {cfg.M}, quantize+stats of both operands of every GEMM "
+            "config": {"workload": f"{cfg.name}: one block ({','.join(L.name for L in cfg.linears)}) x (fwd,dgrad,wgrad) all-FP4 then all-FP8, tokens {cfg.M}, quantize+stats of both operands of every GEMM "
                                    + ("(X, W, dY read once each, two quantized copies per read)" if step.dual else "(one quantizer call per operand)"),
-                       "l2": "inputs larger than L2", "parallelism": "replicas only" if world > 1 else "single GPU"},
+                       "l2": (f"inputs ({input_bytes / 1e6:.0f} MB) larger than L2" if input_bytes > 126e6
+                              else f"inputs ({input_bytes / 1e6:.1f} MB) fit in L2: a test workload, not a measurement"),
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": step.launches_per_step * args.steps,
             "roofline": roofline, "kernels": kernels, "pow2_option": pow2_option, "cpu_baseline": cpu}
     print(json.dumps(line))
