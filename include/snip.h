@@ -5,8 +5,9 @@
  * cores with FP32 accumulation.
  *
  * Conventions
- *   - Every function returns a snip_status_t (0 = SNIP_OK).  Nothing throws, nothing allocates,
- *     nothing synchronizes the host: all device work is enqueued on the caller's stream.
+ *   - Every function returns a snip_status_t (0 = SNIP_OK).  Nothing throws, nothing allocates
+ *     device memory, nothing synchronizes the host: all device work is enqueued on the caller's
+ *     stream.  (The host-only solver snip_select_scheme uses ordinary host heap memory.)
  *   - The caller owns every buffer.  Pointers are DEVICE pointers unless the name ends in
  *     `_host`.  Device pointers must be 16-byte aligned.  Outputs are fully overwritten.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
@@ -269,7 +270,8 @@ int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int 
  * only).  Operand formats: (BF16,BF16), (FP8,FP8), (FP4,FP4), (FP8,FP4), (FP4,FP8); pairs
  * that mix BF16 with a quantized operand return SNIP_ERR_UNSUPPORTED.
  * ws must hold at least gemm_bytes of snip_workspace_size; its first word is the device status
- * word read by snip_poll_status.
+ * word read by snip_poll_status.  The call itself zeroes that word on the stream before the
+ * kernel starts (a 4-byte memset node), so the workspace needs no initialisation by the caller.
  */
 int snip_gemm_quantized(int op, const snip_qtensor_t *a_host, const snip_qtensor_t *b_host,
                         void *out, int out_dtype, int accumulate, void *ws, size_t ws_bytes,
@@ -412,9 +414,28 @@ int snip_select_scheme(int m, int n, const double *q, const int64_t *w, int64_t 
 /* ---- device status ------------------------------------------------------------------------ */
 
 /*
+ * Testing hooks, process-wide and off by default.  (No counterpart in the paper.)
+ *   SNIP_DEBUG_WAIT_LIMIT_NS : bound of every device-side wait of the GEMM kernels (default 2e9).
+ *   SNIP_DEBUG_TX_SKEW_BYTES : a multiple of 16 added to the byte count a pipeline stage's barrier
+ *                              expects.  Non-zero makes the first stage of every GEMM incomplete for
+ *                              ever while every copy still lands: the kernel's waits run out, it
+ *                              leaves on its own and snip_poll_status reports SNIP_ERR_TIMEOUT.
+ *                              Nothing traps or faults; used with a short wait limit by the tests.
+ *   SNIP_DEBUG_GEMM_KERNEL   : 0 = automatic choice, 1 = single-CTA kernels only, 2 = CTA-pair
+ *                              kernels for every quantized GEMM (A/B comparisons in the benchmark).
+ * Returns SNIP_ERR_ARG for an unknown key or a value out of range.
+ */
+#define SNIP_DEBUG_WAIT_LIMIT_NS 0
+#define SNIP_DEBUG_TX_SKEW_BYTES 1
+#define SNIP_DEBUG_GEMM_KERNEL   2
+int snip_debug_set(int key, long long value);
+
+/*
  * Read the device status word of a GEMM workspace.  Call after the stream has been
  * synchronized.  *status_host becomes SNIP_OK or SNIP_ERR_TIMEOUT (a bounded device-side wait
- * expired and the kernel returned early; outputs are then invalid).  Performs a small
+ * expired and the kernel returned early; outputs are then invalid).  Every GEMM entry point
+ * zeroes the word before its kernels run (snip_linear_fwd_bwd once, before its three GEMMs), so
+ * the value always belongs to the last call made with that workspace.  Performs a small
  * device-to-host copy.  (No counterpart in the paper.)
  */
 int snip_poll_status(const void *ws, int *status_host);

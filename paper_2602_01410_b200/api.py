@@ -26,7 +26,7 @@ EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
     "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace", "snip_adamw_sensitivity_workspace", "snip_adamw_sensitivity", "snip_loss_divergence", "snip_weight_divergence", "snip_select_scheme",
-    "snip_poll_status",
+    "snip_poll_status", "snip_debug_set",
 )
 
 
@@ -51,6 +51,8 @@ class QOut(ctypes.Structure):
 
 DUAL_ROW_COLT, DUAL_BLK_BLKT = 0, 1
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
+DEBUG_WAIT_LIMIT_NS, DEBUG_TX_SKEW_BYTES, DEBUG_GEMM_KERNEL = 0, 1, 2
+GEMM_KERNEL_AUTO, GEMM_KERNEL_SINGLE, GEMM_KERNEL_PAIR = 0, 1, 2
 
 
 class LayerTensors(ctypes.Structure):
@@ -98,6 +100,7 @@ def _load():
     lib.snip_weight_divergence.argtypes = [dbl, dbl, i64, i64, dbl, dbl, dbl, i64, dbl, i64]
     lib.snip_select_scheme.argtypes = [i32, i32, vp, vp, i64, i32, vp, vp, vp]
     lib.snip_poll_status.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.snip_debug_set.argtypes = [i32, ctypes.c_longlong]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int and name not in ("snip_version",):
@@ -441,6 +444,11 @@ def snip_select_scheme(q, w, target: int, num_groups: int = 1):
     _check("snip_select_scheme", _lib.snip_select_scheme(m, n, qa.ctypes.data_as(ctypes.c_void_p), wa.ctypes.data_as(ctypes.c_void_p), int(target),
                                                          num_groups, choice.ctypes.data_as(ctypes.c_void_p), ctypes.byref(qt), ctypes.byref(wt)))
     return [int(c) for c in choice], qt.value, wt.value
+
+
+def snip_debug_set(key: int, value: int) -> None:
+    """Testing hooks of the library (process-wide, off by default): see include/snip.h."""
+    _check("snip_debug_set", _lib.snip_debug_set(key, value))
 
 
 def snip_poll_status(ws: torch.Tensor) -> int:

@@ -16,6 +16,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -43,6 +45,7 @@ struct GemmArgs {
     int64_t ldo;
     int32_t accumulate;
     uint32_t stage_tx_bytes;   // bytes the two TMA loads of one stage report to the barrier
+    uint64_t wait_limit_ns;    // bound of every device-side wait
     uint32_t *status;
 };
 
@@ -210,7 +213,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int ks = 0; ks < num_kstages; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
                     mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
                     tma_load_2d(smem_a0 + s * C::kABytes, &tmA, full_bar(s), ks * C::kStageElemsX, m_idx * BM);
                     tma_load_2d(smem_b0 + s * C::kBBytes, &tmB, full_bar(s), ks * C::kStageElemsX, n_idx * BN);
@@ -227,14 +230,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int ks = 0; ks < num_kstages && ok; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, g.wait_limit_ns)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint64_t adesc = make_smem_desc_k128(smem_a0 + s * C::kABytes);
                     const uint64_t bdesc = make_smem_desc_k128(smem_b0 + s * C::kBBytes);
                     if (KIND == MmaKind::F16) {
                         const uint32_t a = cc & 1u;
                         if (ks == 0) {
-                            if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                            if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
                             tc_fence_after_sync();
                         }
 #pragma unroll
@@ -244,7 +247,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         if (ks == num_kstages - 1) { tc_commit<false>(tfull_bar(a)); ++cc; }
                     } else if (KIND == MmaKind::F8F6F4) {
                         const uint32_t a = cc & 1u;
-                        if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
                         tc_fence_after_sync();
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
@@ -258,7 +261,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         for (int h = 0; h < 2; ++h) {
                             if (2 * ks + h < num_chunks) {
                                 const uint32_t a = cc & 1u;
-                                if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                                if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
                                 tc_fence_after_sync();
 #pragma unroll
                                 for (int k = 0; k < 2; ++k)
@@ -409,7 +412,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const uint32_t done_bar = (KIND == MmaKind::F8F6F4) ? empty_bar(cc % S) : tfull_bar(a);
                 const uint32_t done_par = (KIND == MmaKind::F8F6F4) ? ((cc / S) & 1u) : ((cc >> 1) & 1u);
                 {
-                    const bool got = mbar_wait(done_bar, done_par, abort_flag);
+                    const bool got = mbar_wait(done_bar, done_par, abort_flag, g.wait_limit_ns);
                     if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
                 }
                 tc_fence_after_sync();
@@ -643,6 +646,24 @@ int launch_gemm_scale(int scale, bool out_f32, const CUtensorMap &tmA, const CUt
 
 size_t gemm_ws_bytes() { return 256; }
 
+// Testing hooks (snip_debug_set): process-wide, off by default.
+namespace {
+std::atomic<long long> g_wait_limit_ns{2000000000ll};   // bound of every device-side wait of the GEMM kernels
+std::atomic<int> g_tx_skew{0};                           // bytes added to what a stage's barrier expects (a wait that cannot complete)
+std::atomic<int> g_kernel_choice{0};                     // 0 = automatic, 1 = single-CTA kernels only, 2 = CTA-pair kernels where they apply
+}  // namespace
+
+int gemm_pair_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
+                   int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
+                   int out_dtype, int accumulate, uint32_t *status, uint64_t wait_limit_ns, int tx_skew, cudaStream_t st);
+
+// Zeroes the status word of a GEMM workspace (enqueued; allocates nothing).
+int gemm_clear_status(void *ws, cudaStream_t st)
+{
+    SNIP_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(uint32_t), st));
+    return SNIP_OK;
+}
+
 // Shared with the power-of-two-scale GEMMs: 2-D tiled tensor map over a row-major matrix.
 int make_tiled_map_2d(CUtensorMap *map, const void *ptr, int dtype, int64_t rows, int64_t inner_elems, int64_t row_bytes, int box_x_elems,
                       int box_rows, int swizzle)
@@ -664,7 +685,7 @@ int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaSt
 // scale_mode: SCALE_NONE for BF16, SCALE_BLOCK_B (fwd / dgrad), SCALE_VEC_B (wgrad).
 int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
               int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
-              int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st)
+              int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status)
 {
     if (!a_codes || !b_codes || !out) return SNIP_ERR_ARG;
     if (!valid_dim(Mo) || !valid_dim(No) || !valid_dim(Kc) || Mo > INT32_MAX || No > INT32_MAX || Kc > INT32_MAX) return SNIP_ERR_SHAPE;
@@ -678,6 +699,9 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     if (!a16 && (!aligned16(sa) || !aligned16(sb))) return SNIP_ERR_ALIGN;   // scale factors are fetched 16 bytes at a time
     int rc = require_sm100();
     if (rc != SNIP_OK) return rc;
+    // The status word starts at zero for this call unless the caller runs several GEMMs against one word
+    // and has cleared it itself (an earlier GEMM's timeout must survive the later ones).
+    if (clear_status) { rc = gemm_clear_status(ws, st); if (rc) return rc; }
 
     GemmArgs g;
     g.Mo = (int32_t)Mo; g.No = (int32_t)No; g.Kc = (int32_t)Kc;
@@ -686,7 +710,16 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     g.out = out; g.ldo = No; g.accumulate = accumulate;
     g.status = static_cast<uint32_t *>(ws);
     g.stage_tx_bytes = 0;
+    g.wait_limit_ns = (uint64_t)g_wait_limit_ns.load();
+    const int tx_skew = g_tx_skew.load();
     const bool f32 = out_dtype == SNIP_OUT_FP32;
+
+    // Quantized operands: the CTA-pair kernels (256 x 128 tiles) wherever an output has at least one full tile
+    // of rows; shorter outputs stay on the single-CTA kernels below (a pair would idle one of its two SMs).
+    const int choice = g_kernel_choice.load();
+    if (!a16 && choice != 1 && (Mo >= 256 || choice == 2))
+        return gemm_pair_impl(fmt_a, fmt_b, a_codes, b_codes, Mo, No, Kc, sa, sa_chunk_stride, sb, sb_chunk_stride, sb_blk_stride, scale_mode,
+                              out, out_dtype, accumulate, g.status, g.wait_limit_ns, tx_skew, st);
 
     CUtensorMap tmA, tmB, tmO;
     // output boxes of 32 rows x 64 bytes for the TMA stores of the block-mode epilogue
@@ -699,7 +732,7 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
         rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, No, Kc, Kc * 2, 64, 256);
         if (rc) return rc;
         const uint32_t idesc = make_idesc(1, 1, BM, 256);
-        g.stage_tx_bytes = (BM + 256) * 128;
+        g.stage_tx_bytes = (BM + 256) * 128 + tx_skew;
         return f32 ? launch_gemm<MmaKind::F16, 256, SCALE_NONE, true>(tmA, tmB, tmO, g, idesc, st)
                    : launch_gemm<MmaKind::F16, 256, SCALE_NONE, false>(tmA, tmB, tmO, g, idesc, st);
     }
@@ -716,7 +749,7 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
         rc = make_operand_map(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN);
         if (rc) return rc;
         const uint32_t idesc = make_idesc_block_scaled(1, 1, BM, BN);
-        g.stage_tx_bytes = (BM + BN) * 128;
+        g.stage_tx_bytes = (BM + BN) * 128 + tx_skew;
         return launch_gemm_scale<MmaKind::MXF4, BN>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
     }
     // FP8 x FP8, the mixed pairs and FP4 x FP4 over whole chunks: kind::f8f6f4; FP4 operands are expanded by
@@ -739,7 +772,7 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     const uint32_t idesc = make_idesc(a4 ? 5 : 0, b4 ? 5 : 0, BM, BN);
     // an FP4 operand expanded by the TMA unit occupies 128 B per row in shared memory but reports
     // only its 64 packed source bytes to the barrier
-    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128);
+    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128) + tx_skew;
     return launch_gemm_scale<MmaKind::F8F6F4, BN>(scale_mode, f32, tmA, tmB, tmO, g, idesc, st);
 }
 
@@ -777,7 +810,18 @@ extern "C" int snip_gemm_quantized(int op, const snip_qtensor_t *a, const snip_q
     }
     if (!q) mode = SCALE_NONE;
     return gemm_impl(a->fmt, b->fmt, a->codes, b->codes, Mo, No, Kc, sa, sa_cs, sb, sb_cs, sb_bs, mode, out, out_dtype, accumulate,
-                     ws, ws_bytes, static_cast<cudaStream_t>(stream));
+                     ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
+}
+
+extern "C" int snip_debug_set(int key, long long value)
+{
+    using namespace snip;
+    switch (key) {
+        case SNIP_DEBUG_WAIT_LIMIT_NS: if (value <= 0) return SNIP_ERR_ARG; g_wait_limit_ns.store(value); return SNIP_OK;
+        case SNIP_DEBUG_TX_SKEW_BYTES: if (value < 0 || value > 4096 || (value % 16) != 0) return SNIP_ERR_ARG; g_tx_skew.store((int)value); return SNIP_OK;
+        case SNIP_DEBUG_GEMM_KERNEL: if (value < 0 || value > 2) return SNIP_ERR_ARG; g_kernel_choice.store((int)value); return SNIP_OK;
+        default: return SNIP_ERR_ARG;
+    }
 }
 
 extern "C" int snip_poll_status(const void *ws, int *status_host)

@@ -268,11 +268,12 @@ int launch_mx(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap 
 
 int make_tiled_map_2d(CUtensorMap *map, const void *ptr, int dtype, int64_t rows, int64_t inner_elems, int64_t row_bytes, int box_x_elems,
                       int box_rows, int swizzle);
+int gemm_clear_status(void *ws, cudaStream_t st);
 int gemm_sm_count();
 
 // a_codes [Mo][Kc], b_codes [No][Kc] contraction-major; sfa / sfb: UE8M0 atoms [line tile][chunk][512].
 int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, const void *sfa, const void *sfb, int64_t Mo, int64_t No,
-                 int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st)
+                 int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status)
 {
     if (!a_codes || !b_codes || !sfa || !sfb || !out) return SNIP_ERR_ARG;
     if (!valid_dim(Mo) || !valid_dim(No) || !valid_dim(Kc) || Mo > INT32_MAX || No > INT32_MAX || Kc > INT32_MAX) return SNIP_ERR_SHAPE;
@@ -282,6 +283,7 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
     if (!aligned16(a_codes) || !aligned16(b_codes) || !aligned16(sfa) || !aligned16(sfb) || !aligned16(out) || !aligned16(ws)) return SNIP_ERR_ALIGN;
     int rc = require_sm100();
     if (rc != SNIP_OK) return rc;
+    if (clear_status) { rc = gemm_clear_status(ws, st); if (rc) return rc; }   // see gemm_impl
     const bool f32 = out_dtype == SNIP_OUT_FP32;
     const bool a4 = fmt_a == SNIP_FMT_FP4_E2M1, b4 = fmt_b == SNIP_FMT_FP4_E2M1;
 
@@ -342,5 +344,5 @@ extern "C" int snip_gemm_mx(int op, const snip_qtensor_t *a, const void *sf_a, c
         if (a->block != SNIP_BLOCK_COL_128x1 || b->block != SNIP_BLOCK_COL_128x1) return SNIP_ERR_UNSUPPORTED;
         Mo = a->cols; No = b->cols; Kc = a->rows;
     }
-    return gemm_mx_impl(a->fmt, b->fmt, a->codes, b->codes, sf_a, sf_b, Mo, No, Kc, out, out_dtype, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+    return gemm_mx_impl(a->fmt, b->fmt, a->codes, b->codes, sf_a, sf_b, Mo, No, Kc, out, out_dtype, ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
 }

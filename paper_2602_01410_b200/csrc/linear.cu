@@ -9,11 +9,12 @@ int quantize_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt
                   float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st);
 int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
               int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
-              int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st);
+              int out_dtype, int accumulate, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status);
+int gemm_clear_status(void *ws, cudaStream_t st);
 int quantize_impl_ex(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block, uint32_t flags, int pow2, void *sf,
                      void *codes, float *scales, snip_stats_t *stats, double *row_stats, void *ws, size_t ws_bytes, cudaStream_t st);
 int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, const void *sfa, const void *sfb, int64_t Mo, int64_t No,
-                 int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st);
+                 int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status);
 int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st);
 size_t gemm_ws_bytes();
 int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bool blk, int pow2, const DualOut &oa, const DualOut &ob,
@@ -127,7 +128,7 @@ int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int6
                               mx ? 1 : 0, sf_b, codes_b, scales_b, stats_b, nullptr, sws_b, sws_b_bytes, st);
         if (rc) return rc;
         ga = codes_a; gb = codes_b;
-        if (mx) return gemm_mx_impl(fmt_a, fmt_b, ga, gb, sf_a, sf_b, p.Mo, p.No, p.Kc, out, out_dtype, gws, gemm_ws_bytes(), st);
+        if (mx) return gemm_mx_impl(fmt_a, fmt_b, ga, gb, sf_a, sf_b, p.Mo, p.No, p.Kc, out, out_dtype, gws, gemm_ws_bytes(), st, true);
     } else {
         // BF16 tag: identity quantization; only operands whose contraction index is not contiguous are copied
         if (p.tr_a) { rc = transpose_bf16(A, codes_a, p.rows_a, p.cols_a, st); if (rc) return rc; ga = codes_a; }
@@ -140,7 +141,7 @@ int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int6
     else if (op == SNIP_OP_DGRAD) { sb_bs = 1; sb_cs = ceil_div(K, 128); }
     else { sb_bs = 0; sb_cs = p.No; }
     return gemm_impl(fmt_a, fmt_b, ga, gb, p.Mo, p.No, p.Kc, scales_a, sa_cs, scales_b, sb_cs, sb_bs, q ? p.scale_mode : SCALE_NONE, out,
-                     out_dtype, accumulate, gws, gemm_ws_bytes(), st);
+                     out_dtype, accumulate, gws, gemm_ws_bytes(), st, true);
 }
 
 
@@ -272,14 +273,17 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
     };
     auto gemm = [&](int op, int ia, int ib, void *out) -> int {
         const LinearPlan p = plan_for(op, M, N, K);
-        if (mx) return gemm_mx_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], f.sf[ia], f.sf[ib], p.Mo, p.No, p.Kc, out, out_dtype, f.gws, gemm_ws_bytes(), st);
+        if (mx) return gemm_mx_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], f.sf[ia], f.sf[ib], p.Mo, p.No, p.Kc, out, out_dtype, f.gws, gemm_ws_bytes(), st, false);
         int64_t sb_cs, sb_bs;
         if (op == SNIP_OP_FWD) { sb_bs = ceil_div(K, 128); sb_cs = 1; }
         else if (op == SNIP_OP_DGRAD) { sb_bs = 1; sb_cs = ceil_div(K, 128); }
         else { sb_bs = 0; sb_cs = p.No; }
         return gemm_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], p.Mo, p.No, p.Kc, f.scales[ia], p.Mo, f.scales[ib], sb_cs, sb_bs, p.scale_mode, out,
-                         out_dtype, 0, f.gws, gemm_ws_bytes(), st);
+                         out_dtype, 0, f.gws, gemm_ws_bytes(), st, false);
     };
+    // one status word serves the three GEMMs of this call: cleared once, so that a timeout of the first is not erased
+    rc = gemm_clear_status(f.gws, st);
+    if (rc) return rc;
     // forward: X and W are read once each and leave both of their quantized copies behind
     rc = quantize_dual_impl(X, M, K, K, false, mx, out_of(0), out_of(1), f.stats_ws, f.stats_ws_bytes, st);
     if (rc) return rc;
