@@ -15,9 +15,10 @@
 //   warp 0      : TMA producer  - this CTA's halves of the operand tiles into a shared-memory ring;
 //                                 byte counts are reported to the leader's barrier (no multicast)
 //   warp 1      : MMA issuer    - leader CTA only, one thread; owns the tensor-memory allocation
-//   warp 2 (,3) : scale loader  - reads the chunk's scale factors from global memory some chunks
-//                                 ahead, turns them into reciprocal factors and leaves them in a
-//                                 shared-memory ring (warp 3: the per-column factors of wgrad)
+//   warp 2 (,3) : scale loader  - brings the chunks' scale factors into a 32-deep shared-memory ring
+//                                 with cp.async, two dozen chunks ahead of their use, and turns them
+//                                 into reciprocal factors in place (warp 3: the per-column factors
+//                                 of wgrad)
 //   warps 4..19 : promotion     - 32 rows x 32 columns each
 // Every wait is bounded; on a timeout both CTAs leave cleanly and a status word is raised.
 #include <cuda.h>
@@ -35,13 +36,20 @@ int make_tiled_map_2d(CUtensorMap *map, const void *ptr, int dtype, int64_t rows
 
 namespace {
 
-constexpr int kThreads = 640;
-constexpr int kEpiWarps = 16;
+constexpr int kEpiWarps = 16;      // warps 0..15: promotion / epilogue (warp % 4 = tensor-memory lane quarter)
+constexpr int kProducerWarp = 16;
+constexpr int kLoaderWarp = 17;
+constexpr int kIssuerWarp0 = 18;   // warps 18 .. 18 + kIssuers - 1
+constexpr int kIssuers = 2;
+constexpr int kThreads = 32 * (kIssuerWarp0 + kIssuers);
 constexpr int CM = 128;       // rows of A / of the accumulator per CTA
 constexpr int TM = 2 * CM;    // rows of one tile (CTA pair)
 constexpr int TN = 128;       // columns of one tile = one 128-wide scale block of B
 constexpr int kBRows = TN / 2;  // rows of B held by one CTA
-constexpr int kSD = 16;       // depth of the scale-factor ring, in chunks
+constexpr int kSD = 32;       // depth of the scale-factor ring, in chunks
+constexpr int kSBlk = 8;      // chunks per hand-over of the ring (one full / one empty barrier per 8 slots)
+constexpr int kSBlocks = kSD / kSBlk;
+constexpr int kAhead = 16;    // chunks whose scale factors are on their way from global memory (cp.async groups in flight)
 constexpr int kSlotFloats = 256;   // per chunk: [0,128) row factors of this CTA, [128,256) column factors (wgrad)
 constexpr int kSfCols = 32;   // tensor-memory columns of constant scale factors (kind::mxf4)
 
@@ -66,21 +74,17 @@ template <MmaKind KIND>
 struct PCfg {
     static constexpr int kCPS = (KIND == MmaKind::MXF4) ? 2 : 1;       // 128-long chunks per shared-memory stage
     static constexpr int kNBuf = (KIND == MmaKind::MXF4) ? 3 : 4;      // accumulator buffers in tensor memory
-    static constexpr int kStages = (KIND == MmaKind::MXF4) ? 5 : 6;
+    static constexpr int kStages = 8;
     static constexpr int kABytes = CM * 128;
     static constexpr int kBBytes = kBRows * 128;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kRingBytes = kSD * kSlotFloats * 4;
-    static constexpr int kOutBytes = kEpiWarps * 2048;                 // per-warp staging tile: 32 rows x 64 bytes
-    static constexpr int kBarBytes = 512;
+    static constexpr int kOutBytes = 0;
+    static constexpr int kBarBytes = 1024;
     static constexpr int kSmemBytes = kStages * kStageBytes + kRingBytes + kOutBytes + kBarBytes + 1024;
     static constexpr int kSfCol0 = kNBuf * TN;
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     static_assert(kNBuf * TN + (KIND == MmaKind::MXF4 ? kSfCols : 0) <= 512, "tensor memory budget");
-    // A ring slot is rewritten once the stage of its new chunk is free again; by then the promotion warps have
-    // released the buffer of a chunk at most kStages*kCPS + kCPS + kNBuf older, i.e. finished reading its slot.
-    static_assert(kSD >= kStages * kCPS + kCPS + kNBuf, "scale ring too shallow for the implicit slot hand-back");
-    static_assert((2 * kStages + 2 * kNBuf + kSD) * 8 + 8 <= kBarBytes, "barrier area");
 };
 
 __device__ __forceinline__ void pair_tile_coords(int t, int num_m, int num_n, int &m_idx, int &n_idx)
@@ -116,6 +120,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 {
     using C = PCfg<KIND>;
     constexpr int S = C::kStages, NB = C::kNBuf, CPS = C::kCPS;
+    constexpr int ND = S * CPS;      // "chunk done" barriers: one per chunk position of the stage ring
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;   // operand tiles: 1024-byte aligned (128-byte swizzle)
@@ -127,33 +132,37 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t bar0 = out_stage0 + C::kOutBytes;
     uint8_t *bar_gen = smem_gen + S * C::kStageBytes + C::kRingBytes + C::kOutBytes;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };                      // leader: operand bytes of both CTAs have landed
-    auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };               // each CTA: the MMAs reading stage s are done
-    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * S + b); };           // each CTA: buffer b holds a chunk's partial sums
-    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * S + NB + b); };     // leader: all 32 promotion warps have drained buffer b
-    auto sfull_bar = [&](int d) { return bar0 + 8u * (2 * S + 2 * NB + d); };  // each CTA: ring slot d holds a chunk's factors
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * S + 2 * NB + kSD));
+    auto done_bar = [&](int p) { return bar0 + 8u * (S + p); };                // each CTA: the MMAs of the chunk at ring position p are complete
+    auto tempty_bar = [&](int b) { return bar0 + 8u * (S + ND + b); };         // leader: the promotion warps of both CTAs have drained buffer b
+    auto sfull_bar = [&](int k) { return bar0 + 8u * (S + ND + NB + k); };     // each CTA: the 8 slots of ring block k hold their chunks' factors
+    auto sempty_bar = [&](int k) { return bar0 + 8u * (S + ND + NB + kSBlocks + k); };   // each CTA: all 16 promotion warps are done with block k
+    static_assert((S + ND + NB + 2 * kSBlocks) * 8 + 8 <= C::kBarBytes, "barrier area");
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_gen + 8 * (S + ND + NB + 2 * kSBlocks));
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);   // warp-uniform by construction
+    const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();   // 0 = leader
     const int num_m = (g.Mo + TM - 1) / TM, num_n = (g.No + TN - 1) / TN;
     const int num_tiles = num_m * num_n;
     const int first_tile = (int)(blockIdx.x >> 1), tile_step = (int)(gridDim.x >> 1);
+    const int my_tiles = first_tile < num_tiles ? (num_tiles - first_tile + tile_step - 1) / tile_step : 0;
     const int nacc = (g.Kc + 127) / 128;                    // chunks per tile
     const int num_kstages = (nacc + CPS - 1) / CPS;
     const uint64_t limit = g.wait_limit_ns;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < NB; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 2 * kEpiWarps); }
-        for (int d = 0; d < kSD; ++d) mbar_init(sfull_bar(d), SCALE == PSCALE_VEC_B ? 2 : 1);
+        for (int s = 0; s < S; ++s) mbar_init(full_bar(s), 1);
+        for (int p = 0; p < ND; ++p) mbar_init(done_bar(p), 1);
+        for (int b = 0; b < NB; ++b) mbar_init(tempty_bar(b), 2);
+        for (int k = 0; k < kSBlocks; ++k) { mbar_init(sfull_bar(k), 1); mbar_init(sempty_bar(k), kEpiWarps); }
         *abort_flag = 0u;
         fence_barrier_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
         prefetch_tensormap(&tmO);
     }
-    if (warp == 1) {
+    if (warp == kIssuerWarp0) {
         tmem_alloc<true>(smem_u32(tmem_slot), 512);
         tmem_relinquish<true>();
     }
@@ -163,9 +172,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
     if (KIND == MmaKind::MXF4) {
         // constant scale factors 2^0 (UE8M0 byte 127) for every row of A and B, in both CTAs
-        if (warp >= 4 && warp < 8) {
-            const uint32_t q = warp & 3;
-            for (int c = 0; c < kSfCols; ++c) tmem_st1(tmem_base + ((q * 32u) << 16) + C::kSfCol0 + c, 0x7F7F7F7Fu);
+        if (warp < 4) {
+            for (int c = 0; c < kSfCols; ++c) tmem_st1(tmem_base + (((uint32_t)warp * 32u) << 16) + C::kSfCol0 + c, 0x7F7F7F7Fu);
             tmem_st_wait();
         }
         tc_fence_before_sync();
@@ -185,10 +193,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         return got;
     };
 
-    if (warp == 0) {
+    // the same for a whole converged warp, with one answer for all its lanes
+    auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xFFFFFFFFu, wait(bar, parity)) != 0; };
+
+    if (warp == kProducerWarp) {
         // ================= TMA producer (both CTAs) =================
-        if (lane == 0) {
-            uint32_t it = 0, cs = 0;
+        // The whole warp walks the loop (so that every value in it is warp-uniform); one elected lane issues.
+        {
+            uint32_t it = 0;
             bool ok = true;
             const uint32_t lead_full0 = mapa(full_bar(0), 0);
             for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
@@ -197,208 +209,249 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int ks = 0; ks < num_kstages; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
-                    if (!wait(empty_bar(s), ph ^ 1u)) { ok = false; break; }
-                    // The factors of this stage's chunks are in the ring before its operands are requested, so a
-                    // promotion warp that sees the chunk's partial sums complete may read them without a wait of its own.
-                    const int here = min(CPS, nacc - ks * CPS);
-                    for (int h = 0; h < here && ok; ++h, ++cs) ok = wait(sfull_bar(cs % kSD), (cs / kSD) & 1u);
+                    // a stage is free when the MMAs of all of its chunk positions are complete
+#pragma unroll
+                    for (int h = 0; h < CPS; ++h) ok = ok && wait_all(done_bar(s * CPS + h), ph ^ 1u);
                     if (!ok) break;
-                    if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * g.stage_tx_bytes);
-                    tma_load_2d_pair(smem_a0 + s * C::kABytes, &tmA, lead_full0 + 8u * s, ks * 128, m_idx * TM + (int)rank * CM);
-                    tma_load_2d_pair(smem_b0 + s * C::kBBytes, &tmB, lead_full0 + 8u * s, ks * 128, n_idx * TN + (int)rank * kBRows);
+                    if (elect_one()) {
+                        if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * g.stage_tx_bytes);
+                        tma_load_2d_pair(smem_a0 + s * C::kABytes, &tmA, lead_full0 + 8u * s, ks * 128, m_idx * TM + (int)rank * CM);
+                        tma_load_2d_pair(smem_b0 + s * C::kBBytes, &tmB, lead_full0 + 8u * s, ks * 128, n_idx * TN + (int)rank * kBRows);
+                    }
+                    __syncwarp();
                 }
             }
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer (leader only) =================
-        if (lane == 0 && rank == 0) {
-            uint32_t it = 0, cc = 0;
-            bool ok = true;
+    } else if (warp >= kIssuerWarp0 && warp < kIssuerWarp0 + kIssuers) {
+        // ================= MMA issuers (leader only) =================
+        // The whole warp walks the loop, one elected lane issues; issuer i takes the chunk positions p = i, i + kIssuers, ... of the sequence of
+        // all stages' positions (a tcgen05.commit costs its thread a few hundred cycles, more than a chunk's MMAs
+        // take to run, so one thread alone cannot keep the tensor core busy).  Chunks are independent of one
+        // another: each has its own accumulator buffer and its own commit.
+        if (rank == 0) {
+            const int me = warp - kIssuerWarp0;
             const uint32_t sfa = tmem_base + C::kSfCol0, sfb = tmem_base + C::kSfCol0 + 16;
-            // completion of everything issued so far, signalled to the same barrier of both CTAs
-            auto commit_both = [&](uint32_t bar) {
-                tc_commit<true>(bar);
-                tc_commit<true>(mapa(bar, 1));
-            };
-            for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
-                for (int ks = 0; ks < num_kstages && ok; ++ks, ++it) {
-                    const int s = it % S;
-                    const uint32_t ph = (it / S) & 1u;
-                    if (!wait(full_bar(s), ph)) { ok = false; break; }
+            const uint32_t pos_per_tile = (uint32_t)num_kstages * CPS;
+            const uint32_t total_pos = (uint32_t)my_tiles * pos_per_tile;
+            const uint32_t holes_per_tile = pos_per_tile - (uint32_t)nacc;   // positions of a tile's last stage without a chunk
+            const uint32_t done_peer0 = mapa(done_bar(0), 1);
+            bool ok = true;
+            for (uint32_t p = (uint32_t)me; p < total_pos && ok; p += kIssuers) {
+                const uint32_t it = p / CPS, h = p % CPS;
+                const uint32_t tile_seq = p / pos_per_tile, in_tile = p - tile_seq * pos_per_tile;
+                const int s = it % S;
+                const uint32_t ph = (it / S) & 1u;
+                // The stage's operands have landed; this also puts the commit below behind the hand-over of the
+                // position's previous occupant (the producer refilled the stage only after seeing that one complete).
+                if (!wait_all(full_bar(s), ph)) { ok = false; break; }
+                if (in_tile < (uint32_t)nacc) {
+                    const uint32_t cc = p - tile_seq * holes_per_tile;   // number of the chunk among the real chunks
+                    const uint32_t b = cc % NB;
+                    if (!wait_all(tempty_bar(b), ((cc / NB) & 1u) ^ 1u)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint64_t adesc = make_smem_desc_k128(smem_a0 + s * C::kABytes);
                     const uint64_t bdesc = make_smem_desc_k128(smem_b0 + s * C::kBBytes);
+                    constexpr int kPerChunk = 4 / CPS;   // 32-byte K steps per chunk
+                    if (elect_one()) {
 #pragma unroll
-                    for (int h = 0; h < CPS; ++h) {
-                        if (ks * CPS + h < nacc) {
-                            const uint32_t b = cc % NB;
-                            if (!wait(tempty_bar(b), ((cc / NB) & 1u) ^ 1u)) { ok = false; break; }
-                            tc_fence_after_sync();
-                            constexpr int kPerChunk = 4 / CPS;   // 32-byte K steps per chunk
-#pragma unroll
-                            for (int k = 0; k < kPerChunk; ++k)
-                                mma_ss<KIND, true>(tmem_base + b * TN, adesc + 2 * (kPerChunk * h + k), bdesc + 2 * (kPerChunk * h + k), idesc,
-                                                   k > 0 ? 1u : 0u, sfa, sfb);
-                            commit_both(tfull_bar(b));
-                            ++cc;
-                        }
-                    }
-                    if (ok) commit_both(empty_bar(s));
-                }
-            }
-        }
-    } else if (warp == 2 || warp == 3) {
-        // ================= scale loaders =================
-        // warp 2: factors of this CTA's 128 rows; block mode: 1/(S_a*S_b), vector mode: 1/S_a.
-        // warp 3 (vector mode only): 1/S_b of the tile's 128 columns.
-        const bool rows_side = (warp == 2);
-        if (rows_side || SCALE == PSCALE_VEC_B) {
-            constexpr int PD = 4;        // chunks whose global loads are in flight in registers
-            float4 qv[PD];
-            float qb[PD];
-            int pt = first_tile, pj = 0;   // tile and chunk of the next load to issue
-            auto issue = [&](float4 &dv, float &db) {
-                dv = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
-                db = 1.0f;
-                if (pt < num_tiles) {
-                    int m_idx, n_idx;
-                    pair_tile_coords(pt, num_m, num_n, m_idx, n_idx);
-                    if (rows_side) {
-                        // rows outside the matrix repeat the last four rows' factors (their sums are never stored)
-                        const int r = min(m_idx * TM + (int)rank * CM + 4 * lane, g.Mo - 4);
-                        dv = __ldg(reinterpret_cast<const float4 *>(g.sa + (int64_t)pj * g.sa_chunk_stride + r));
-                        if (SCALE == PSCALE_BLOCK_B) db = __ldg(g.sb + (int64_t)n_idx * g.sb_blk_stride + (int64_t)pj * g.sb_chunk_stride);
-                    } else {
-                        const int c = min(n_idx * TN + 4 * lane, g.No - 4);
-                        dv = __ldg(reinterpret_cast<const float4 *>(g.sb + (int64_t)pj * g.sb_chunk_stride + c));
-                    }
-                    if (++pj == nacc) { pj = 0; pt += tile_step; }
-                }
-            };
-#pragma unroll
-            for (int u = 0; u < PD; ++u) issue(qv[u], qb[u]);
-            // Chunks are walked as one sequence over all of this pair's tiles, PD at a time, so that the register
-            // slot of a chunk is a compile-time index (a run-time choice among the slots would wait for every load
-            // in flight, not only for the chunk's own).
-            const int my_tiles = first_tile < num_tiles ? (num_tiles - first_tile + tile_step - 1) / tile_step : 0;
-            const uint32_t total = (uint32_t)my_tiles * (uint32_t)nacc;
-            uint32_t it_base = 0;   // first stage of the tile being consumed
-            int cj = 0;             // chunk within that tile
-            bool ok = true;
-            for (uint32_t c0 = 0; c0 < total && ok; c0 += PD) {
-#pragma unroll
-                for (int u = 0; u < PD; ++u) {
-                    const uint32_t cc = c0 + u;
-                    if (cc < total && ok) {
-                        const float4 v = qv[u];
-                        const float bsc = qb[u];
-                        issue(qv[u], qb[u]);   // chunk cc + PD
-                        float4 r;
-                        r.x = rcp_fast(v.x * bsc); r.y = rcp_fast(v.y * bsc); r.z = rcp_fast(v.z * bsc); r.w = rcp_fast(v.w * bsc);
-                        // the slot is free once the stage this chunk travels in is free (see PCfg)
-                        const uint32_t its = it_base + (uint32_t)(cj / CPS);
-                        if (!wait(empty_bar(its % S), ((its / S) & 1u) ^ 1u)) { ok = false; }
-                        else {
-                            const uint32_t d = cc % kSD;
-                            *reinterpret_cast<float4 *>(ring + d * kSlotFloats + (rows_side ? 0 : 128) + 4 * lane) = r;
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(sfull_bar(d));
-                            if (++cj == nacc) { cj = 0; it_base += (uint32_t)num_kstages; }
-                        }
+                        for (int k = 0; k < kPerChunk; ++k)
+                            mma_ss<KIND, true>(tmem_base + b * TN, adesc + 2 * (kPerChunk * h + k), bdesc + 2 * (kPerChunk * h + k), idesc,
+                                               k > 0 ? 1u : 0u, sfa, sfb);
                     }
                 }
-            }
-        }
-    } else {
-        // ================= promotion / epilogue warps =================
-        const int e = warp - 4;          // 0..15
-        const int q = warp & 3;          // tensor-memory lane quarter this warp may access (= e & 3)
-        const int cg = e >> 2;           // 32-column group
-        const uint32_t stage_u32 = out_stage0 + e * 2048;
-        const uint32_t tempty_lead0 = mapa(tempty_bar(0), 0);
-        uint32_t cc = 0;
-        bool ok = true;
-        for (int t = first_tile; t < num_tiles && ok; t += tile_step) {
-            int m_idx, n_idx;
-            pair_tile_coords(t, num_m, num_n, m_idx, n_idx);
-            const int row0 = m_idx * TM + (int)rank * CM + q * 32;
-            const int row = row0 + lane;
-            const int col0 = n_idx * TN + cg * 32;
-            float2 acc[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = make_float2(0.0f, 0.0f);
-            for (int j = 0; j < nacc; ++j, ++cc) {
-                const uint32_t b = cc % NB;
-                const float *slot = ring + (cc % kSD) * kSlotFloats;
-                {
-                    const bool got = wait(tfull_bar(b), (cc / NB) & 1u);
-                    if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+                // (a position without a chunk - the second half of a last stage - is committed all the same: the
+                // producer and the peer CTA count positions)
+                if (elect_one()) {
+                    tc_commit<true>(done_bar(s * CPS + h));
+                    tc_commit<true>(done_peer0 + 8u * (s * CPS + h));
                 }
-                tc_fence_after_sync();
-                uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + b * TN + cg * 32, v);
-                const float f = slot[q * 32 + lane];   // in the shadow of the load
-                tmem_ld_wait();
-                // this warp's reads of buffer b are done: hand it back to the MMA issuer
-                tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(tempty_lead0 + 8u * b);
-                const float2 ff = make_float2(f, f);
-                if (SCALE == PSCALE_BLOCK_B) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        acc[i] = __ffma2_rn(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), ff, acc[i]);
-                } else {
-                    const float4 *cf = reinterpret_cast<const float4 *>(slot + 128 + cg * 32);   // reciprocal column scales, broadcast reads
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 s4 = cf[i];
-                        const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1])), make_float2(s4.x, s4.y));
-                        const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])), make_float2(s4.z, s4.w));
-                        acc[2 * i] = __ffma2_rn(p0, ff, acc[2 * i]);
-                        acc[2 * i + 1] = __ffma2_rn(p1, ff, acc[2 * i + 1]);
+            }
+        }
+    } else if (warp == kLoaderWarp) {
+        // ================= scale loader =================
+        // Lane l brings the factors of rows 4l..4l+3 of this CTA (block mode: 1/(S_a*S_b); vector mode: 1/S_a and,
+        // for the tile's columns 4l..4l+3, 1/S_b).  Chunks are walked as one sequence over all of this pair's
+        // tiles.  Chunk c + kAhead is requested (16-byte cp.async copies, one commit group) as soon as the promotion
+        // warps have let go of the ring slot it lands in; chunk c is then awaited, turned into reciprocals in
+        // place by the lanes that fetched it, and published.  Neither the operand pipeline nor the tensor core
+        // ever waits for a scale factor's trip from global memory.
+        const uint32_t total = (uint32_t)my_tiles * (uint32_t)nacc;
+        const uint32_t ring_u32 = smem_u32(ring);
+        int pt = first_tile, pj = 0;   // tile and chunk of the next request
+        uint32_t pc = 0;               // its position in the sequence
+        bool ok = true;
+        // source addresses of the requested tile's first chunk (recomputed when the tile changes)
+        const float *src_a = g.sa, *src_b = g.sb;
+        auto tile_sources = [&]() {
+            int m_idx, n_idx;
+            pair_tile_coords(pt < num_tiles ? pt : first_tile, num_m, num_n, m_idx, n_idx);
+            // rows / columns outside the matrix repeat the last four factors (their sums are never stored)
+            src_a = g.sa + min(m_idx * TM + (int)rank * CM + 4 * lane, g.Mo - 4);
+            if (SCALE == PSCALE_BLOCK_B) src_b = g.sb + (int64_t)n_idx * g.sb_blk_stride;
+            else src_b = g.sb + min(n_idx * TN + 4 * lane, g.No - 4);
+        };
+        tile_sources();
+        auto request = [&]() {
+            if (pc < total && ok) {
+                const uint32_t d = pc % kSD;
+                // the first slot of a ring block is requested once the promotion warps have handed the block back
+                if ((pc % kSBlk) == 0 && !wait(sempty_bar(d / kSBlk), ((pc / kSD) & 1u) ^ 1u)) ok = false;
+                else {
+                    const uint32_t slot = ring_u32 + d * (kSlotFloats * 4);
+                    cp_async_16(slot + 16u * lane, src_a);
+                    if (SCALE == PSCALE_BLOCK_B) {
+                        if (lane == 0) cp_async_4(slot + 512u, src_b);
+                    } else {
+                        cp_async_16(slot + 512u + 16u * lane, src_b);
                     }
+                    src_a += g.sa_chunk_stride;
+                    src_b += g.sb_chunk_stride;
+                    if (++pj == nacc) { pj = 0; pt += tile_step; tile_sources(); }
                 }
             }
-            if (!ok) break;
-            const float *av = reinterpret_cast<const float *>(acc);
-            if (!g.accumulate) {
-                // round, stage 32 rows x 64 bytes (16-byte pieces XOR-swizzled as the output map's 64-byte swizzle
-                // expects) and let the TMA unit write the box; parts outside the matrix are clipped by the hardware
-                constexpr int kPerBox = OUT_F32 ? 16 : 32;
+            ++pc;
+            cp_async_commit();   // one group per position, empty past the end, so that the count below stays uniform
+        };
+        for (int i = 0; i < kAhead; ++i) request();
+        for (uint32_t cc = 0; cc < total && ok; ++cc) {
+            request();                  // position cc + kAhead
+            cp_async_wait<kAhead>();    // this lane's copies of position cc have landed
+            const uint32_t d = cc % kSD;
+            float4 *mine = reinterpret_cast<float4 *>(ring + d * kSlotFloats + 4 * lane);
+            const float4 v = *mine;
+            if (SCALE == PSCALE_BLOCK_B) {
+                __syncwarp();           // lane 0's copy of the block scale is visible to the warp
+                const float bsc = ring[d * kSlotFloats + 128];
+                *mine = make_float4(rcp_fast(v.x * bsc), rcp_fast(v.y * bsc), rcp_fast(v.z * bsc), rcp_fast(v.w * bsc));
+            } else {
+                const float4 w = mine[32];
+                *mine = make_float4(rcp_fast(v.x), rcp_fast(v.y), rcp_fast(v.z), rcp_fast(v.w));
+                mine[32] = make_float4(rcp_fast(w.x), rcp_fast(w.y), rcp_fast(w.z), rcp_fast(w.w));
+            }
+            __syncwarp();
+            // a block is published when its last slot (or the last chunk of all) is ready
+            if (lane == 0 && ((cc % kSBlk) == kSBlk - 1 || cc + 1 == total)) mbar_arrive(sfull_bar(d / kSBlk));
+        }
+        cp_async_wait<0>();
+    } else if (warp < kEpiWarps) {
+        // ================= promotion / epilogue warps =================
+        // Per chunk a warp has little arithmetic (16 packed multiply-adds) against several hand-offs, so the loop is
+        // arranged for the hand-offs not to wait on one another: the scale ring is taken and given back eight
+        // chunks at a time, the next chunk's completion barrier is tested (without blocking) while this chunk's
+        // tensor-memory load is in flight, and buffers go back with relaxed arrivals that nobody waits for.
+        const int e = warp;              // 0..15
+        const int q = warp & 3;          // tensor-memory lane quarter this warp may access
+        const int cg = e >> 2;           // 32-column group
+        const uint32_t tempty_lead0 = mapa(tempty_bar(0), 0);
+        const uint32_t total = (uint32_t)my_tiles * (uint32_t)nacc;
+        const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16) + cg * 32;
+        // ring position of the current chunk: stage s (parity sph), chunk h of the stage; buffer b; chunk j of the tile
+        uint32_t s = 0, sph = 0, h = 0, b = 0;
+        int j = 0, t = first_tile;
+        int row0 = 0, col0 = 0;
+        bool have = false;               // the current chunk's completion has already been seen
+        bool ok = true;
+        float2 acc[16];
+        for (uint32_t cc = 0; cc < total && ok; ++cc) {
+            if (j == 0) {
+                int m_idx, n_idx;
+                pair_tile_coords(t, num_m, num_n, m_idx, n_idx);
+                row0 = m_idx * TM + (int)rank * CM + q * 32;
+                col0 = n_idx * TN + cg * 32;
 #pragma unroll
-                for (int bx = 0; bx < 32 / kPerBox; ++bx) {
-                    if (lane == 0) bulk_wait_read0();     // the previous box has left the staging tile
-                    __syncwarp();
-                    const float *src = av + bx * kPerBox;
+                for (int i = 0; i < 16; ++i) acc[i] = make_float2(0.0f, 0.0f);
+            }
+            const uint32_t d = cc % kSD;
+            const float *slot = ring + d * kSlotFloats;
+            const uint32_t dp = s * CPS + h;
+            if ((cc % kSBlk) == 0) {
+                const bool got = wait(sfull_bar(d / kSBlk), (cc / kSD) & 1u);
+                if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+            }
+            if (!have) {
+                const bool got = wait(done_bar(dp), sph);
+                if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+            }
+            tc_fence_after_sync();
+            uint32_t v[32];
+            tmem_ld32(taddr0 + b * TN, v);
+            const float f = slot[q * 32 + lane];
+            // position of the next chunk (the tile's last stage may have fewer chunks than positions)
+            const bool tile_end = (j + 1 == nacc);
+            uint32_t ns = s, nsph = sph, nh = h + 1;
+            if (nh == CPS || tile_end) { nh = 0; if (++ns == S) { ns = 0; nsph ^= 1u; } }
+            // non-blocking look at the next chunk's barrier while the load is in flight
+            const bool next_seen = (cc + 1 < total) && mbar_test_wait(done_bar(ns * CPS + nh), nsph);
+            tmem_ld_wait();
+            // this warp's reads of buffer b are done: hand it back to the MMA issuers
+            // (the sixteen warps meet on a hardware barrier - one per buffer, fifteen arrive without waiting - and
+            // the warp that waits sends ONE arrival per CTA: arrivals on one mbarrier are served one after the other,
+            // and thirty-two of them per chunk would take longer than the chunk's MMAs)
+            tc_fence_before_sync();
+            if (e == (int)b) {
+                named_bar_sync(1 + b, 32 * kEpiWarps);
+                if (lane == 0) mbar_arrive_cluster_relaxed(tempty_lead0 + 8u * b);
+            } else {
+                named_bar_arrive(1 + b, 32 * kEpiWarps);
+            }
+            const float2 ff = make_float2(f, f);
+            if (SCALE == PSCALE_BLOCK_B) {
 #pragma unroll
-                    for (int p = 0; p < 4; ++p) {
-                        uint4 o;
-                        if (OUT_F32) o = make_uint4(__float_as_uint(src[4 * p]), __float_as_uint(src[4 * p + 1]), __float_as_uint(src[4 * p + 2]), __float_as_uint(src[4 * p + 3]));
-                        else o = make_uint4(bf16x2_bits(src[8 * p], src[8 * p + 1]), bf16x2_bits(src[8 * p + 2], src[8 * p + 3]),
-                                            bf16x2_bits(src[8 * p + 4], src[8 * p + 5]), bf16x2_bits(src[8 * p + 6], src[8 * p + 7]));
-                        st_shared_v4(stage_u32 + lane * 64 + ((p ^ ((lane >> 1) & 3)) << 4), o);
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    const int col = col0 + bx * kPerBox;
-                    if (lane == 0 && col < g.No && row0 < g.Mo) { tma_store_2d(&tmO, stage_u32, col, row0); bulk_commit(); }
+                for (int i = 0; i < 16; ++i)
+                    acc[i] = __ffma2_rn(make_float2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), ff, acc[i]);
+            } else {
+                const float4 *cf = reinterpret_cast<const float4 *>(slot + 128 + cg * 32);   // reciprocal column scales, broadcast reads
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 s4 = cf[i];
+                    const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1])), make_float2(s4.x, s4.y));
+                    const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3])), make_float2(s4.z, s4.w));
+                    acc[2 * i] = __ffma2_rn(p0, ff, acc[2 * i]);
+                    acc[2 * i + 1] = __ffma2_rn(p1, ff, acc[2 * i + 1]);
                 }
-            } else if (row < g.Mo) {
-                // FP32 accumulation into the existing output (gradient accumulation)
-                float *dst = static_cast<float *>(g.out) + (int64_t)row * g.ldo + col0;
+            }
+            have = __all_sync(0xFFFFFFFFu, next_seen);
+            if ((cc % kSBlk) == kSBlk - 1) {
+                // every lane's reads of the block's slots are behind this warp barrier (their values have been used)
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sempty_bar(d / kSBlk));
+            }
+            s = ns; sph = nsph; h = nh;
+            if (++b == NB) b = 0;
+            if (!tile_end) { ++j; continue; }
+            // ---- the tile is complete: round and store ----
+            j = 0;
+            const int row = row0 + lane;
+            const float *av = reinterpret_cast<const float *>(acc);
+            if (row < g.Mo) {
+                // each lane owns 32 consecutive outputs of its row: 16-byte stores (L2 merges them into whole sectors)
+                if (OUT_F32) {
+                    float *dst = static_cast<float *>(g.out) + (int64_t)row * g.ldo + col0;
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    if (col0 + i < g.No) {
-                        float4 o = *reinterpret_cast<const float4 *>(dst + i);
-                        o.x += av[i]; o.y += av[i + 1]; o.z += av[i + 2]; o.w += av[i + 3];
-                        *reinterpret_cast<float4 *>(dst + i) = o;
+                    for (int i = 0; i < 32; i += 4) {
+                        if (col0 + i < g.No) {
+                            float4 o = make_float4(av[i], av[i + 1], av[i + 2], av[i + 3]);
+                            if (g.accumulate) {   // gradient accumulation into the existing FP32 output
+                                const float4 p = *reinterpret_cast<const float4 *>(dst + i);
+                                o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+                            }
+                            *reinterpret_cast<float4 *>(dst + i) = o;
+                        }
+                    }
+                } else {
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(g.out) + (int64_t)row * g.ldo + col0;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        if (col0 + i < g.No)
+                            *reinterpret_cast<uint4 *>(dst + i) = make_uint4(bf16x2_bits(av[i], av[i + 1]), bf16x2_bits(av[i + 2], av[i + 3]),
+                                                                             bf16x2_bits(av[i + 4], av[i + 5]), bf16x2_bits(av[i + 6], av[i + 7]));
                     }
                 }
             }
             __syncwarp();
+            t += tile_step;
         }
-        if (lane == 0) bulk_wait_all0();   // outstanding output stores have read their staging tiles
     }
 
     // ---- teardown: every role ends here; tensor memory is always released ---------------------
@@ -413,7 +466,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (threadIdx.x == 0) atomicExch(g.status, (uint32_t)SNIP_ERR_TIMEOUT);
         __syncthreads();
     }
-    if (warp == 1) {
+    if (warp == kIssuerWarp0) {
         tc_fence_after_sync();
         tmem_dealloc<true>(tmem_base, 512);
     }

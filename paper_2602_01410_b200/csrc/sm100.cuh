@@ -25,6 +25,20 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
 template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
+// One lane of a converged warp (the same one every time), chosen in a way the compiler knows to be
+// warp-uniform: code under `if (elect_one())` keeps its operands in uniform registers, which is what
+// the TMA and tcgen05 instructions read (a `lane == 0` branch forces a move per operand per instruction).
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xFFFFFFFF;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // ---- thread-block clusters (pairs of CTAs sharing one MMA) -------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
@@ -49,10 +63,29 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Same without release semantics: for hand-offs that publish no ordinary memory (a tensor-memory buffer whose
+// loads have been waited for; shared-memory values that have already been consumed).  A release at cluster
+// scope would first wait for every earlier memory operation of the thread.
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // Plain 32-bit store into the shared memory of a CTA of the cluster.
 __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v)
 {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+
+// ---- named CTA barriers (hardware barriers 1..15; 0 is __syncthreads) -----------------------
+// `count` threads in all take part, each either arriving (does not wait) or synchronising (waits for
+// the others).  Whole warps only.
+__device__ __forceinline__ void named_bar_arrive(uint32_t id, uint32_t count)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
 
 // ---- mbarrier ------------------------------------------------------------------------------
