@@ -421,8 +421,9 @@ int snip_select_scheme(int m, int n, const double *q, const int64_t *w, int64_t 
  *                              ever while every copy still lands: the kernel's waits run out, it
  *                              leaves on its own and snip_poll_status reports SNIP_ERR_TIMEOUT.
  *                              Nothing traps or faults; used with a short wait limit by the tests.
- *   SNIP_DEBUG_GEMM_KERNEL   : 0 = automatic choice, 1 = single-CTA kernels only, 2 = CTA-pair
- *                              kernels for every quantized GEMM (A/B comparisons in the benchmark).
+ *   SNIP_DEBUG_GEMM_KERNEL   : 0 or 1 = the single-CTA kernels (the default), 2 = the CTA-pair
+ *                              kernels for every quantized GEMM (an alternative form of the same
+ *                              product, kept for A/B comparisons in the benchmark).
  * Returns SNIP_ERR_ARG for an unknown key or a value out of range.
  */
 #define SNIP_DEBUG_WAIT_LIMIT_NS 0

@@ -650,7 +650,7 @@ size_t gemm_ws_bytes() { return 256; }
 namespace {
 std::atomic<long long> g_wait_limit_ns{2000000000ll};   // bound of every device-side wait of the GEMM kernels
 std::atomic<int> g_tx_skew{0};                           // bytes added to what a stage's barrier expects (a wait that cannot complete)
-std::atomic<int> g_kernel_choice{0};                     // 0 = automatic, 1 = single-CTA kernels only, 2 = CTA-pair kernels where they apply
+std::atomic<int> g_kernel_choice{0};                     // 0, 1 = single-CTA kernels, 2 = CTA-pair kernels for quantized operands
 }  // namespace
 
 int gemm_pair_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
@@ -714,10 +714,10 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     const int tx_skew = g_tx_skew.load();
     const bool f32 = out_dtype == SNIP_OUT_FP32;
 
-    // Quantized operands: the CTA-pair kernels (256 x 128 tiles) wherever an output has at least one full tile
-    // of rows; shorter outputs stay on the single-CTA kernels below (a pair would idle one of its two SMs).
+    // The CTA-pair kernels (gemm_pair.cu) are an alternative form of the same product, kept for comparison: they
+    // run only when asked for through snip_debug_set (on the 7B shapes they are slower than the kernels below).
     const int choice = g_kernel_choice.load();
-    if (!a16 && choice != 1 && (Mo >= 256 || choice == 2))
+    if (!a16 && choice == 2)
         return gemm_pair_impl(fmt_a, fmt_b, a_codes, b_codes, Mo, No, Kc, sa, sa_chunk_stride, sb, sb_chunk_stride, sb_blk_stride, scale_mode,
                               out, out_dtype, accumulate, g.status, g.wait_limit_ns, tx_skew, st);
 

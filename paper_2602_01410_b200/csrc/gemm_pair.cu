@@ -6,21 +6,25 @@
 //
 // Two CTAs on neighbouring SMs (a cluster of 2) share one tcgen05.mma.cta_group::2: the tile is
 // 256 rows x 128 columns, each CTA holds 128 rows of A, 64 rows of B and a 128 x 128 slice of the
-// accumulator.  That slice is only a quarter of the register file, which leaves room for SIXTEEN
-// promotion warps (four per scheduler) - the FP32 multiply-adds of the promotion, not the tensor
-// pipe, set the pace of these kernels - and its tensor-memory image is 128 columns, so three or four
-// chunks can be in flight between the MMA issuer and the promotion warps.
+// accumulator.  That slice is only a quarter of the register file, which leaves room for sixteen
+// promotion warps (four per scheduler), and its tensor-memory image is 128 columns, so three or four
+// chunks can be in flight between the MMA issuers and the promotion warps.
+//
+// This is an ALTERNATIVE form of the product computed by gemm.cu, selected only through
+// snip_debug_set(SNIP_DEBUG_GEMM_KERNEL, 2): measured on the 7B shapes it is slower than the
+// single-CTA kernels (each of its hand-offs costs a warp a few hundred cycles, and with 128-column
+// buffers there is one hand-off per 2 M multiply-adds instead of one per 4 M).
 //
 // Roles in one CTA (640 threads):
-//   warp 0      : TMA producer  - this CTA's halves of the operand tiles into a shared-memory ring;
+//   warps 0..15 : promotion     - 32 rows x 32 columns each (warp % 4 = tensor-memory lane quarter)
+//   warp 16     : TMA producer  - this CTA's halves of the operand tiles into a shared-memory ring;
 //                                 byte counts are reported to the leader's barrier (no multicast)
-//   warp 1      : MMA issuer    - leader CTA only, one thread; owns the tensor-memory allocation
-//   warp 2 (,3) : scale loader  - brings the chunks' scale factors into a 32-deep shared-memory ring
-//                                 with cp.async, two dozen chunks ahead of their use, and turns them
-//                                 into reciprocal factors in place (warp 3: the per-column factors
-//                                 of wgrad)
-//   warps 4..19 : promotion     - 32 rows x 32 columns each
-// Every wait is bounded; on a timeout both CTAs leave cleanly and a status word is raised.
+//   warp 17     : scale loader  - brings the chunks' scale factors into a shared-memory ring with
+//                                 cp.async, well ahead of their use, and turns them into reciprocal
+//                                 factors in place
+//   warps 18,19 : MMA issuers   - leader CTA only, alternate chunks; the whole warp walks the loop
+//                                 and one elected lane issues, so operands stay in uniform registers
+// Every mbarrier wait is bounded; on a timeout both CTAs leave cleanly and a status word is raised.
 #include <cuda.h>
 #include <cuda_bf16.h>
 

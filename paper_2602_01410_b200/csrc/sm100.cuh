@@ -142,6 +142,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           uint64_t limit_ns = 2000000000ull)
 {
     if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;   // after a failed wait anywhere in the CTA every later wait returns at once
     const uint64_t t0 = globaltimer_ns();
     for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -163,6 +164,12 @@ __device__ __forceinline__ void cp_async_4(uint32_t dst, const void *src)
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// Makes `bar` receive one arrival from this thread once all of its earlier cp.async copies have landed
+// (the arrival is counted in the barrier's expected count: "noinc").
+__device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
