@@ -357,7 +357,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         bool have = false;               // the current chunk's completion has already been seen
         bool ok = true;
         float2 acc[16];
-        for (uint32_t cc = 0; cc < total && ok; ++cc) {
+        for (uint32_t cc = 0; cc < total; ++cc) {   // never left early: the other warps wait for this one on hardware barriers
+            // (after a failed wait every later wait returns at once)
             if (j == 0) {
                 int m_idx, n_idx;
                 pair_tile_coords(t, num_m, num_n, m_idx, n_idx);
@@ -371,11 +372,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t dp = s * CPS + h;
             if ((cc % kSBlk) == 0) {
                 const bool got = wait(sfull_bar(d / kSBlk), (cc / kSD) & 1u);
-                if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+                if (!__all_sync(0xFFFFFFFFu, got)) ok = false;
             }
             if (!have) {
                 const bool got = wait(done_bar(dp), sph);
-                if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+                if (!__all_sync(0xFFFFFFFFu, got)) ok = false;
             }
             tc_fence_after_sync();
             uint32_t v[32];
@@ -428,7 +429,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             j = 0;
             const int row = row0 + lane;
             const float *av = reinterpret_cast<const float *>(acc);
-            if (row < g.Mo) {
+            if (row < g.Mo && ok) {
                 // each lane owns 32 consecutive outputs of its row: 16-byte stores (L2 merges them into whole sectors)
                 if (OUT_F32) {
                     float *dst = static_cast<float *>(g.out) + (int64_t)row * g.ldo + col0;

@@ -284,19 +284,23 @@ extern "C" int snip_layer_stats(const snip_layer_tensors_t *t, uint32_t fmt_mask
     rc = require_sm100();
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    SNIP_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(snip_layer_stats_t), st));
     const int64_t M = t->M, N = t->N, K = t->K;
     struct T { const void *p; int64_t r, c; int qidx; } tens[6] = {
         {t->X, M, K, 0}, {t->W, N, K, 1}, {t->Y, M, N, -1}, {t->dY, M, N, 2}, {t->dX, M, K, -1}, {t->dW, N, K, -1}};
+    // every argument is checked before anything is enqueued
+    for (int i = 0; i < 6; ++i) {
+        if (!tens[i].p) continue;
+        if (!aligned16(tens[i].p)) return SNIP_ERR_ALIGN;
+        if (ceil_div(tens[i].r, kTile) > 65535) return SNIP_ERR_SHAPE;
+    }
+    SNIP_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(snip_layer_stats_t), st));
     uint8_t *cursor = static_cast<uint8_t *>(ws);
     for (int i = 0; i < 6; ++i) {
         const size_t region = tensor_ws_bytes(tens[i].r, tens[i].c);
         StatsPartial *parts = reinterpret_cast<StatsPartial *>(cursor);
         cursor += region;
         if (!tens[i].p) continue;
-        if (!aligned16(tens[i].p)) return SNIP_ERR_ALIGN;
         const int64_t tr = ceil_div(tens[i].r, kTile), tc = ceil_div(tens[i].c, kTile);
-        if (tr > 65535) return SNIP_ERR_SHAPE;
         LayerStatsArgs a;
         a.x = static_cast<const uint16_t *>(tens[i].p);
         a.rows = tens[i].r; a.cols = tens[i].c;

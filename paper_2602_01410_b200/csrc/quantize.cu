@@ -1027,7 +1027,8 @@ extern "C" int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, 
 {
     using namespace snip;
     if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
-    const size_t need = stats_ws_bytes(rows, cols, false);
+    // only the statistics use scratch: a call without SNIP_Q_STATS never touches the built-in array
+    const size_t need = (flags & SNIP_Q_STATS) ? stats_ws_bytes(rows, cols, false) : 0;
     if (need > kStaticScratchBytes) {
         snprintf(last_error_buffer(), 256, "snip_quantize_noalloc: %lld x %lld needs %zu bytes of scratch, the built-in array holds %zu",
                  (long long)rows, (long long)cols, need, kStaticScratchBytes);

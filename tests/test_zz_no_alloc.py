@@ -47,3 +47,18 @@ def test_inputs_beyond_the_built_in_scratch_are_rejected():
                                                                            api.Q_STATS, api._p(codes), api._p(scales), api._p(stats), None))
     assert e.value.status == api.ERR_WORKSPACE
     assert b"built-in array" in api._lib.snip_last_cuda_error()
+
+
+def test_without_statistics_the_size_limit_does_not_apply():
+    # No SNIP_Q_STATS: the built-in array is not used, so a tensor of more than 16384 tiles goes through
+    # and gives what snip_quantize gives.
+    from paper_2602_01410_b200 import api
+    rows, cols = 129 * 128, 128 * 128          # 16512 tiles
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    x = torch.randn(rows, cols, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    want_codes, want_scales, _, _ = api.snip_quantize(x, api.FMT_FP8_E4M3, api.BLOCK_ROW, 0)
+    codes = torch.full_like(want_codes, 0xAA)
+    scales = torch.full_like(want_scales, -1.0)
+    api.snip_quantize_noalloc(x, api.FMT_FP8_E4M3, api.BLOCK_ROW, 0, codes, scales, None)
+    torch.cuda.synchronize()
+    assert torch.equal(codes, want_codes) and torch.equal(scales, want_scales)
