@@ -17,7 +17,7 @@ stream, into one of two input sets, so that the copy of one step overlaps the ke
 previous one) and reads the statistics back.  `cpu_baseline` times the CPU oracle on a bounded
 sample on this machine's host cores.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 7b|1b|small]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload 7b|1b|small|3b|70b]
 """
 from __future__ import annotations
 
@@ -108,7 +108,11 @@ WORKLOADS = {
     "7b": (3, None),
     "1b": (1, None),
     "small": (0, None),
+    # table-driven precision mix: every GEMM takes the tag the configuration's seeded table gives it
+    "3b": (2, None),
+    "70b": (4, None),
 }
+TAGGED_LAYERS = 4   # layers of a table-driven workload kept resident and run per step
 
 
 def make_device_inputs(cfg, torch, device, seed):
@@ -211,7 +215,7 @@ class Step:
         self.sf = [torch.empty(cb // 32 + 4096, dtype=torch.uint8, device=dev) for _ in range(nbuf)]   # UE8M0 atoms (power-of-two option)
         self.gws = torch.zeros(1024, dtype=torch.uint8, device=dev)
 
-    def run_decomposed(self, events=None, mx=False):
+    def run_decomposed(self, events=None, mx=False, qevents=None):
         api, torch = self.api, self.torch
         if not hasattr(self, "codes"):
             self._alloc_decomposed()
@@ -232,7 +236,14 @@ class Step:
             r, c = x.shape
             outs = [api.QOut(fmt, 0, p(self.codes[slot + j]), p(self.scales[slot + j]), p(self.sf[slot + j]) if mx else None,
                              p(stats_row[24 * j:24 * j + 24]), 0) for j in range(2)]
+            if qevents is not None:
+                q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                q0.record()
             api._check("snip_quantize_dual", lib.snip_quantize_dual(p(x), r, c, c, kind, int(mx), outs[0], outs[1], p(self.qws), self.qws.numel(), st))
+            if qevents is not None:
+                q1.record()
+                # algorithmic bytes: one bf16 read, two code + scale outputs
+                qevents.append((fmt, (2.0 + 2.0 * ((1.0 if fmt == FMT_FP8 else 0.5) + 4.0 / 128.0)) * r * c, q0, q1))
 
         def gemm(op, fmt, ra, ca, blka, ta, rb, cb_, blkb, tb, out, flops, sa=0, sb_=1):
             a = api.make_qtensor(self.codes[sa], self.scales[sa], ra, ca, fmt, blka, ta)
@@ -269,6 +280,63 @@ class Step:
                 gemm(api.OP_DGRAD, f, M, N, api.BLOCK_ROW, 0, N, K, api.BLOCK_BLK, 1, dx, fl)
                 quant(dy, f, api.BLOCK_COL, T, 0, self.stats[2 * i]); quant(x, f, api.BLOCK_COL, T, 1, self.stats[2 * i + 1]); i += 1
                 gemm(api.OP_WGRAD, f, M, N, api.BLOCK_COL, 1, M, K, api.BLOCK_COL, 1, dw, fl)
+
+
+class TaggedStep:
+    """A table-driven workload (3B: each GEMM drawn FP4 / FP8 / BF16; 70B slice: at least 80 % of the linear-layer
+    FLOPs in FP4, the rest FP8): `layers` layers resident, every linear's forward, input-gradient and weight-gradient
+    GEMM through snip_linear_fwd / dgrad / wgrad with the tag of that GEMM on both operands, statistics on."""
+
+    def __init__(self, api, torch, cfg, device, layers):
+        from paper_2602_01410_b200 import workloads as wl
+        self.api, self.torch, self.cfg, self.layers = api, torch, cfg, layers
+        self.tags = wl.precision_tags(cfg)[:layers]
+        self.inputs = [make_device_inputs(cfg, torch, device, 260201410 + 17 * l) for l in range(layers)]
+        M = cfg.M
+        self.out = [(torch.empty(M, L.N, dtype=torch.bfloat16, device=device), torch.empty(M, L.K, dtype=torch.bfloat16, device=device),
+                     torch.empty(L.N, L.K, dtype=torch.bfloat16, device=device)) for L in cfg.linears]
+        ws_bytes = 0
+        for L in cfg.linears:
+            for op in (api.OP_FWD, api.OP_DGRAD, api.OP_WGRAD):
+                for f in (FMT_BF16, FMT_FP8, FMT_FP4):
+                    ws_bytes = max(ws_bytes, api.snip_workspace_size(op, M, L.N, L.K, f, f)[1])
+        self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
+        n_gemm = layers * len(cfg.linears) * 3
+        self.stats = torch.zeros(n_gemm * 2, 32, dtype=torch.uint8, device=device)
+        self.flops = layers * sum(2.0 * M * L.N * L.K * 3 for L in cfg.linears)
+        self.flops_by_fmt = {}
+        for l in range(layers):
+            for j, L in enumerate(cfg.linears):
+                for gi in range(3):
+                    f = int(self.tags[l, j, gi])
+                    self.flops_by_fmt[f] = self.flops_by_fmt.get(f, 0.0) + 2.0 * M * L.N * L.K
+        # per GEMM: quantized tags: 2 quantizers + 2 reductions + 1 GEMM; BF16 tags: statistics kernels + reductions + GEMM (+ transposes)
+        self.launches_per_step = n_gemm * 5
+
+    def run(self, events=None, inputs=None, before=None):
+        api, torch = self.api, self.torch
+        lib, p, st = api._lib, api._p, api._stream()
+        inputs = self.inputs if inputs is None else inputs
+        i = 0
+        for l in range(self.layers):
+            for j, ((x, w, dy), (y, dx, dw)) in enumerate(zip(inputs[l], self.out)):
+                if before is not None:
+                    before(l, j)
+                M, K = x.shape
+                N = w.shape[0]
+                calls = (("snip_linear_fwd", lambda f, sa, sb: lib.snip_linear_fwd(p(x), p(w), p(y), M, N, K, f, f, api.OUT_BF16, p(sa), p(sb), p(self.ws), self.ws.numel(), st)),
+                         ("snip_linear_dgrad", lambda f, sa, sb: lib.snip_linear_dgrad(p(dy), p(w), p(dx), M, N, K, f, f, api.OUT_BF16, p(sa), p(sb), p(self.ws), self.ws.numel(), st)),
+                         ("snip_linear_wgrad", lambda f, sa, sb: lib.snip_linear_wgrad(p(dy), p(x), p(dw), M, N, K, f, f, api.OUT_BF16, 0, p(sa), p(sb), p(self.ws), self.ws.numel(), st)))
+                for gi, (name, call) in enumerate(calls):
+                    f = int(self.tags[l, j, gi])
+                    if events is not None:
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                    api._check(name, call(f, self.stats[2 * i], self.stats[2 * i + 1]))
+                    if events is not None:
+                        e1.record()
+                        events.append((f, 2.0 * M * N * K, e0, e1))
+                    i += 1
 
 
 class KernelTimer:
@@ -507,6 +575,101 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_tagged(args, api, torch, dist, wl, cfg, device, world, rank, local_rank, barrier, peaks):
+    """Contract line of a table-driven workload (--workload 3b | 70b)."""
+    from paper_2602_01410_b200.replicas import combine_replicas
+    layers = min(cfg.layers, TAGGED_LAYERS)
+    step = TaggedStep(api, torch, cfg, device, layers)
+    for _ in range(max(args.warmup, 3)):
+        step.run()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    events = []
+    e0.record()
+    for _ in range(args.steps):
+        step.run(events)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total, flops_job = combine_replicas(ms_total, step.flops, dist if world > 1 else None, device)
+    assert api.snip_poll_status(step.ws) == 0, "device-side timeout reported"
+    ms_per_step = ms_total / args.steps
+    value = flops_job / (ms_per_step * 1e-3) / 1e12
+    # per operand format: the linear calls (quantizers + GEMM) of the timed region against the GEMM's tensor peak
+    per_format = {}
+    for f, fl, a, b in events:
+        d = per_format.setdefault(f, {"flops": 0.0, "ms": 0.0, "calls": 0})
+        d["flops"] += fl; d["ms"] += a.elapsed_time(b); d["calls"] += 1
+    pf = {}
+    for f, d in per_format.items():
+        ach = d["flops"] / (d["ms"] * 1e-3) / 1e12
+        pk = peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f]
+        pf[FMT_NAME[f]] = {"achieved": ach, "peak": pk, "frac": ach / pk, "calls": d["calls"], "share_of_step": d["ms"] / ms_total,
+                           "share_of_flops": step.flops_by_fmt.get(f, 0.0) / step.flops}
+    worst = min(pf, key=lambda k: pf[k]["frac"])
+    roofline = {"kernel": f"snip_linear_fwd/dgrad/wgrad calls (two quantizer passes with statistics + GEMM), headline = {worst} tags",
+                "bound": "tensor", "achieved": pf[worst]["achieved"], "peak": pf[worst]["peak"], "unit": "TFLOP/s", "frac": pf[worst]["frac"],
+                "traffic": None, "per_format": pf,
+                "peak_source": f"{peaks['source']} cuBLAS bf16 sustained x nominal format ratio (x1 bf16, x2 fp8, x4 fp4)"}
+    # end to end: every step copies the layers' inputs from pinned host memory and reads the statistics back
+    host = [[tuple(t.cpu().pin_memory() for t in trip) for trip in layer] for layer in step.inputs]
+    h2d = sum(t.numel() * 2 for layer in host for trip in layer for t in trip)
+    stats_host = torch.empty_like(step.stats, device="cpu").pin_memory()
+    copy_stream = torch.cuda.Stream(device=device)
+    main_stream = torch.cuda.current_stream(device)
+    state = {"free": None}
+
+    def e2e_step():
+        ready = {}
+        with torch.cuda.stream(copy_stream):
+            if state["free"] is not None:
+                copy_stream.wait_event(state["free"])
+            for l, layer in enumerate(host):
+                for j, trip_h in enumerate(layer):
+                    for d_, h_ in zip(step.inputs[l][j], trip_h):
+                        d_.copy_(h_, non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(copy_stream)
+                    ready[(l, j)] = ev
+        step.run(before=lambda l, j: main_stream.wait_event(ready[(l, j)]))
+        stats_host.copy_(step.stats, non_blocking=True)
+        state["free"] = torch.cuda.Event()
+        state["free"].record(main_stream)
+    e2e_step(); barrier()
+    n_e2e = max(2, min(args.steps, 5))
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    copy_stream.wait_event(s0)
+    for _ in range(n_e2e):
+        e2e_step()
+    s1.record()
+    barrier()
+    ms_e2e, flops_e2e = combine_replicas(s0.elapsed_time(s1) / n_e2e, step.flops, dist if world > 1 else None, device)
+    e2e = {"value": flops_e2e / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": stats_host.numel(), "steps": n_e2e, "overlap": "copies on a second stream, one input set"}
+    if rank != 0:
+        return
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, cores, sample = cpu_baseline_sample(cfg, tokens=2048)
+        cpu = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+    input_bytes = layers * sum(2 * (cfg.M * L.K + L.N * L.K + cfg.M * L.N) for L in cfg.linears)
+    mix = ", ".join(f"{FMT_NAME[f]} {100.0 * v / step.flops:.0f} % of FLOPs" for f, v in sorted(step.flops_by_fmt.items()))
+    line = {"metric": "mixed-precision linear fwd+dgrad+wgrad TFLOP/s", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "seeded mix of bf16 / fp8_e4m3 / fp4_e2m1 per GEMM (fp32 accumulate)", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: {layers} of {cfg.layers} layers x ({','.join(L.name for L in cfg.linears)}) x (fwd,dgrad,wgrad), tokens {cfg.M}, "
+                                   f"per-GEMM precision tags of the seeded table '{cfg.tag_rule}' ({mix}), quantize+stats of both operands of every GEMM",
+                       "l2": f"inputs ({input_bytes / 1e6:.0f} MB) larger than L2", "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": step.launches_per_step * args.steps, "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -547,6 +710,11 @@ def main():
         torch.cuda.synchronize()
 
     cfg = wl.CONFIGS[WORKLOADS[args.workload][0]]
+    if args.workload in ("3b", "70b"):
+        run_tagged(args, api, torch, dist, wl, cfg, device, world, rank, local_rank, barrier, load_peaks())
+        if world > 1:
+            dist.destroy_process_group()
+        return
     formats = (FMT_FP4, FMT_FP8)
     step = Step(api, torch, cfg, device, formats, dual=(args.quantizer == "dual"))
     peaks = load_peaks()
@@ -560,10 +728,10 @@ def main():
         sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    events = []
+    events, qevents = [], []
     e0.record()
     for _ in range(args.steps):
-        step.run_decomposed(events)
+        step.run_decomposed(events, qevents=qevents if step.dual else None)
     e1.record()
     barrier()
     ms_total = e0.elapsed_time(e1)
@@ -674,15 +842,37 @@ def main():
             fam[f] = {"achieved": tot_fl / (tot_ms * 1e-3) / 1e12, "peak": peak, "per_op": per_op, "ms": tot_ms}
             kernels[f"gemm_{FMT_NAME[f]}"] = {"tflops": fam[f]["achieved"], "frac_of_peak": fam[f]["achieved"] / peak,
                                               "peak_tflops": peak, "per_op": per_op}
-    dom = max(in_region, key=lambda f: in_region[f]["ms"])
-    d = in_region[dom]
-    dom_peak = peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[dom]
-    roofline = {"kernel": f"gemm_kernel, {FMT_NAME[dom]} operands (all {d['launches']} launches of the timed region)", "bound": "tensor",
-                "achieved": d["flops"] / (d["ms"] * 1e-3) / 1e12, "peak": dom_peak, "unit": "TFLOP/s",
-                "frac": d["flops"] / (d["ms"] * 1e-3) / 1e12 / dom_peak, "traffic": NCU_TRAFFIC.get(dom),
+    # One roofline object for the step's two kernel families.  GEMMs (tensor-bound): every launch of the timed region,
+    # per operand format, against the measured sustained cuBLAS bf16 rate x the nominal format ratio; the headline
+    # `frac` is the LOWER of the two formats.  Quantizers (HBM-bound): the two-output calls with statistics that the
+    # step runs, algorithmic bytes / event time against the measured copy bandwidth.
+    per_format = {}
+    for f, d in in_region.items():
+        ach = d["flops"] / (d["ms"] * 1e-3) / 1e12
+        pk = peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f]
+        per_format[FMT_NAME[f]] = {"achieved": ach, "peak": pk, "frac": ach / pk, "launches": d["launches"], "share_of_step": d["ms"] / ms_total,
+                                   "nominal_dense_peak": 2250.0 * NOMINAL_RATIO[f], "frac_of_nominal": ach / (2250.0 * NOMINAL_RATIO[f]),
+                                   "traffic": NCU_TRAFFIC.get(f)}
+    worst = min(per_format, key=lambda k: per_format[k]["frac"])
+    qleg = None
+    if qevents:
+        qfmt = {}
+        for fmt, by, a_, b_ in qevents:
+            q = qfmt.setdefault(fmt, {"bytes": 0.0, "ms": 0.0, "calls": 0})
+            q["bytes"] += by; q["ms"] += a_.elapsed_time(b_); q["calls"] += 1
+        qleg = {"kernel": "quantize_dual_kernel + stats_reduce_kernel (two outputs with statistics, every call of the timed region)",
+                "bound": "hbm", "unit": "GB/s", "peak": peaks["hbm_gbs"],
+                "per_format": {FMT_NAME[f]: {"achieved": q["bytes"] / (q["ms"] * 1e-3) / 1e9, "frac": q["bytes"] / (q["ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                             "calls": q["calls"], "share_of_step": q["ms"] / ms_total} for f, q in qfmt.items()}}
+        qleg["achieved"] = min(v["achieved"] for v in qleg["per_format"].values())
+        qleg["frac"] = min(v["frac"] for v in qleg["per_format"].values())
+        qleg["traffic"] = "DRAM bytes of one call equal the algorithmic bytes within 1 % (ncu, profiles/quantize_dual_kernel_*)"
+    roofline = {"kernel": f"gemm_kernel (tcgen05, per-chunk FP32 promotion), headline = {worst} operands: the lower fraction of the two formats",
+                "bound": "tensor", "achieved": per_format[worst]["achieved"], "peak": per_format[worst]["peak"], "unit": "TFLOP/s",
+                "frac": per_format[worst]["frac"], "traffic": per_format[worst]["traffic"],
                 "traffic_case": "one launch, fwd 16384x12288x4096 (ncu, profiles/)",
-                "share_of_step": d["ms"] / ms_total,
-                "peak_source": f"{peaks['source']} cuBLAS bf16 sustained x{NOMINAL_RATIO[dom]:.0f} (nominal {FMT_NAME[dom]}/bf16 ratio)"}
+                "per_format": per_format, "quantizer": qleg,
+                "peak_source": f"{peaks['source']} cuBLAS bf16 sustained x nominal format ratio (x2 fp8, x4 fp4); nominal dense peaks printed beside"}
     for f, d in in_region.items():
         kernels[f"gemm_{FMT_NAME[f]}_in_step"] = {"tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12, "ms_per_step": d["ms"] / args.steps,
                                                    "frac_of_sustained_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f])}
