@@ -60,14 +60,6 @@ __device__ __forceinline__ float tile_scale(float amax, int pow2)
     float s = __fdiv_rn(kMax, amax);
     return fminf(s, FLT_MAX);  // +inf -> FLT_MAX
 }
-// -1/S for the error term.  Paper's rule: amax/FPX_MAX equals 1/S to within one rounding, which the
-// statistics (1e-4) do not see; power-of-two rule: exact.  For an empty tile the value is irrelevant.
-template <int FMT>
-__device__ __forceinline__ float neg_inv_scale(float amax, float s, int pow2)
-{
-    constexpr float kMax = (FMT == SNIP_FMT_FP8_E4M3) ? 448.0f : 6.0f;
-    return pow2 ? -__fdiv_rn(1.0f, s) : -amax * (1.0f / kMax);
-}
 // UE8M0 byte of 1/S for a power-of-two S, replicated into the four bytes of a word
 __device__ __forceinline__ uint32_t sf_word(float s) { return (254u - (__float_as_uint(s) >> 23)) * 0x01010101u; }
 
@@ -98,38 +90,6 @@ __device__ __forceinline__ float2 dec_e2m1x2(uint32_t c)
     asm("{ .reg .b8 t, u; mov.b16 {t, u}, %1; cvt.rn.f16x2.e2m1x2 %0, t; }"
         : "=r"(h2) : "h"((uint16_t)c));
     return __half22float2(*reinterpret_cast<__half2 *>(&h2));
-}
-
-// Quantize 8 consecutive elements (one 128-bit load).  s2[i] / ninv2[i]: scale and negated
-// reciprocal scale of elements (2i, 2i+1).  Returns the packed codes (FP8: 8 bytes in out[0..1];
-// FP4: 4 bytes in out[0]) and adds to the statistics.  The products x*S are IEEE binary32
-// products (packed mul.rn.f32x2), exactly what the scalar definition asks for.
-template <int FMT, bool STATS>
-__device__ __forceinline__ void quant8(const uint4 &v, const float2 (&s2)[4], const float2 (&ninv2)[4],
-                                       uint32_t out[2], float2 &sx2, float2 &se2)
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t c[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float2 x = make_float2(bf16lo(w[i]), bf16hi(w[i]));
-        const float2 t = __fmul2_rn(x, s2[i]);
-        if (FMT == SNIP_FMT_FP8_E4M3) c[i] = cvt_e4m3x2(t.x, t.y);
-        else c[i] = cvt_e2m1x2(t.x, t.y);
-        if (STATS) {
-            const float2 d = (FMT == SNIP_FMT_FP8_E4M3) ? dec_e4m3x2(c[i]) : dec_e2m1x2(c[i]);
-            const float2 e = __ffma2_rn(d, ninv2[i], x);  // x - value(code)/S
-            sx2 = __ffma2_rn(x, x, sx2);
-            se2 = __ffma2_rn(e, e, se2);
-        }
-    }
-    if (FMT == SNIP_FMT_FP8_E4M3) {
-        out[0] = c[0] | (c[1] << 16);
-        out[1] = c[2] | (c[3] << 16);
-    } else {
-        out[0] = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
-        out[1] = 0;
-    }
 }
 
 // ---- stochastic rounding (paper Sec. 6.1: FP4 output gradients) ------------------------------------

@@ -4,12 +4,14 @@
 // code = RNE_fmt(x * S);  and per tensor (Sec. 3.1, Step 1)  sum x^2 and sum (x - code/S)^2.
 // Tile kinds: 1x128 along the columns (ROW), 128x1 along the rows (COL), 128x128 (BLK).
 //
-// Memory-bound design: one CTA owns a 128x128 bf16 tile; each of its 256 threads holds an
-// 8x8 sub-block in registers (eight 128-bit loads in flight per thread), so every element is
-// read from HBM exactly once and the three tile kinds differ only in how the block-amax is
-// reduced (16-lane shuffles for ROW, a small shared-memory exchange for COL, both for BLK).
-// Codes are written with 64/128-bit stores; transposed outputs are staged through an
-// XOR-swizzled shared-memory tile so that the global stores stay fully coalesced.
+// Design: persistent kernels, 256 threads per CTA, several CTAs per SM; a CTA walks over 128x128 bf16 tiles.
+// Every thread fetches its own 8x8 sub-block with eight 16-byte cp.async copies into a private slot of a
+// shared-memory tile and reads it back itself (the only wait is cp.async.wait_group); the next tile's fetch is
+// in flight while this one is encoded, so every element is read from HBM exactly once.  The three tile kinds
+// differ only in how the tile maxima are reduced (16-lane exchange for ROW, a small shared-memory exchange
+// for COL, both for BLK).  Codes as stored leave straight from registers; transposed codes go through
+// byte-permute 8x8 transposes and an XOR-swizzled shared-memory tile so that the global stores stay coalesced.
+// The two-output form (quantize_dual_kernel) encodes each element under two scales in the same pass.
 #include <cuda_bf16.h>
 #include <float.h>
 
