@@ -478,6 +478,10 @@ def run_profile_case(name):
     if name.startswith("layer_stats"):
         return run_layer_stats_case(api, torch, device, parts[2] if len(parts) > 2 else "x")
     mx = parts[1].startswith("mx")
+    if parts[1].startswith("pair"):
+        # the CTA-pair form of the paper-rule GEMM (an alternative kept for comparison; see include/snip.h, snip_debug_set)
+        api.snip_debug_set(api.DEBUG_GEMM_KERNEL, api.GEMM_KERNEL_PAIR)
+        parts[1] = parts[1][4:]
     fmt = {"bf16": FMT_BF16, "fp8": FMT_FP8, "fp4": FMT_FP4, "mxfp8": FMT_FP8, "mxfp4": FMT_FP4}[parts[1]]
     nostats = parts[-1] == "nostats"
     if nostats:
@@ -683,7 +687,7 @@ def main():
     ap.add_argument("--no-kernel-legs", action="store_true")
     ap.add_argument("--profile-case", default=None,
                     help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t|dual_rowcol|dual_blk> "
-                         "or gemm_<fp8|fp4|mxfp8|mxfp4>_<fwd|dgrad|wgrad>[_MxNxK] or layer_stats_<x|w|plain>")
+                         "or gemm_<fp8|fp4|mxfp8|mxfp4|pairfp8|pairfp4>_<fwd|dgrad|wgrad>[_MxNxK] or layer_stats_<x|w|plain>")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
