@@ -6,7 +6,8 @@
 // Structure of one CTA (persistent, one per SM, 384 threads):
 //   warp 0      : TMA producer - streams 128-byte-wide operand tiles into a shared-memory ring
 //   warp 1      : MMA issuer   - one thread issues tcgen05.mma; owns the tensor-memory allocation
-//   warps 2..3  : idle (they only give their registers to the epilogue warps)
+//   warps 2..3  : weight-gradient product: loaders of the per-row / per-column scale factors (one ring of ready
+//                 reciprocals for the CTA); otherwise idle (they only give their registers to the epilogue warps)
 //   warps 4..11 : promotion / epilogue - pull each chunk's partial sums out of tensor memory,
 //                 multiply by 1/(S_a*S_b) of that chunk and add into FP32 register accumulators
 //                 (so the scaling overlaps the next chunk's MMAs, which write the other
@@ -28,7 +29,7 @@ using namespace sm100;
 namespace {
 
 constexpr int BM = 128;
-constexpr int kGemmThreads = 384;  // warps 0-3: producer, MMA issuer, 2 idle; warps 4-11: epilogue
+constexpr int kGemmThreads = 384;  // warps 0-3: producer, MMA issuer, 2 scale loaders (wgrad) or idle; warps 4-11: epilogue
 constexpr int kNumEpiWarps = 8;
 constexpr int kSfCols = 32;  // tensor-memory columns holding constant scale factors (kind::mxf4)
 
@@ -58,15 +59,15 @@ struct Cfg {
     static constexpr int kBBytes = BN * 128;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = (BN >= 256) ? 4 : 5;
-    static constexpr int kScaleDepth = 4;                        // chunks of scale factors in flight per warp
-    static constexpr int kRingB = 256;                           // vector mode: float offset of the per-column B scale slots (after two S_a groups)
-    // a slot holds 32 A scales, 4 block scales and, in vector mode, BN/2 column scales
-    static constexpr int kRingFloatsPerSlot = (SCALE == 2) ? BN / 2 : 64;   // vector mode: one chunk's column scales of a warp
     // block mode (fwd / dgrad) fetches four chunks of scale factors per instruction into two alternating group slots:
     // [4 chunks][32 rows] S_a, then [2 blocks][4 chunks] S_b
     static constexpr int kGroupFloats = 144;
-    static constexpr int kRingFloatsPerWarp = (SCALE == 1) ? 2 * kGroupFloats : kRingB + kScaleDepth * kRingFloatsPerSlot;
-    static constexpr int kSbInvBytes = kNumEpiWarps * kRingFloatsPerWarp * 4;
+    static constexpr int kRingFloatsPerWarp = 2 * kGroupFloats;
+    // vector mode (wgrad): ONE ring for the CTA, filled by the two loader warps: per chunk 128 row factors 1/S_a and BN column
+    // factors 1/S_b, kVecDepth chunks deep, handed over kVecBlock chunks at a time
+    static constexpr int kVecDepth = 16, kVecBlock = 4, kVecAhead = 8;
+    static constexpr int kVecSlotFloats = 128 + BN;
+    static constexpr int kSbInvBytes = (SCALE == 2) ? kVecDepth * kVecSlotFloats * 4 : kNumEpiWarps * kRingFloatsPerWarp * 4;
     // block mode (fwd / dgrad) writes its output through per-warp 2 KB staging tiles and TMA stores
     static constexpr bool kTmaOut = (SCALE == 1);
     static constexpr int kOutStageBytes = kTmaOut ? kNumEpiWarps * 2048 : 0;
@@ -162,7 +163,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * S + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * S + 2 + a); };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 4);
+    constexpr int kVBlocks = C::kVecDepth / C::kVecBlock;
+    auto vfull_bar = [&](int k) { return bar0 + 8u * (2 * S + 4 + k); };              // vector mode: ring block k holds its chunks' factors
+    auto vempty_bar = [&](int k) { return bar0 + 8u * (2 * S + 4 + kVBlocks + k); };  // vector mode: the eight epilogue warps are done with block k
+    static_assert((2 * S + 4 + 2 * kVBlocks) * 8 + 8 <= 256, "barrier area");
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * S + 4 + 2 * kVBlocks);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -174,6 +179,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kNumEpiWarps); }
+        for (int k = 0; k < kVBlocks; ++k) { mbar_init(vfull_bar(k), 2); mbar_init(vempty_bar(k), kNumEpiWarps); }
         *abort_flag = 0u;
         fence_barrier_init();
         prefetch_tensormap(&tmA);
@@ -276,6 +282,72 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
             }
         }
+      } else if (SCALE == SCALE_VEC_B) {
+        // ================= warps 2, 3: scale loaders of the weight-gradient product =================
+        // Both factors of a chunk are vectors here (1/S_a per output row, 1/S_b per output column).  Warp 2 brings the 128
+        // row scales, warp 3 the BN column scales of every chunk into one ring for the CTA (cp.async, kVecAhead chunks
+        // ahead), turns them into reciprocals in place and publishes them kVecBlock chunks at a time, so that the epilogue
+        // warps only read ready factors: no copies, reciprocals or warp barriers of their own on the per-chunk path.
+        const bool rows_side = (warp == 2);
+        const int my_tiles = (int)blockIdx.x < num_tiles ? (num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+        const uint32_t total = (uint32_t)my_tiles * (uint32_t)num_chunks;
+        const uint32_t ring_u32 = smem_u32(scale_ring);
+        int pt = blockIdx.x, pj = 0;   // tile and chunk of the next request
+        uint32_t pc = 0;               // its position in the sequence of this CTA's chunks
+        bool ok = true;
+        const float *src0 = nullptr, *src1 = nullptr;
+        int64_t stride = 0;
+        auto tile_sources = [&]() {
+            int m_idx, n_idx;
+            tile_coords(pt < num_tiles ? pt : (int)blockIdx.x, num_m, num_n, m_idx, n_idx);
+            // rows / columns outside the matrix repeat the last four factors (their sums are never stored)
+            if (rows_side) {
+                src0 = g.sa + min(m_idx * BM + 4 * lane, g.Mo - 4);
+                stride = g.sa_chunk_stride;
+            } else {
+                src0 = g.sb + min(n_idx * BN + 4 * lane, g.No - 4);
+                src1 = g.sb + min(n_idx * BN + 128 + 4 * lane, g.No - 4);
+                stride = g.sb_chunk_stride;
+            }
+        };
+        tile_sources();
+        auto request = [&]() {
+            if (pc < total && ok) {
+                const uint32_t d = pc % C::kVecDepth;
+                if ((pc % C::kVecBlock) == 0 && !__all_sync(0xFFFFFFFFu, mbar_wait(vempty_bar(d / C::kVecBlock), ((pc / C::kVecDepth) & 1u) ^ 1u, abort_flag, g.wait_limit_ns))) ok = false;
+                else {
+                    const uint32_t slot = ring_u32 + d * (C::kVecSlotFloats * 4);
+                    if (rows_side) {
+                        cp_async_16(slot + 16u * lane, src0);
+                    } else {
+                        cp_async_16(slot + 512u + 16u * lane, src0);
+                        if (128 + 4 * lane < BN) cp_async_16(slot + 1024u + 16u * lane, src1);
+                    }
+                    src0 += stride;
+                    src1 += stride;
+                    if (++pj == num_chunks) { pj = 0; pt += gridDim.x; tile_sources(); }
+                }
+            }
+            ++pc;
+            cp_async_commit();   // one group per position, empty past the end, so that the wait below stays uniform
+        };
+        for (int i = 0; i < C::kVecAhead; ++i) request();
+        for (uint32_t cc = 0; cc < total && ok; ++cc) {
+            request();                       // position cc + kVecAhead
+            cp_async_wait<C::kVecAhead>();   // this lane's copies of position cc have landed
+            const uint32_t d = cc % C::kVecDepth;
+            float4 *mine = reinterpret_cast<float4 *>(scale_ring + d * C::kVecSlotFloats + (rows_side ? 0 : 128) + 4 * lane);
+            const float4 v = mine[0];
+            mine[0] = make_float4(rcp_approx(v.x), rcp_approx(v.y), rcp_approx(v.z), rcp_approx(v.w));
+            if (!rows_side && 128 + 4 * lane < BN) {
+                const float4 w = mine[32];
+                mine[32] = make_float4(rcp_approx(w.x), rcp_approx(w.y), rcp_approx(w.z), rcp_approx(w.w));
+            }
+            __syncwarp();
+            // a block is published when its last slot (or the last chunk of all) is ready
+            if (lane == 0 && ((cc % C::kVecBlock) == C::kVecBlock - 1 || cc + 1 == total)) mbar_arrive(vfull_bar(d / C::kVecBlock));
+        }
+        cp_async_wait<0>();
       }
     } else {
         reg_alloc<232>();    // needs (232-168)*256 = 16384 <= 16384 (an unsatisfiable request would block forever)
@@ -283,11 +355,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int e = warp - 4;          // 0..7
         const int q = warp & 3;          // tensor-memory lane quarter this warp may access
         const int h = e >> 2;            // column half
-        // Per-warp scale-factor buffers, filled ahead with cp.async so that no global-memory latency sits
-        // between two chunks.  S_a of this warp's 32 rows comes four chunks at a time into two alternating
-        // group slots [4 chunks][32 rows]; block mode keeps the S_b of its one or two 128-column blocks next
-        // to them ([2 blocks][4 chunks] at float 128 of the group), vector mode keeps kScaleDepth per-chunk
-        // slots of HALF column scales from float kRingB on.
+        // Block mode: per-warp scale-factor buffers, filled ahead with cp.async so that no global-memory latency
+        // sits between two chunks.  S_a of this warp's 32 rows comes four chunks at a time into two alternating
+        // group slots [4 chunks][32 rows], with the S_b of its one or two 128-column blocks next to them
+        // ([2 blocks][4 chunks] at float 128 of the group).  Vector mode reads the CTA's ring of ready factors.
         float *ring = scale_ring + e * C::kRingFloatsPerWarp;
         const uint32_t ring_u32 = smem_u32(ring);
         const uint32_t stage_u32 = out_stage0 + e * 2048;   // this warp's staging tile: 32 rows x 64 bytes
@@ -303,22 +374,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const int nacc = (KIND == MmaKind::F16) ? 1 : num_chunks;
             const int blk0 = col0 >> 7;
             const int blk_last = (g.No - 1) >> 7;
-
-            // Vector mode (wgrad): chunk cn's column scales (one 16-byte copy per lane) and, with every fourth chunk,
-            // the S_a of four chunks (as in block mode, see below) travel in one commit group.
-            auto prefetch_scales = [&](int cn) {
-                if (SCALE == SCALE_VEC_B && cn < nacc) {
-                    const uint32_t slot = ring_u32 + (C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot) * 4;
-                    const int n = col0 + 4 * lane;
-                    if (4 * lane < HALF && n < g.No) cp_async_16(slot + 4 * lane * 4, g.sb + (int64_t)cn * g.sb_chunk_stride + n);
-                    if ((cn & 3) == 0) {
-                        const uint32_t grp = ring_u32 + ((cn >> 2) & 1) * 128 * 4;
-                        const int ci = lane >> 3, r4 = (lane & 7) * 4, chunk = cn + ci;
-                        if (row0 < g.Mo && chunk < nacc) cp_async_16(grp + (ci * 32 + r4) * 4, g.sa + (int64_t)chunk * g.sa_chunk_stride + row0 + r4);
-                    }
-                }
-                cp_async_commit();
-            };
 
             // Block mode: the scale factors of four consecutive chunks with two instructions per warp.  Lane L
             // fetches 16 bytes = S_a of rows 4*(L%8) .. +3 of chunk 4*gn + L/8 (the warp's 32 rows lie inside or
@@ -343,15 +398,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (SCALE != SCALE_NONE) {
 #pragma unroll
                 for (int i = 0; i < HALF / 2; ++i) acc[i] = make_float2(0.0f, 0.0f);
-                // out-of-range rows / columns read 1.0 (their products are zero anyway)
-                for (int i = lane; i < C::kRingFloatsPerWarp; i += 32) ring[i] = 1.0f;
-                __syncwarp();
                 if (SCALE == SCALE_BLOCK_B) {
+                    // out-of-range rows / columns read 1.0 (their products are zero anyway)
+                    for (int i = lane; i < C::kRingFloatsPerWarp; i += 32) ring[i] = 1.0f;
+                    __syncwarp();
                     prefetch_group(0);
                     prefetch_group(1);
-                } else {
-#pragma unroll
-                    for (int d = 0; d < C::kScaleDepth; ++d) prefetch_scales(d);
                 }
             }
             // Block mode: the reciprocal factors 1/(S_a*S_b) of the four chunks of group gn, from its slot (which must
@@ -368,41 +420,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     if (kBlocksPerWarp == 2) fq[1][j] = rcp_approx(sa * sl[132 + j]);
                 }
             };
-            // Vector mode: 1/S_a of chunk cn from its group slot (the group landed with an earlier chunk).
-            auto prepare_factors = [&](int cn, float (&fo)[G]) {
-                fo[0] = rcp_approx(ring[((cn >> 2) & 1) * 128 + (cn & 3) * 32 + lane]);
-            };
-            // Vector mode: turns chunk cn's column scales into reciprocals in place (4 per lane).  Done two chunks
-            // ahead of their use, at the end of an iteration, so that the load - reciprocal - store chain never
-            // sits in front of FMAs.
-            auto convert_columns = [&](int cn) {
-                if (4 * lane < HALF) {
-                    float4 *p4 = reinterpret_cast<float4 *>(ring + C::kRingB + (cn % C::kScaleDepth) * C::kRingFloatsPerSlot + 4 * lane);
-                    const float4 s4 = *p4;
-                    *p4 = make_float4(rcp_approx(s4.x), rcp_approx(s4.y), rcp_approx(s4.z), rcp_approx(s4.w));
-                }
-                __syncwarp();
-            };
-            float f_next[G];
             if (SCALE == SCALE_BLOCK_B) {
                 cp_async_wait<1>();   // group 0
                 __syncwarp();
                 load_factors(0);
-            } else if (SCALE == SCALE_VEC_B) {
-                cp_async_wait<C::kScaleDepth - 2>();   // chunks 0 and 1
-                __syncwarp();
-                convert_columns(0);
-                convert_columns(1);
-                prepare_factors(0, f_next);
             }
             for (int c = 0; c < nacc; ++c, ++cc) {
                 const uint32_t a = cc & 1u;
                 float f[G];
-                const float *slot = ring + C::kRingB + (c % C::kScaleDepth) * C::kRingFloatsPerSlot;   // vector mode: this chunk's column reciprocals
+                // vector mode: this chunk's slot of the CTA's factor ring (filled by warps 2 and 3), taken over a block at a time
+                const uint32_t vd = cc % C::kVecDepth;
+                const float *vslot = scale_ring + vd * C::kVecSlotFloats;
+                const float *slot = vslot + 128 + h * HALF;   // this warp's column reciprocals
+                if (SCALE == SCALE_VEC_B && (cc % C::kVecBlock) == 0) {
+                    const bool got = mbar_wait(vfull_bar(vd / C::kVecBlock), (cc / C::kVecDepth) & 1u, abort_flag, g.wait_limit_ns);
+                    if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
+                }
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) {
                     if (SCALE == SCALE_BLOCK_B) f[gi] = (kBlocksPerWarp == 1 || ((col0 + 32 * gi) >> 7) == blk0) ? fq[0][0] : fq[kBlocksPerWarp - 1][0];
-                    else f[gi] = f_next[gi];
+                    else f[gi] = vslot[q * 32 + lane];
                 }
                 if (SCALE == SCALE_BLOCK_B) {
 #pragma unroll
@@ -433,8 +470,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             load_factors((c >> 2) + 1);
                             prefetch_group((c >> 2) + 2);
                         }
-                    } else {
-                        prepare_factors(c + 1, f_next);   // vector mode: 1/S_a only
                     }
                 }
                 // all of this warp's reads of buffer `a` are done: hand it back to the MMA warp
@@ -485,11 +520,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         }
                     }
                 }
-                if (SCALE == SCALE_VEC_B) {
-                    cp_async_wait<1>();                  // chunk c+2 has landed (c+3 may be in flight)
-                    __syncwarp();                        // ... for every lane, and every lane has read slot c
-                    convert_columns(c + 2);
-                    prefetch_scales(c + C::kScaleDepth); // refill slot c for a later chunk
+                if (SCALE == SCALE_VEC_B && (cc % C::kVecBlock) == C::kVecBlock - 1) {
+                    __syncwarp();                        // every lane has read the block's slots
+                    if (lane == 0) mbar_arrive(vempty_bar(vd / C::kVecBlock));
                 }
             }
             if (SCALE != SCALE_NONE) {
