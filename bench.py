@@ -213,7 +213,8 @@ class Step:
         self.scales = [torch.empty(sb // 4, dtype=torch.float32, device=dev) for _ in range(nbuf)]
         self.qws = torch.empty(2 * wb, dtype=torch.uint8, device=dev)
         self.sf = [torch.empty(cb // 32 + 4096, dtype=torch.uint8, device=dev) for _ in range(nbuf)]   # UE8M0 atoms (power-of-two option)
-        self.gws = torch.zeros(1024, dtype=torch.uint8, device=dev)
+        # GEMM workspace: the size the library reports for a weight-gradient product (room for its contraction slices)
+        self.gws = torch.zeros(max(1024, api.snip_workspace_size(api.OP_WGRAD, 16384, 4096, 4096, api.FMT_FP8_E4M3, api.FMT_FP8_E4M3)[0]), dtype=torch.uint8, device=dev)
 
     def run_decomposed(self, events=None, mx=False, qevents=None):
         api, torch = self.api, self.torch
@@ -367,7 +368,7 @@ class KernelTimer:
             qa = quant(A, fmt, api.BLOCK_COL, api.Q_TRANSPOSED); qb = quant(B, fmt, api.BLOCK_COL, api.Q_TRANSPOSED)
             a = api.make_qtensor(qa[0], qa[1], M, N, fmt, api.BLOCK_COL, True); b = api.make_qtensor(qb[0], qb[1], M, K, fmt, api.BLOCK_COL, True)
         out = torch.empty(out_shape, dtype=torch.bfloat16, device=self.device)
-        ws = torch.zeros(1024, dtype=torch.uint8, device=self.device)
+        ws = torch.zeros(max(1024, api.snip_workspace_size(op, M, N, K, fmt, fmt)[0]), dtype=torch.uint8, device=self.device)
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.device)
         times = []
         for i in range(warmup + iters):

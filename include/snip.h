@@ -250,7 +250,11 @@ int snip_quantize_mx(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
 
 /*
  * Workspace bytes for one GEMM call of the given op and shape, and for the snip_linear_* call
- * of the same op (which also holds the quantized operands).  Host-only.
+ * of the same op (which also holds the quantized operands).  Host-only.  For SNIP_OP_WGRAD over
+ * quantized operands gemm_bytes includes room (about 21 MB) that lets the kernel cut the tiles of
+ * its last, partly filled wave over the SMs into slices of the contraction (their FP32 sums are
+ * added in slice order, so results do not depend on timing); any GEMM also runs, unsliced, with
+ * the 256-byte minimum.
  */
 int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int fmt_b,
                         size_t *gemm_bytes_host, size_t *linear_bytes_host);
@@ -269,8 +273,8 @@ int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int 
  * to bf16 or stored as FP32.  accumulate != 0 adds to the existing contents of out (FP32 output
  * only).  Operand formats: (BF16,BF16), (FP8,FP8), (FP4,FP4), (FP8,FP4), (FP4,FP8); pairs
  * that mix BF16 with a quantized operand return SNIP_ERR_UNSUPPORTED.
- * ws must hold at least gemm_bytes of snip_workspace_size; its first word is the device status
- * word read by snip_poll_status.  The call itself zeroes that word on the stream before the
+ * ws must hold at least 256 bytes (gemm_bytes of snip_workspace_size to allow slicing, see there);
+ * its first word is the device status word read by snip_poll_status.  The call itself zeroes that word on the stream before the
  * kernel starts (a 4-byte memset node), so the workspace needs no initialisation by the caller.
  */
 int snip_gemm_quantized(int op, const snip_qtensor_t *a_host, const snip_qtensor_t *b_host,
@@ -424,11 +428,14 @@ int snip_select_scheme(int m, int n, const double *q, const int64_t *w, int64_t 
  *   SNIP_DEBUG_GEMM_KERNEL   : 0 or 1 = the single-CTA kernels (the default), 2 = the CTA-pair
  *                              kernels for every quantized GEMM (an alternative form of the same
  *                              product, kept for A/B comparisons in the benchmark).
+ *   SNIP_DEBUG_GEMM_SLICING  : 1 (default) = the weight-gradient product may slice its last wave
+ *                              when its workspace has room (snip_workspace_size), 0 = never.
  * Returns SNIP_ERR_ARG for an unknown key or a value out of range.
  */
 #define SNIP_DEBUG_WAIT_LIMIT_NS 0
 #define SNIP_DEBUG_TX_SKEW_BYTES 1
 #define SNIP_DEBUG_GEMM_KERNEL   2
+#define SNIP_DEBUG_GEMM_SLICING  3
 int snip_debug_set(int key, long long value);
 
 /*

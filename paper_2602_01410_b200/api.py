@@ -51,7 +51,7 @@ class QOut(ctypes.Structure):
 
 DUAL_ROW_COLT, DUAL_BLK_BLKT = 0, 1
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
-DEBUG_WAIT_LIMIT_NS, DEBUG_TX_SKEW_BYTES, DEBUG_GEMM_KERNEL = 0, 1, 2
+DEBUG_WAIT_LIMIT_NS, DEBUG_TX_SKEW_BYTES, DEBUG_GEMM_KERNEL, DEBUG_GEMM_SLICING = 0, 1, 2, 3
 GEMM_KERNEL_AUTO, GEMM_KERNEL_SINGLE, GEMM_KERNEL_PAIR = 0, 1, 2
 
 

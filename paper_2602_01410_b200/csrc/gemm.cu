@@ -31,6 +31,10 @@ namespace {
 constexpr int BM = 128;
 constexpr int kGemmThreads = 384;  // warps 0-3: producer, MMA issuer, 2 scale loaders (wgrad) or idle; warps 4-11: epilogue
 constexpr int kNumEpiWarps = 8;
+// Slicing of the weight-gradient product's last wave (see launch_gemm)
+constexpr int kMaxSlices = 4, kMinSliceStages = 8, kMaxSlicedItems = 160;
+constexpr size_t kSliceCountersOffset = 256, kSliceCountersBytes = 8192;   // counters: [sliced tile][epilogue warp], 32 bits each
+static_assert((size_t)kMaxSlicedItems / 2 * kNumEpiWarps * 4 <= kSliceCountersBytes, "counter area");
 constexpr int kSfCols = 32;  // tensor-memory columns holding constant scale factors (kind::mxf4)
 
 enum ScaleMode { SCALE_NONE = 0, SCALE_BLOCK_B = 1, SCALE_VEC_B = 2 };
@@ -48,7 +52,35 @@ struct GemmArgs {
     uint32_t stage_tx_bytes;   // bytes the two TMA loads of one stage report to the barrier
     uint64_t wait_limit_ns;    // bound of every device-side wait
     uint32_t *status;
+    // Work items: item w < split_first is tile w over the whole contraction; the tiles from split_first on (the last,
+    // partial wave of a persistent grid) are cut into nsplit contraction slices each, item split_first + r * nsplit + j
+    // being slice j of tile split_first + r.  nsplit == 1: no slicing, num_items == number of tiles.
+    int32_t split_first, nsplit, num_items;
+    float *partials;           // [tail tile r][slice j][epilogue warp][column quad][row lane][4]: FP32 sums of a slice
+    uint32_t *counters;        // [tail tile r][epilogue warp]: slices that have delivered their sums (zero at launch)
 };
+
+struct WorkItem {
+    int t, ks0, ks1;       // tile, stage range of the contraction
+    int tail, slice, nsl;  // index of a sliced tile among the sliced tiles, slice, number of slices (1: whole tile)
+};
+template <bool SLICED>   // false: every item is a whole tile (known at compile time)
+__device__ __forceinline__ WorkItem work_item(const GemmArgs &g, int w, int num_kstages)
+{
+    WorkItem wi;
+    if (!SLICED || w < g.split_first) {
+        wi.t = w; wi.ks0 = 0; wi.ks1 = num_kstages; wi.tail = 0; wi.slice = 0; wi.nsl = 1;
+    } else {
+        const int i = w - g.split_first;
+        wi.tail = i / g.nsplit;
+        wi.slice = i - wi.tail * g.nsplit;
+        wi.nsl = g.nsplit;
+        wi.t = g.split_first + wi.tail;
+        wi.ks0 = (int)((int64_t)wi.slice * num_kstages / g.nsplit);
+        wi.ks1 = (int)((int64_t)(wi.slice + 1) * num_kstages / g.nsplit);
+    }
+    return wi;
+}
 
 template <MmaKind KIND, int BN, int SCALE>
 struct Cfg {
@@ -172,7 +204,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_m = (g.Mo + BM - 1) / BM, num_n = (g.No + BN - 1) / BN;
-    const int num_tiles = num_m * num_n;
     const int num_chunks = (g.Kc + C::kChunkElems - 1) / C::kChunkElems;
     const int num_kstages = (g.Kc + C::kStageK - 1) / C::kStageK;
 
@@ -213,10 +244,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            for (int w = blockIdx.x; w < g.num_items && ok; w += gridDim.x) {
+                const WorkItem wi = work_item<SCALE == SCALE_VEC_B>(g, w, num_kstages);
                 int m_idx, n_idx;
-                tile_coords(t, num_m, num_n, m_idx, n_idx);
-                for (int ks = 0; ks < num_kstages; ++ks, ++it) {
+                tile_coords(wi.t, num_m, num_n, m_idx, n_idx);
+                for (int ks = wi.ks0; ks < wi.ks1; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
@@ -232,8 +264,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             uint32_t it = 0, cc = 0;
             bool ok = true;
             const uint32_t sfa = tmem_base + C::kSfCol0, sfb = tmem_base + C::kSfCol0 + 16;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-                for (int ks = 0; ks < num_kstages && ok; ++ks, ++it) {
+            for (int w = blockIdx.x; w < g.num_items && ok; w += gridDim.x) {
+                const WorkItem wi = work_item<SCALE == SCALE_VEC_B>(g, w, num_kstages);
+                for (int ks = wi.ks0; ks < wi.ks1 && ok; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag, g.wait_limit_ns)) { ok = false; break; }
@@ -242,15 +275,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const uint64_t bdesc = make_smem_desc_k128(smem_b0 + s * C::kBBytes);
                     if (KIND == MmaKind::F16) {
                         const uint32_t a = cc & 1u;
-                        if (ks == 0) {
+                        if (ks == wi.ks0) {
                             if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
                             tc_fence_after_sync();
                         }
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            mma_ss<KIND, false>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (ks > 0 || k > 0) ? 1u : 0u, 0, 0);
+                            mma_ss<KIND, false>(tmem_base + a * BN, adesc + 2 * k, bdesc + 2 * k, idesc, (ks > wi.ks0 || k > 0) ? 1u : 0u, 0, 0);
                         tc_commit<false>(empty_bar(s));
-                        if (ks == num_kstages - 1) { tc_commit<false>(tfull_bar(a)); ++cc; }
+                        if (ks == wi.ks1 - 1) { tc_commit<false>(tfull_bar(a)); ++cc; }
                     } else if (KIND == MmaKind::F8F6F4) {
                         const uint32_t a = cc & 1u;
                         if (!mbar_wait(tempty_bar(a), ((cc >> 1) & 1u) ^ 1u, abort_flag, g.wait_limit_ns)) { ok = false; break; }
@@ -289,28 +322,35 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // ahead), turns them into reciprocals in place and publishes them kVecBlock chunks at a time, so that the epilogue
         // warps only read ready factors: no copies, reciprocals or warp barriers of their own on the per-chunk path.
         const bool rows_side = (warp == 2);
-        const int my_tiles = (int)blockIdx.x < num_tiles ? (num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-        const uint32_t total = (uint32_t)my_tiles * (uint32_t)num_chunks;
+        constexpr int kChunksPerStage = C::kStageK / C::kChunkElems;
+        uint32_t total = 0;            // chunks of all of this CTA's work items
+        for (int w = blockIdx.x; w < g.num_items; w += gridDim.x) {
+            const WorkItem wi = work_item<SCALE == SCALE_VEC_B>(g, w, num_kstages);
+            total += (uint32_t)(min(kChunksPerStage * wi.ks1, num_chunks) - kChunksPerStage * wi.ks0);
+        }
         const uint32_t ring_u32 = smem_u32(scale_ring);
-        int pt = blockIdx.x, pj = 0;   // tile and chunk of the next request
+        int pw = blockIdx.x, pj = 0, pn = 0;   // work item and chunk of the next request, chunks of that item
         uint32_t pc = 0;               // its position in the sequence of this CTA's chunks
         bool ok = true;
         const float *src0 = nullptr, *src1 = nullptr;
         int64_t stride = 0;
-        auto tile_sources = [&]() {
+        auto item_sources = [&]() {
+            const WorkItem wi = work_item<SCALE == SCALE_VEC_B>(g, pw < g.num_items ? pw : (int)blockIdx.x, num_kstages);
             int m_idx, n_idx;
-            tile_coords(pt < num_tiles ? pt : (int)blockIdx.x, num_m, num_n, m_idx, n_idx);
+            tile_coords(wi.t, num_m, num_n, m_idx, n_idx);
+            const int c0 = kChunksPerStage * wi.ks0;
+            pn = min(kChunksPerStage * wi.ks1, num_chunks) - c0;
             // rows / columns outside the matrix repeat the last four factors (their sums are never stored)
             if (rows_side) {
-                src0 = g.sa + min(m_idx * BM + 4 * lane, g.Mo - 4);
                 stride = g.sa_chunk_stride;
+                src0 = g.sa + c0 * stride + min(m_idx * BM + 4 * lane, g.Mo - 4);
             } else {
-                src0 = g.sb + min(n_idx * BN + 4 * lane, g.No - 4);
-                src1 = g.sb + min(n_idx * BN + 128 + 4 * lane, g.No - 4);
                 stride = g.sb_chunk_stride;
+                src0 = g.sb + c0 * stride + min(n_idx * BN + 4 * lane, g.No - 4);
+                src1 = g.sb + c0 * stride + min(n_idx * BN + 128 + 4 * lane, g.No - 4);
             }
         };
-        tile_sources();
+        item_sources();
         auto request = [&]() {
             if (pc < total && ok) {
                 const uint32_t d = pc % C::kVecDepth;
@@ -325,7 +365,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                     src0 += stride;
                     src1 += stride;
-                    if (++pj == num_chunks) { pj = 0; pt += gridDim.x; tile_sources(); }
+                    if (++pj == pn) { pj = 0; pw += gridDim.x; item_sources(); }
                 }
             }
             ++pc;
@@ -364,14 +404,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const uint32_t stage_u32 = out_stage0 + e * 2048;   // this warp's staging tile: 32 rows x 64 bytes
         uint32_t cc = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        for (int w = blockIdx.x; w < g.num_items && ok; w += gridDim.x) {
+            const WorkItem wi = work_item<SCALE == SCALE_VEC_B>(g, w, num_kstages);
             int m_idx, n_idx;
-            tile_coords(t, num_m, num_n, m_idx, n_idx);
+            tile_coords(wi.t, num_m, num_n, m_idx, n_idx);
             const int row0 = m_idx * BM + q * 32;
             const int row = row0 + lane;
             const int col0 = n_idx * BN + h * HALF;
             const bool row_ok = row < g.Mo;
-            const int nacc = (KIND == MmaKind::F16) ? 1 : num_chunks;
+            constexpr int kChunksPerStage = C::kStageK / C::kChunkElems;
+            const int nacc = (KIND == MmaKind::F16) ? 1 : min(kChunksPerStage * wi.ks1, num_chunks) - kChunksPerStage * wi.ks0;
             const int blk0 = col0 >> 7;
             const int blk_last = (g.No - 1) >> 7;
 
@@ -551,9 +593,42 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             const int col = col0 + b * kPerBox;
                             if (lane == 0 && col < g.No && row0 < g.Mo) { tma_store_2d(&tmO, stage_u32, col, row0); bulk_commit(); }
                         }
-                    } else if (row_ok) {
+                    } else {
+                        bool write_out = true;
+                        if (SCALE == SCALE_VEC_B && wi.nsl > 1) {
+                            // A slice of a sliced tile: this warp's 32 x HALF sums go to the slice's slot (512 contiguous bytes
+                            // per store instruction); the warp that delivers a sub-tile's last slice adds all slices in slice
+                            // order, whoever came last, so the result does not depend on the order of arrival.
+                            float *av = reinterpret_cast<float *>(acc);
+                            constexpr size_t kWarpFloats = 32 * HALF;
+                            float *first = g.partials + (size_t)(wi.tail * wi.nsl) * kNumEpiWarps * kWarpFloats + e * kWarpFloats + lane * 4;
+                            float *mine = first + (size_t)wi.slice * kNumEpiWarps * kWarpFloats;
 #pragma unroll
-                        for (int gi = 0; gi < HALF / 32; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, reinterpret_cast<const float *>(acc) + 32 * gi);
+                            for (int j4 = 0; j4 < HALF / 4; ++j4)
+                                __stcg(reinterpret_cast<float4 *>(mine + j4 * 128), make_float4(av[4 * j4], av[4 * j4 + 1], av[4 * j4 + 2], av[4 * j4 + 3]));
+                            __threadfence();
+                            __syncwarp();
+                            uint32_t old = 0;
+                            if (lane == 0) old = atomicAdd(g.counters + wi.tail * kNumEpiWarps + e, 1u);
+                            old = __shfl_sync(0xFFFFFFFFu, old, 0);
+                            write_out = (old == (uint32_t)wi.nsl - 1u);
+                            if (write_out) {
+                                __threadfence();
+#pragma unroll
+                                for (int j4 = 0; j4 < HALF / 4; ++j4) {
+                                    float4 v = __ldcg(reinterpret_cast<const float4 *>(first + j4 * 128));
+                                    for (int sl = 1; sl < wi.nsl; ++sl) {
+                                        const float4 u = __ldcg(reinterpret_cast<const float4 *>(first + (size_t)sl * kNumEpiWarps * kWarpFloats + j4 * 128));
+                                        v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+                                    }
+                                    av[4 * j4] = v.x; av[4 * j4 + 1] = v.y; av[4 * j4 + 2] = v.z; av[4 * j4 + 3] = v.w;
+                                }
+                            }
+                        }
+                        if (write_out && row_ok) {
+#pragma unroll
+                            for (int gi = 0; gi < HALF / 32; ++gi) store32<OUT_F32>(g, row, col0 + 32 * gi, reinterpret_cast<const float *>(acc) + 32 * gi);
+                        }
                     }
                 }
                 __syncwarp();
@@ -658,8 +733,24 @@ int launch_gemm(const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMa
     // a per-function, per-device attribute; setting it on every launch is cheap and correct on any device
     SNIP_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
     const int num_tiles = (int)(ceil_div(g.Mo, BM) * ceil_div(g.No, BN));
-    const int grid = num_tiles < sm_count() ? num_tiles : sm_count();
-    kern<<<grid, kGemmThreads, C::kSmemBytes, st>>>(tmA, tmB, tmO, g, idesc);
+    const int sms = sm_count();
+    GemmArgs ga = g;
+    ga.split_first = num_tiles; ga.nsplit = 1; ga.num_items = num_tiles;
+    if (SCALE == SCALE_VEC_B && g.partials && sms > 0) {
+        // The tiles of the last, partial wave (all tiles, if there are fewer than SMs) are cut along the contraction into as
+        // many slices as there are SMs to take them: at most kMaxSlices, none shorter than kMinSliceStages stages.
+        const int full = (num_tiles / sms) * sms, rest = num_tiles - full;
+        const int num_kstages = (int)ceil_div(g.Kc, C::kStageK);
+        int ns = rest > 0 ? sms / rest : 1;
+        if (ns > kMaxSlices) ns = kMaxSlices;
+        while (ns > 1 && (num_kstages / ns < kMinSliceStages || rest * ns > kMaxSlicedItems)) --ns;
+        if (ns > 1) {
+            ga.split_first = full; ga.nsplit = ns; ga.num_items = full + rest * ns;
+            SNIP_CUDA_TRY(cudaMemsetAsync(g.counters, 0, (size_t)rest * kNumEpiWarps * sizeof(uint32_t), st));
+        }
+    }
+    const int grid = ga.num_items < sms ? ga.num_items : sms;
+    kern<<<grid, kGemmThreads, C::kSmemBytes, st>>>(tmA, tmB, tmO, ga, idesc);
     SNIP_CUDA_TRY(cudaGetLastError());
     return SNIP_OK;
 }
@@ -678,11 +769,15 @@ int launch_gemm_scale(int scale, bool out_f32, const CUtensorMap &tmA, const CUt
 }  // namespace
 
 size_t gemm_ws_bytes() { return 256; }
+// Workspace with which the weight-gradient product may slice the tiles of its last wave along the contraction:
+// status word, arrival counters, one FP32 tile per slice.
+size_t gemm_ws_bytes_sliced() { return kSliceCountersOffset + kSliceCountersBytes + (size_t)kMaxSlicedItems * BM * 256 * sizeof(float); }
 
 // Testing hooks (snip_debug_set): process-wide, off by default.
 namespace {
 std::atomic<long long> g_wait_limit_ns{2000000000ll};   // bound of every device-side wait of the GEMM kernels
 std::atomic<int> g_tx_skew{0};                           // bytes added to what a stage's barrier expects (a wait that cannot complete)
+std::atomic<int> g_slicing{1};                           // 0: the weight-gradient product never slices its last wave
 std::atomic<int> g_kernel_choice{0};                     // 0, 1 = single-CTA kernels, 2 = CTA-pair kernels for quantized operands
 }  // namespace
 
@@ -742,6 +837,12 @@ int gemm_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, in
     g.sb = sb; g.sb_chunk_stride = sb_chunk_stride; g.sb_blk_stride = sb_blk_stride;
     g.out = out; g.ldo = No; g.accumulate = accumulate;
     g.status = static_cast<uint32_t *>(ws);
+    g.split_first = 0; g.nsplit = 1; g.num_items = 0;   // set per launch
+    g.partials = nullptr; g.counters = nullptr;
+    if (!a16 && scale_mode == SCALE_VEC_B && ws_bytes >= gemm_ws_bytes_sliced() && g_slicing.load()) {
+        g.counters = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(ws) + kSliceCountersOffset);
+        g.partials = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + kSliceCountersOffset + kSliceCountersBytes);
+    }
     g.stage_tx_bytes = 0;
     g.wait_limit_ns = (uint64_t)g_wait_limit_ns.load();
     const int tx_skew = g_tx_skew.load();
@@ -853,6 +954,7 @@ extern "C" int snip_debug_set(int key, long long value)
         case SNIP_DEBUG_WAIT_LIMIT_NS: if (value <= 0) return SNIP_ERR_ARG; g_wait_limit_ns.store(value); return SNIP_OK;
         case SNIP_DEBUG_TX_SKEW_BYTES: if (value < 0 || value > 4096 || (value % 16) != 0) return SNIP_ERR_ARG; g_tx_skew.store((int)value); return SNIP_OK;
         case SNIP_DEBUG_GEMM_KERNEL: if (value < 0 || value > 2) return SNIP_ERR_ARG; g_kernel_choice.store((int)value); return SNIP_OK;
+        case SNIP_DEBUG_GEMM_SLICING: if (value < 0 || value > 1) return SNIP_ERR_ARG; g_slicing.store((int)value); return SNIP_OK;
         default: return SNIP_ERR_ARG;
     }
 }

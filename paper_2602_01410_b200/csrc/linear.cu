@@ -17,6 +17,7 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
                  int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status);
 int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st);
 size_t gemm_ws_bytes();
+size_t gemm_ws_bytes_sliced();   // with room for the weight-gradient product's contraction slices
 int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bool blk, int pow2, const DualOut &oa, const DualOut &ob,
                        void *ws, size_t ws_bytes, cudaStream_t st);
 
@@ -84,7 +85,7 @@ size_t linear_ws_bytes(int op, int64_t M, int64_t N, int64_t K, int fmt_a, int f
 {
     const LinearPlan p = plan_for(op, M, N, K);
     Carve c(nullptr, 0);
-    c.take(gemm_ws_bytes());
+    c.take(gemm_ws_bytes_sliced());
     const bool need_a = fmt_a != SNIP_FMT_BF16 || p.tr_a, need_b = fmt_b != SNIP_FMT_BF16 || p.tr_b;
     if (need_a) { c.take(code_bytes(fmt_a, p.rows_a, p.cols_a)); c.take(scale_bytes(p.block_a, p.rows_a, p.cols_a)); }
     if (need_b) { c.take(code_bytes(fmt_b, p.rows_b, p.cols_b)); c.take(scale_bytes(p.block_b, p.rows_b, p.cols_b)); }
@@ -106,7 +107,7 @@ int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int6
     if (!aligned16(ws)) return SNIP_ERR_ALIGN;
     const LinearPlan p = plan_for(op, M, N, K);
     Carve c(ws, ws_bytes);
-    void *gws = c.take(gemm_ws_bytes());
+    void *gws = c.take(gemm_ws_bytes_sliced());
     const bool q = fmt_a != SNIP_FMT_BF16;
     const bool need_a = q || p.tr_a, need_b = q || p.tr_b;
     void *codes_a = nullptr, *codes_b = nullptr;
@@ -141,7 +142,7 @@ int linear_impl(int op, const void *A, const void *B, void *out, int64_t M, int6
     else if (op == SNIP_OP_DGRAD) { sb_bs = 1; sb_cs = ceil_div(K, 128); }
     else { sb_bs = 0; sb_cs = p.No; }
     return gemm_impl(fmt_a, fmt_b, ga, gb, p.Mo, p.No, p.Kc, scales_a, sa_cs, scales_b, sb_cs, sb_bs, q ? p.scale_mode : SCALE_NONE, out,
-                     out_dtype, accumulate, gws, gemm_ws_bytes(), st, true);
+                     out_dtype, accumulate, gws, gemm_ws_bytes_sliced(), st, true);
 }
 
 
@@ -167,7 +168,7 @@ FwdBwdCarve carve_fwd_bwd(void *ws, int64_t M, int64_t N, int64_t K, const int (
                           SNIP_BLOCK_COL_128x1};
     FwdBwdCarve f{};
     Carve c(ws, 0);
-    f.gws = c.take(gemm_ws_bytes());
+    f.gws = c.take(gemm_ws_bytes_sliced());
     for (int i = 0; i < 6; ++i) {
         f.codes[i] = c.take(code_bytes(fmt[i], rows[i], cols[i]));
         f.scales[i] = static_cast<float *>(c.take(scale_bytes(block[i], rows[i], cols[i])));
@@ -192,7 +193,7 @@ extern "C" int snip_workspace_size(int op, int64_t M, int64_t N, int64_t K, int 
     using namespace snip;
     if (op < SNIP_OP_FWD || op > SNIP_OP_WGRAD || !valid_fmt(fmt_a) || !valid_fmt(fmt_b)) return SNIP_ERR_ARG;
     if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
-    if (gemm_bytes) *gemm_bytes = gemm_ws_bytes();
+    if (gemm_bytes) *gemm_bytes = (op == SNIP_OP_WGRAD && fmt_a != SNIP_FMT_BF16 && fmt_b != SNIP_FMT_BF16) ? gemm_ws_bytes_sliced() : gemm_ws_bytes();
     if (linear_bytes) *linear_bytes = linear_ws_bytes(op, M, N, K, fmt_a, fmt_b);
     return SNIP_OK;
 }
@@ -279,7 +280,7 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
         else if (op == SNIP_OP_DGRAD) { sb_bs = 1; sb_cs = ceil_div(K, 128); }
         else { sb_bs = 0; sb_cs = p.No; }
         return gemm_impl(fmt[ia], fmt[ib], f.codes[ia], f.codes[ib], p.Mo, p.No, p.Kc, f.scales[ia], p.Mo, f.scales[ib], sb_cs, sb_bs, p.scale_mode, out,
-                         out_dtype, 0, f.gws, gemm_ws_bytes(), st, false);
+                         out_dtype, 0, f.gws, gemm_ws_bytes_sliced(), st, false);
     };
     // one status word serves the three GEMMs of this call: cleared once, so that a timeout of the first is not erased
     rc = gemm_clear_status(f.gws, st);
