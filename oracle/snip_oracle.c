@@ -44,8 +44,12 @@
 #endif
 
 enum { ORC_FMT_BF16 = 0, ORC_FMT_FP8_E4M3 = 1, ORC_FMT_FP4_E2M1 = 2 };
-enum { ORC_BLOCK_ROW = 0, ORC_BLOCK_COL = 1, ORC_BLOCK_BLK = 2 };
+enum { ORC_BLOCK_ROW = 0, ORC_BLOCK_COL = 1, ORC_BLOCK_BLK = 2,
+       /* added option (the paper lets further quantization methods plug in as options, Sec. 3.2): 32-long tiles as in
+        * the microscaling formats the paper cites; meant for the power-of-two scale rule */
+       ORC_BLOCK_ROW32 = 3, ORC_BLOCK_COL32 = 4 };
 #define ORC_TILE 128
+#define ORC_SUBTILE 32
 
 /* ---------------------------------------------------------------------------------------- */
 /* Number formats                                                                            */
@@ -282,11 +286,14 @@ static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
  *   ROW: [ceil(cols/128)][rows]    one scale per 1x128 tile, tile index outermost
  *   COL: [ceil(rows/128)][cols]    one scale per 128x1 tile
  *   BLK: [ceil(rows/128)][ceil(cols/128)]
+ *   ROW32: [ceil(cols/32)][rows]   one scale per 1x32 tile;   COL32: [ceil(rows/32)][cols]   one per 32x1 tile
  */
 void orc_scale_shape(int64_t rows, int64_t cols, int block, int64_t *d0, int64_t *d1)
 {
     if (block == ORC_BLOCK_ROW) { *d0 = ceil_div(cols, ORC_TILE); *d1 = rows; }
     else if (block == ORC_BLOCK_COL) { *d0 = ceil_div(rows, ORC_TILE); *d1 = cols; }
+    else if (block == ORC_BLOCK_ROW32) { *d0 = ceil_div(cols, ORC_SUBTILE); *d1 = rows; }
+    else if (block == ORC_BLOCK_COL32) { *d0 = ceil_div(rows, ORC_SUBTILE); *d1 = cols; }
     else { *d0 = ceil_div(rows, ORC_TILE); *d1 = ceil_div(cols, ORC_TILE); }
 }
 
@@ -295,6 +302,8 @@ static int64_t orc_scale_index(int64_t rows, int64_t cols, int block, int64_t r,
 {
     if (block == ORC_BLOCK_ROW) return (c / ORC_TILE) * rows + r;
     if (block == ORC_BLOCK_COL) return (r / ORC_TILE) * cols + c;
+    if (block == ORC_BLOCK_ROW32) return (c / ORC_SUBTILE) * rows + r;
+    if (block == ORC_BLOCK_COL32) return (r / ORC_SUBTILE) * cols + c;
     return (r / ORC_TILE) * ceil_div(cols, ORC_TILE) + (c / ORC_TILE);
 }
 
@@ -346,7 +355,7 @@ static int orc_quantize_impl(const uint16_t *x, int64_t rows, int64_t cols, int 
 {
     if (!x || rows < 0 || cols < 0) return -1;
     if (fmt != ORC_FMT_BF16 && !orc_format(fmt)) return -1;
-    if (block < ORC_BLOCK_ROW || block > ORC_BLOCK_BLK) return -1;
+    if (block < ORC_BLOCK_ROW || block > ORC_BLOCK_COL32) return -1;
     const orc_minifloat_t *f = orc_format(fmt);
 
     int64_t sd0 = 0, sd1 = 0;

@@ -19,6 +19,7 @@ import numpy as np
 
 FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 0, 1, 2
 BLOCK_ROW, BLOCK_COL, BLOCK_BLK = 0, 1, 2
+BLOCK_ROW32, BLOCK_COL32 = 3, 4   # added option: 1x32 / 32x1 tiles (block-32 power-of-two scales)
 TILE = 128
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -270,23 +271,36 @@ def gemm_wgrad(dyhat: np.ndarray, xhat: np.ndarray) -> np.ndarray:
 # ---- the three GEMMs of one linear layer under a precision choice (Fig. 5) -------------------
 
 def linear_fwd(x_bits, w_bits, fmt_x, fmt_w, pow2_scale=False):
-    """Quantize X with 1x128 tiles along K and W with 128x128 blocks, then Y = Xhat What^T."""
-    qx = quantize(x_bits, fmt_x, BLOCK_ROW, pow2_scale)
-    qw = quantize(w_bits, fmt_w, BLOCK_BLK, pow2_scale)
+    """Quantize X with 1x128 tiles along K and W with 128x128 blocks, then Y = Xhat What^T.
+    pow2_scale = 2 (added option): power-of-two scales on 32-long tiles along the contraction of both operands."""
+    if pow2_scale == 2:
+        qx = quantize(x_bits, fmt_x, BLOCK_ROW32, True)
+        qw = quantize(w_bits, fmt_w, BLOCK_ROW32, True)
+    else:
+        qx = quantize(x_bits, fmt_x, BLOCK_ROW, pow2_scale)
+        qw = quantize(w_bits, fmt_w, BLOCK_BLK, pow2_scale)
     return gemm_fwd(qx.xhat, qw.xhat), qx, qw
 
 
 def linear_dgrad(dy_bits, w_bits, fmt_dy, fmt_w, pow2_scale=False):
     """Quantize dY with 1x128 tiles along N and W with 128x128 blocks, then dX = dYhat What."""
-    qdy = quantize(dy_bits, fmt_dy, BLOCK_ROW, pow2_scale)
-    qw = quantize(w_bits, fmt_w, BLOCK_BLK, pow2_scale)
+    if pow2_scale == 2:   # contraction over N: 1x32 tiles of dY, 32x1 tiles of W[N,K]
+        qdy = quantize(dy_bits, fmt_dy, BLOCK_ROW32, True)
+        qw = quantize(w_bits, fmt_w, BLOCK_COL32, True)
+    else:
+        qdy = quantize(dy_bits, fmt_dy, BLOCK_ROW, pow2_scale)
+        qw = quantize(w_bits, fmt_w, BLOCK_BLK, pow2_scale)
     return gemm_dgrad(qdy.xhat, qw.xhat), qdy, qw
 
 
 def linear_wgrad(dy_bits, x_bits, fmt_dy, fmt_x, pow2_scale=False):
     """Quantize dY and X with 128x1 tiles along M (the contraction), then dW = dYhat^T Xhat."""
-    qdy = quantize(dy_bits, fmt_dy, BLOCK_COL, pow2_scale)
-    qx = quantize(x_bits, fmt_x, BLOCK_COL, pow2_scale)
+    if pow2_scale == 2:
+        qdy = quantize(dy_bits, fmt_dy, BLOCK_COL32, True)
+        qx = quantize(x_bits, fmt_x, BLOCK_COL32, True)
+    else:
+        qdy = quantize(dy_bits, fmt_dy, BLOCK_COL, pow2_scale)
+        qx = quantize(x_bits, fmt_x, BLOCK_COL, pow2_scale)
     return gemm_wgrad(qdy.xhat, qx.xhat), qdy, qx
 
 
@@ -319,7 +333,8 @@ def sf_atoms(q: Quantized, transposed: bool) -> np.ndarray:
     """UE8M0 scale-factor atoms of a power-of-two-scaled Quantized, in the library's layout: one
     512-byte atom per 128x128 tile, indexed [operand row tile][contraction chunk] for the orientation
     the GEMM consumes; inside an atom the byte 127 - e of tile line r (S = 2^e) sits four times at
-    (r % 32) * 16 + (r // 32) * 4.  Lines beyond the matrix hold 127."""
+    (r % 32) * 16 + (r // 32) * 4.  Lines beyond the matrix hold 127.  With 32-long tiles the four bytes are those
+    of the line's four tiles inside the 128-long chunk, in order (tiles beyond the matrix: 127)."""
     tr, tc = -(-q.rows // TILE), -(-q.cols // TILE)
     exps = np.frexp(q.scales.astype(np.float64))[1] - 1            # S = 2^e exactly
     byte = (127 - exps).astype(np.uint8)
@@ -330,6 +345,16 @@ def sf_atoms(q: Quantized, transposed: bool) -> np.ndarray:
                 lines = byte[j, i * TILE:min((i + 1) * TILE, q.rows)]
             elif q.block == BLOCK_COL:     # line = column inside the tile; scales[i][col]
                 lines = byte[i, j * TILE:min((j + 1) * TILE, q.cols)]
+            elif q.block in (BLOCK_ROW32, BLOCK_COL32):
+                # ROW32: line = row, chunk j, scales[4j + k][row];  COL32: line = column, chunk i, scales[4i + k][col]
+                line_tile, chunk = (i, j) if q.block == BLOCK_ROW32 else (j, i)
+                nlines = (q.rows if q.block == BLOCK_ROW32 else q.cols)
+                atom = out[j, i] if transposed else out[i, j]
+                for r in range(min(TILE, nlines - line_tile * TILE)):
+                    for k in range(4):
+                        if 4 * chunk + k < byte.shape[0]:
+                            atom[(r % 32) * 4 + r // 32, k] = byte[4 * chunk + k, line_tile * TILE + r]
+                continue
             else:
                 lines = np.full(TILE, byte[i, j], dtype=np.uint8)
             atom = out[j, i] if transposed else out[i, j]
