@@ -51,7 +51,11 @@ typedef enum { SNIP_FMT_BF16 = 0, SNIP_FMT_FP8_E4M3 = 1, SNIP_FMT_FP4_E2M1 = 2 }
  * and gradients, 128x128 blocks for weights.  A 1x128 tile runs along the contraction dimension
  * of the GEMM that consumes the operand: ROW = along the contiguous (column) index,
  * COL = along the row index (128 consecutive rows of one column). */
-typedef enum { SNIP_BLOCK_ROW_1x128 = 0, SNIP_BLOCK_COL_128x1 = 1, SNIP_BLOCK_BLK_128x128 = 2 } snip_block_t;
+typedef enum {
+    SNIP_BLOCK_ROW_1x128 = 0, SNIP_BLOCK_COL_128x1 = 1, SNIP_BLOCK_BLK_128x128 = 2,
+    /* 32-long tiles, power-of-two scales only (snip_quantize_mx, snip_quantize_dual with pow2_scale): an added option */
+    SNIP_BLOCK_ROW_1x32 = 3, SNIP_BLOCK_COL_32x1 = 4
+} snip_block_t;
 
 /* Output element type of a GEMM.  BF16 is the paper's choice (Sec. 2.2 keeps GEMM outputs in
  * BF16 while the operands are FPX); FP32 exposes the accumulator for parity checks and for
@@ -127,7 +131,8 @@ typedef struct {
 /* Tile kinds of the two outputs of snip_quantize_dual. */
 typedef enum {
     SNIP_DUAL_ROW_COLT = 0, /* as stored: 1x128 tiles along the columns; transposed: 128x1 tiles along the rows */
-    SNIP_DUAL_BLK_BLKT = 1  /* 128x128 blocks, as stored and transposed */
+    SNIP_DUAL_BLK_BLKT = 1, /* 128x128 blocks, as stored and transposed */
+    SNIP_DUAL_ROW32_COL32T = 2 /* 1x32 tiles as stored, 32x1 tiles transposed; power-of-two scales only */
 } snip_dual_kind_t;
 
 /* ---- library information ----------------------------------------------------------------- */
@@ -200,6 +205,8 @@ int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, int64_t ld,
  *   transposed: kind ROW_COLT -> (fmt, SNIP_BLOCK_COL_128x1, SNIP_Q_TRANSPOSED); BLK_BLKT -> (fmt, BLK, SNIP_Q_TRANSPOSED)
  * with independent formats, so codes, scales and statistics are bit-identical to those calls.
  * pow2_scale != 0 selects the power-of-two rule of snip_quantize_mx (and allows sf != NULL).
+ * kind ROW32_COL32T (needs pow2_scale != 0): as_stored = (fmt, SNIP_BLOCK_ROW_1x32), transposed =
+ * (fmt, SNIP_BLOCK_COL_32x1, SNIP_Q_TRANSPOSED), the block-32 form of snip_quantize_mx.
  * Algorithmic bytes per element: 2 + the two outputs' code and scale bytes, instead of 4 + those.
  * The paper does not prescribe how the copies are produced; it only fixes what they contain (Sec. 2.3).
  * ws_bytes >= snip_quantize_dual_workspace() when statistics are requested (else ws may be NULL).
@@ -240,6 +247,12 @@ int snip_quantize_sr(const void *x, int64_t rows, int64_t cols, int64_t ld, int 
  * consumes (ROW: as stored; COL: transposed storage required; BLK: follows SNIP_Q_TRANSPOSED);
  * inside an atom the byte of tile line r is stored four times at (r % 32) * 16 + (r / 32) * 4.
  * snip_quantize_mx_sizes gives the byte size of sf.  Per-row statistics are not offered here.
+ * Block-32 form (the tile length of the microscaling formats): block = SNIP_BLOCK_ROW_1x32 (as stored) or
+ * SNIP_BLOCK_COL_32x1 (with SNIP_Q_TRANSPOSED) gives every 32-long piece of a 128-long tile its own scale by
+ * the same rule.  `scales` is then [ceil(cols/32)][rows] resp. [ceil(rows/32)][cols] (snip_quantize_sizes
+ * knows these kinds), and the four bytes of a tile line in its atom are those of its four pieces in order
+ * instead of one byte four times; snip_gemm_mx consumes such atoms unchanged (the tensor core applies one
+ * byte per 32 elements either way).  Only snip_gemm_mx can multiply these operands.
  */
 int snip_quantize_mx_sizes(int64_t rows, int64_t cols, size_t *sf_bytes_host);
 int snip_quantize_mx(const void *x, int64_t rows, int64_t cols, int64_t ld, int fmt, int block,

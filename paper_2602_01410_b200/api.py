@@ -14,6 +14,7 @@ import torch
 
 FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 0, 1, 2
 BLOCK_ROW, BLOCK_COL, BLOCK_BLK = 0, 1, 2
+BLOCK_ROW32, BLOCK_COL32 = 3, 4   # 32-long tiles, power-of-two scales only
 OUT_BF16, OUT_FP32 = 0, 1
 OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
 Q_TRANSPOSED, Q_STATS, Q_NO_CODES = 1, 2, 4
@@ -49,7 +50,7 @@ class QOut(ctypes.Structure):
                 ("sf", ctypes.c_void_p), ("stats", ctypes.c_void_p), ("seed", ctypes.c_uint64)]
 
 
-DUAL_ROW_COLT, DUAL_BLK_BLKT = 0, 1
+DUAL_ROW_COLT, DUAL_BLK_BLKT, DUAL_ROW32_COL32T = 0, 1, 2
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 DEBUG_WAIT_LIMIT_NS, DEBUG_TX_SKEW_BYTES, DEBUG_GEMM_KERNEL, DEBUG_GEMM_SLICING = 0, 1, 2, 3
 GEMM_KERNEL_AUTO, GEMM_KERNEL_SINGLE, GEMM_KERNEL_PAIR = 0, 1, 2
@@ -235,7 +236,7 @@ def snip_quantize_dual(x: torch.Tensor, kind: int, fmt_stored: int, fmt_transpos
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
     rows, cols = x.shape
     dev = x.device
-    blocks = (BLOCK_ROW, BLOCK_COL) if kind == DUAL_ROW_COLT else (BLOCK_BLK, BLOCK_BLK)
+    blocks = {DUAL_ROW_COLT: (BLOCK_ROW, BLOCK_COL), DUAL_BLK_BLKT: (BLOCK_BLK, BLOCK_BLK), DUAL_ROW32_COL32T: (BLOCK_ROW32, BLOCK_COL32)}[kind]
     outs, structs = [], []
     for i, fmt in enumerate((fmt_stored, fmt_transposed)):
         if bufs is not None:

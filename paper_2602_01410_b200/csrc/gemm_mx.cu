@@ -175,7 +175,12 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                             for (int k = 0; k < kMmas; ++k) {
                                 const int kk = h * kMmas + k;
-                                mma_ss<KIND, false>(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc, (ks > 0 || kk > 0) ? 1u : 0u, sfa, sfb);
+                                // which of the line's four scale bytes this MMA applies: byte k for the 32-long blocks of
+                                // kind::mxf8f6f4, bytes 2k and 2k+1 for the two halves of kind::mxf4's 64-long step
+                                // (descriptor fields b_sf_id at bit 4, a_sf_id at bit 29)
+                                const uint32_t sf_id = (KIND == MmaKind::MXF4) ? 2u * k : (uint32_t)k;
+                                mma_ss<KIND, false>(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc | (sf_id << 4) | (sf_id << 29),
+                                                    (ks > 0 || kk > 0) ? 1u : 0u, sfa, sfb);
                             }
                         }
                     }
@@ -333,15 +338,19 @@ extern "C" int snip_gemm_mx(int op, const snip_qtensor_t *a, const void *sf_a, c
     int64_t Mo, No, Kc;
     if (op == SNIP_OP_FWD) {
         if (a->cols != b->cols || a->transposed || b->transposed) return SNIP_ERR_SHAPE;
-        if (a->block != SNIP_BLOCK_ROW_1x128 || b->block != SNIP_BLOCK_BLK_128x128) return SNIP_ERR_UNSUPPORTED;
+        // the paper's tiles, or 32-long tiles along the contraction on both sides
+        if (!((a->block == SNIP_BLOCK_ROW_1x128 && b->block == SNIP_BLOCK_BLK_128x128) || (a->block == SNIP_BLOCK_ROW_1x32 && b->block == SNIP_BLOCK_ROW_1x32)))
+            return SNIP_ERR_UNSUPPORTED;
         Mo = a->rows; No = b->rows; Kc = a->cols;
     } else if (op == SNIP_OP_DGRAD) {
         if (a->cols != b->rows || a->transposed || !b->transposed) return SNIP_ERR_SHAPE;
-        if (a->block != SNIP_BLOCK_ROW_1x128 || b->block != SNIP_BLOCK_BLK_128x128) return SNIP_ERR_UNSUPPORTED;
+        if (!((a->block == SNIP_BLOCK_ROW_1x128 && b->block == SNIP_BLOCK_BLK_128x128) || (a->block == SNIP_BLOCK_ROW_1x32 && b->block == SNIP_BLOCK_COL_32x1)))
+            return SNIP_ERR_UNSUPPORTED;
         Mo = a->rows; No = b->cols; Kc = a->cols;
     } else {
         if (a->rows != b->rows || !a->transposed || !b->transposed) return SNIP_ERR_SHAPE;
-        if (a->block != SNIP_BLOCK_COL_128x1 || b->block != SNIP_BLOCK_COL_128x1) return SNIP_ERR_UNSUPPORTED;
+        if (!((a->block == SNIP_BLOCK_COL_128x1 && b->block == SNIP_BLOCK_COL_128x1) || (a->block == SNIP_BLOCK_COL_32x1 && b->block == SNIP_BLOCK_COL_32x1)))
+            return SNIP_ERR_UNSUPPORTED;
         Mo = a->cols; No = b->cols; Kc = a->rows;
     }
     return gemm_mx_impl(a->fmt, b->fmt, a->codes, b->codes, sf_a, sf_b, Mo, No, Kc, out, out_dtype, ws, ws_bytes, static_cast<cudaStream_t>(stream), true);

@@ -18,7 +18,7 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
 int transpose_bf16(const void *in, void *out, int64_t rows, int64_t cols, cudaStream_t st);
 size_t gemm_ws_bytes();
 size_t gemm_ws_bytes_sliced();   // with room for the weight-gradient product's contraction slices
-int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bool blk, int pow2, const DualOut &oa, const DualOut &ob,
+int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int kind, int pow2, const DualOut &oa, const DualOut &ob,
                        void *ws, size_t ws_bytes, cudaStream_t st);
 
 namespace {
@@ -34,7 +34,9 @@ size_t code_bytes(int fmt, int64_t rows, int64_t cols)
 size_t scale_bytes(int block, int64_t rows, int64_t cols)
 {
     const int64_t tr = ceil_div(rows, 128), tc = ceil_div(cols, 128);
-    const int64_t n = block == SNIP_BLOCK_ROW_1x128 ? tc * rows : block == SNIP_BLOCK_COL_128x1 ? tr * cols : tr * tc;
+    int64_t n = block == SNIP_BLOCK_ROW_1x128 ? tc * rows : block == SNIP_BLOCK_COL_128x1 ? tr * cols : tr * tc;
+    if (block == SNIP_BLOCK_ROW_1x32) n = ceil_div(cols, 32) * rows;
+    if (block == SNIP_BLOCK_COL_32x1) n = ceil_div(rows, 32) * cols;
     return (size_t)n * sizeof(float);
 }
 size_t stats_bytes(int64_t rows, int64_t cols)
@@ -160,12 +162,17 @@ struct FwdBwdCarve {
     size_t total;
 };
 
-FwdBwdCarve carve_fwd_bwd(void *ws, int64_t M, int64_t N, int64_t K, const int (&fmt)[6], bool mx)
+// mx: 0 = the paper's scale rule, 1 = power-of-two scales on the paper's tiles, 2 = power-of-two scales on 32-long tiles
+// (every tensor, W included, then has 1x32 tiles as stored and 32x1 tiles transposed).
+FwdBwdCarve carve_fwd_bwd(void *ws, int64_t M, int64_t N, int64_t K, const int (&fmt)[6], int mx)
 {
     // index: 0 X/ROW, 1 X/COL^T, 2 W/BLK, 3 W/BLK^T, 4 dY/ROW, 5 dY/COL^T
     const int64_t rows[6] = {M, M, N, N, M, M}, cols[6] = {K, K, K, K, N, N};
-    const int block[6] = {SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_COL_128x1, SNIP_BLOCK_BLK_128x128, SNIP_BLOCK_BLK_128x128, SNIP_BLOCK_ROW_1x128,
-                          SNIP_BLOCK_COL_128x1};
+    const int block128[6] = {SNIP_BLOCK_ROW_1x128, SNIP_BLOCK_COL_128x1, SNIP_BLOCK_BLK_128x128, SNIP_BLOCK_BLK_128x128, SNIP_BLOCK_ROW_1x128,
+                             SNIP_BLOCK_COL_128x1};
+    const int block32[6] = {SNIP_BLOCK_ROW_1x32, SNIP_BLOCK_COL_32x1, SNIP_BLOCK_ROW_1x32, SNIP_BLOCK_COL_32x1, SNIP_BLOCK_ROW_1x32,
+                            SNIP_BLOCK_COL_32x1};
+    const int (&block)[6] = mx == 2 ? block32 : block128;
     FwdBwdCarve f{};
     Carve c(ws, 0);
     f.gws = c.take(gemm_ws_bytes_sliced());
@@ -247,7 +254,8 @@ extern "C" int snip_linear_fwd_bwd_workspace(int64_t M, int64_t N, int64_t K, in
     const int fmt[6] = {fmt_fwd, fmt_wgrad, fmt_fwd, fmt_dgrad, fmt_dgrad, fmt_wgrad};
     for (int f : fmt)
         if (f != SNIP_FMT_FP8_E4M3 && f != SNIP_FMT_FP4_E2M1) return SNIP_ERR_UNSUPPORTED;
-    *bytes = carve_fwd_bwd(nullptr, M, N, K, fmt, pow2_scale != 0).total;
+    if (pow2_scale < 0 || pow2_scale > 2) return SNIP_ERR_ARG;
+    *bytes = carve_fwd_bwd(nullptr, M, N, K, fmt, pow2_scale).total;
     return SNIP_OK;
 }
 
@@ -265,7 +273,10 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool mx = pow2_scale != 0;
     const int fmt[6] = {fmt_fwd, fmt_wgrad, fmt_fwd, fmt_dgrad, fmt_dgrad, fmt_wgrad};
-    const FwdBwdCarve f = carve_fwd_bwd(ws, M, N, K, fmt, mx);
+    const FwdBwdCarve f = carve_fwd_bwd(ws, M, N, K, fmt, pow2_scale);
+    if (pow2_scale == 2 && dy_rounding == SNIP_ROUND_STOCHASTIC) return SNIP_ERR_UNSUPPORTED;
+    const int kind_xdy = pow2_scale == 2 ? SNIP_DUAL_ROW32_COL32T : SNIP_DUAL_ROW_COLT;
+    const int kind_w = pow2_scale == 2 ? SNIP_DUAL_ROW32_COL32T : SNIP_DUAL_BLK_BLKT;
     if (dy_rounding != SNIP_ROUND_NEAREST_EVEN && dy_rounding != SNIP_ROUND_STOCHASTIC) return SNIP_ERR_ARG;
     // stochastic rounding applies to the FP4 copies of dY (indices 4 and 5); an FP8 copy keeps nearest-even
     auto out_of = [&](int i) {
@@ -286,14 +297,14 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
     rc = gemm_clear_status(f.gws, st);
     if (rc) return rc;
     // forward: X and W are read once each and leave both of their quantized copies behind
-    rc = quantize_dual_impl(X, M, K, K, false, mx, out_of(0), out_of(1), f.stats_ws, f.stats_ws_bytes, st);
+    rc = quantize_dual_impl(X, M, K, K, kind_xdy, mx, out_of(0), out_of(1), f.stats_ws, f.stats_ws_bytes, st);
     if (rc) return rc;
-    rc = quantize_dual_impl(W, N, K, K, true, mx, out_of(2), out_of(3), f.stats_ws, f.stats_ws_bytes, st);
+    rc = quantize_dual_impl(W, N, K, K, kind_w, mx, out_of(2), out_of(3), f.stats_ws, f.stats_ws_bytes, st);
     if (rc) return rc;
     rc = gemm(SNIP_OP_FWD, 0, 2, Y);
     if (rc) return rc;
     // backward: dY is read once; dgrad and wgrad consume the stored copies
-    rc = quantize_dual_impl(dY, M, N, N, false, mx, out_of(4), out_of(5), f.stats_ws, f.stats_ws_bytes, st);
+    rc = quantize_dual_impl(dY, M, N, N, kind_xdy, mx, out_of(4), out_of(5), f.stats_ws, f.stats_ws_bytes, st);
     if (rc) return rc;
     rc = gemm(SNIP_OP_DGRAD, 4, 3, dX);
     if (rc) return rc;

@@ -60,6 +60,13 @@ struct QuantShared {
     double red_d[8][4];
 };
 
+// Scratch of the 32-long tile kinds (kernels that use them ask for this much more shared memory): the scale of every
+// 1x32 / 32x1 tile of the 128x128 tile, [32-block][line].
+struct QuantShared32 {
+    __align__(16) float row_scale[4][kTile];
+    __align__(16) float col_scale[4][kTile];
+};
+
 // Tile (r, c) of an nr x nc grid of 128x128 tiles.
 struct Tile {
     int r, c, nr, nc;
@@ -267,15 +274,15 @@ struct SubScales {
 template <class O>
 __device__ __forceinline__ float2 scale_pair(const SubScales &sc, int p, int i)
 {
-    if (O::BLOCK == SNIP_BLOCK_ROW_1x128) return make_float2(sc.s_row[p], sc.s_row[p]);
-    if (O::BLOCK == SNIP_BLOCK_COL_128x1) return make_float2(sc.s_col[2 * i], sc.s_col[2 * i + 1]);
+    if (O::BLOCK == SNIP_BLOCK_ROW_1x128 || O::BLOCK == SNIP_BLOCK_ROW_1x32) return make_float2(sc.s_row[p], sc.s_row[p]);
+    if (O::BLOCK == SNIP_BLOCK_COL_128x1 || O::BLOCK == SNIP_BLOCK_COL_32x1) return make_float2(sc.s_col[2 * i], sc.s_col[2 * i + 1]);
     return make_float2(sc.s_blk, sc.s_blk);
 }
 template <class O>
 __device__ __forceinline__ float2 ninv_pair(const SubScales &sc, int p, int i)
 {
-    if (O::BLOCK == SNIP_BLOCK_ROW_1x128) return make_float2(sc.n_row[p], sc.n_row[p]);
-    if (O::BLOCK == SNIP_BLOCK_COL_128x1) return make_float2(sc.n_col[2 * i], sc.n_col[2 * i + 1]);
+    if (O::BLOCK == SNIP_BLOCK_ROW_1x128 || O::BLOCK == SNIP_BLOCK_ROW_1x32) return make_float2(sc.n_row[p], sc.n_row[p]);
+    if (O::BLOCK == SNIP_BLOCK_COL_128x1 || O::BLOCK == SNIP_BLOCK_COL_32x1) return make_float2(sc.n_col[2 * i], sc.n_col[2 * i + 1]);
     return make_float2(sc.n_blk, sc.n_blk);
 }
 
@@ -357,6 +364,94 @@ __device__ __forceinline__ void col_scales(const QuantArgs &a, const Tile &tl, Q
     sc.n_col[4] = n1.x; sc.n_col[5] = n1.y; sc.n_col[6] = n1.z; sc.n_col[7] = n1.w;
 }
 
+// -1/S of a power-of-two S, from its exponent field (exact).
+__device__ __forceinline__ float neg_inv_pow2(float s) { return __uint_as_float(0x80000000u | ((254u << 23) - __float_as_uint(s))); }
+
+// 1x32 tiles (power-of-two scales only).  The four lanes that share a 32-column piece of a row group combine their
+// maxima with an exchange-halving butterfly (2 shuffles): lane tx then holds rows 4*bit1(tx) + 2*bit0(tx) and the next
+// one of piece tx / 4.  It derives both scales, writes them out and publishes them; after a warp barrier every lane
+// reads the eight scales of its own piece, and lanes 0..7 of the row group assemble the atom words of rows 8*ty + tx
+// (the bytes of the row's four pieces in order).
+template <class O>
+__device__ __forceinline__ void row32_scales(const QuantArgs &a, const Tile &tl, QuantShared32 &s32, const uint32_t (&rmax)[8], int tx, int ty,
+                                             int64_t rbase, SubScales &sc, float &amax_acc)
+{
+    uint32_t pk[4];   // rows 2q (low half) and 2q+1 (high half)
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        pk[q] = max2(__byte_perm(rmax[2 * q], rmax[2 * q + 1], 0x5410) & 0x7FFF7FFFu, __byte_perm(rmax[2 * q], rmax[2 * q + 1], 0x7632) & 0x7FFF7FFFu);
+    const bool b1 = (tx & 2) != 0, b0 = (tx & 1) != 0;
+    uint32_t k0 = b1 ? pk[2] : pk[0], k1 = b1 ? pk[3] : pk[1];
+    const uint32_t g0 = b1 ? pk[0] : pk[2], g1 = b1 ? pk[1] : pk[3];
+    k0 = max2(k0, __shfl_xor_sync(0xFFFFFFFFu, g0, 2));
+    k1 = max2(k1, __shfl_xor_sync(0xFFFFFFFFu, g1, 2));
+    uint32_t k = b0 ? k1 : k0;
+    const uint32_t g = b0 ? k0 : k1;
+    k = max2(k, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+    const int piece = tx >> 2, r2 = (b1 ? 4 : 0) + (b0 ? 2 : 0);
+    const float am0 = bf16lo(k), am1 = bf16hi(k);
+    amax_acc = fmaxf(amax_acc, fmaxf(am0, am1));
+    const float s0 = tile_scale<O::FMT>(am0, 1), s1 = tile_scale<O::FMT>(am1, 1);
+    *reinterpret_cast<float2 *>(&s32.row_scale[piece][8 * ty + r2]) = make_float2(s0, s1);
+    if (O::CODES && (int64_t)tl.c * kTile + 32 * piece < a.cols) {
+        float *dst = a.scales + ((int64_t)tl.c * 4 + piece) * a.rows + rbase + r2;   // scales[32-piece j][row]
+        if (rbase + r2 < a.rows) dst[0] = s0;
+        if (rbase + r2 + 1 < a.rows) dst[1] = s1;
+    }
+    __syncwarp();
+    const float4 v0 = *reinterpret_cast<const float4 *>(&s32.row_scale[piece][8 * ty]);
+    const float4 v1 = *reinterpret_cast<const float4 *>(&s32.row_scale[piece][8 * ty + 4]);
+    sc.s_row[0] = v0.x; sc.s_row[1] = v0.y; sc.s_row[2] = v0.z; sc.s_row[3] = v0.w;
+    sc.s_row[4] = v1.x; sc.s_row[5] = v1.y; sc.s_row[6] = v1.z; sc.s_row[7] = v1.w;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) sc.n_row[p] = neg_inv_pow2(sc.s_row[p]);
+    if (O::CODES && a.sf && tx < 8) {
+        const int r = 8 * ty + tx;
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) word |= ((254u - (__float_as_uint(s32.row_scale[b][r]) >> 23)) & 0xFFu) << (8 * b);
+        a.sf[((int64_t)tl.r * tl.nc + tl.c) * 128 + (r & 31) * 4 + (r >> 5)] = (rbase + tx < a.rows) ? word : 0x7F7F7F7Fu;
+    }
+}
+
+// 32x1 tiles (power-of-two scales only).  sh.col_amax holds each warp's maxima of its 16 rows; a 32-row piece is two
+// warps.  Thread tid owns column tid % 128 and the pieces 2*(tid / 128) and the next one; after the second barrier
+// every thread reads the eight scales of its columns in its own piece, and threads 0..127 assemble the atom word of
+// their column.
+template <class O>
+__device__ __forceinline__ void col32_scales(const QuantArgs &a, const Tile &tl, QuantShared &sh, QuantShared32 &s32, int tid, int tx, int ty,
+                                             int64_t r0, int64_t c0, SubScales &sc)
+{
+    __syncthreads();   // sh.col_amax complete
+    {
+        const uint16_t *h = reinterpret_cast<const uint16_t *>(&sh.col_amax[0][0]);
+        const int col = tid & (kTile - 1);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int piece = 2 * (tid >> 7) + j;
+            const uint32_t m = max((uint32_t)h[(2 * piece) * kTile + col] & 0x7FFFu, (uint32_t)h[(2 * piece + 1) * kTile + col] & 0x7FFFu);
+            const float s = tile_scale<O::FMT>(__uint_as_float(m << 16), 1);
+            s32.col_scale[piece][col] = s;
+            if (O::CODES && c0 + col < a.cols && r0 + 32 * piece < a.rows) a.scales[((int64_t)tl.r * 4 + piece) * a.cols + c0 + col] = s;
+        }
+    }
+    __syncthreads();
+    const int piece = ty >> 2;
+    const float4 v0 = *reinterpret_cast<const float4 *>(&s32.col_scale[piece][8 * tx]);
+    const float4 v1 = *reinterpret_cast<const float4 *>(&s32.col_scale[piece][8 * tx + 4]);
+    sc.s_col[0] = v0.x; sc.s_col[1] = v0.y; sc.s_col[2] = v0.z; sc.s_col[3] = v0.w;
+    sc.s_col[4] = v1.x; sc.s_col[5] = v1.y; sc.s_col[6] = v1.z; sc.s_col[7] = v1.w;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sc.n_col[j] = neg_inv_pow2(sc.s_col[j]);
+    if (O::CODES && a.sf && tid < kTile) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) word |= ((254u - (__float_as_uint(s32.col_scale[b][tid]) >> 23)) & 0xFFu) << (8 * b);
+        // atom [column tile][row tile] (the operand is consumed transposed): one word per column
+        a.sf[((int64_t)tl.c * tl.nr + tl.r) * 128 + (tid & 31) * 4 + (tid >> 5)] = (c0 + tid < a.cols) ? word : 0x7F7F7F7Fu;
+    }
+}
+
 template <class O>
 __device__ __forceinline__ void blk_scales(const QuantArgs &a, const Tile &tl, float blk_am, int tid, SubScales &sc)
 {
@@ -374,11 +469,14 @@ __device__ __forceinline__ void blk_scales(const QuantArgs &a, const Tile &tl, f
 // the last read of the slot has been issued (the caller starts the next tile's fetch there).
 template <class A, class B, bool STATS, bool ROWSTATS, class AfterReads>
 __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArgs &qb, const Tile &tl, const uint4 *slot, QuantShared &sh,
-                                             ThreadStats &ts, AfterReads after_reads)
+                                             QuantShared32 *s32, ThreadStats &ts, AfterReads after_reads)
 {
     static_assert(!(A::TRANSPOSED && B::TRANSPOSED), "one transposed output per pass");
     constexpr bool kRow = (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128) || (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128);
     constexpr bool kCol = (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_128x1) || (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_128x1);
+    constexpr bool kRow32 = (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x32) || (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x32);
+    constexpr bool kCol32 = (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_32x1) || (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_32x1);
+    static_assert(!((kRow && kRow32) || (kCol && kCol32)), "one row-tiled and one column-tiled output per pass");
     constexpr bool kBlk = (A::kQuant && A::BLOCK == SNIP_BLOCK_BLK_128x128) || (B::kQuant && B::BLOCK == SNIP_BLOCK_BLK_128x128);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tx = tid & 15, ty = tid >> 4;
@@ -393,33 +491,38 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
             const uint4 vp = slot[p * kThreads];
-            if (kRow) rmax[p] = absmax2x(absmax2x(vp.x, vp.y), absmax2x(vp.z, vp.w));
-            if (kCol || kBlk || !kRow) {
+            if (kRow || kRow32) rmax[p] = absmax2x(absmax2x(vp.x, vp.y), absmax2x(vp.z, vp.w));
+            if (kCol || kCol32 || kBlk || !(kRow || kRow32)) {
                 cm[0] = absmax2x(cm[0], vp.x);
                 cm[1] = absmax2x(cm[1], vp.y);
                 cm[2] = absmax2x(cm[2], vp.z);
                 cm[3] = absmax2x(cm[3], vp.w);
             }
         }
-        if (kRow) {
+        if (kRow || kRow32) {
             static_assert(!(A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128 && B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128), "one row-tiled output per pass");
+            static_assert(!(A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x32 && B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x32), "one row-tiled output per pass");
             float am = 0.0f;
             if (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128) row_scales<A>(qa, tl, sh, rmax, tx, ty, rbase, sa, am);
             if (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128) row_scales<B>(qb, tl, sh, rmax, tx, ty, rbase, sb, am);
+            if (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x32) row32_scales<A>(qa, tl, *s32, rmax, tx, ty, rbase, sa, am);
+            if (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x32) row32_scales<B>(qb, tl, *s32, rmax, tx, ty, rbase, sb, am);
             if (STATS) ts.amax = fmaxf(ts.amax, am);
         }
-        if (kCol) {
+        if (kCol || kCol32) {
             // the two row groups of a warp, then the 8 warps through shared memory
 #pragma unroll
             for (int q = 0; q < 4; ++q) cm[q] = absmax2x(cm[q], __shfl_xor_sync(0xFFFFFFFFu, cm[q], 16));
             if (lane < 16) *reinterpret_cast<uint4 *>(&sh.col_amax[warp][4 * tx]) = make_uint4(cm[0], cm[1], cm[2], cm[3]);
             if (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_128x1) col_scales<A>(qa, tl, sh, tid, tx, c0, sa);
             if (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_128x1) col_scales<B>(qb, tl, sh, tid, tx, c0, sb);
+            if (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_32x1) col32_scales<A>(qa, tl, sh, *s32, tid, tx, ty, r0, c0, sa);
+            if (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_32x1) col32_scales<B>(qb, tl, sh, *s32, tid, tx, ty, r0, c0, sb);
         }
-        if (kBlk || (!kRow && STATS)) {
+        if (kBlk || (!(kRow || kRow32) && STATS)) {
             uint32_t m = absmax2x(absmax2x(cm[0], cm[1]), absmax2x(cm[2], cm[3])) & 0x7FFF7FFFu;
             m = max(m & 0xFFFFu, m >> 16);
-            if (!kRow && STATS) ts.amax = fmaxf(ts.amax, __uint_as_float(m << 16));
+            if (!(kRow || kRow32) && STATS) ts.amax = fmaxf(ts.amax, __uint_as_float(m << 16));
             if (kBlk) {
                 m = __reduce_max_sync(0xFFFFFFFFu, m);
                 if (lane == 0) sh.red_m[warp] = m;
@@ -584,6 +687,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
 {
     extern __shared__ __align__(128) uint8_t smem[];
     QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
+    QuantShared32 *s32 = reinterpret_cast<QuantShared32 *>(smem + kSmemBytes);   // present only for the 32-long tile kinds
     const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
     // this grid may have been scheduled before the kernel ahead of it on the stream has finished (see
     // launch_persistent): nothing is read or written before that kernel is complete
@@ -599,7 +703,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
         w.next();
-        process_tile<Out<FMT, BLOCK, TRANSPOSED, CODES, SR>, NoOut, STATS, ROWSTATS>(a, a, tl, slot, sh, ts, [&] {
+        process_tile<Out<FMT, BLOCK, TRANSPOSED, CODES, SR>, NoOut, STATS, ROWSTATS>(a, a, tl, slot, sh, s32, ts, [&] {
             if (w.valid()) prefetch_tile(a, w.r, w.c, smem);   // this thread's reads of its slot are done
             prefetch_commit();
         });
@@ -614,11 +718,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) quantize_kernel(const Qu
 struct DualArgs {
     QuantArgs a, b;
 };
-template <int FMT_A, int FMT_B, bool BLK, bool STATS, bool SR_A = false, bool SR_B = false>
+template <int FMT_A, int FMT_B, bool BLK, bool STATS, bool SR_A = false, bool SR_B = false, bool SUB32 = false>
 __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel(const DualArgs d)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
+    QuantShared32 *s32 = reinterpret_cast<QuantShared32 *>(smem + kSmemBytes);   // present only with SUB32
     const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -630,9 +735,9 @@ __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
         w.next();
-        using A = Out<FMT_A, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true, SR_A>;
-        using B = Out<FMT_B, BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true, SR_B>;
-        process_tile<A, B, STATS, false>(d.a, d.b, tl, slot, sh, ts, [&] {
+        using A = Out<FMT_A, SUB32 ? SNIP_BLOCK_ROW_1x32 : BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_ROW_1x128, false, true, SR_A>;
+        using B = Out<FMT_B, SUB32 ? SNIP_BLOCK_COL_32x1 : BLK ? SNIP_BLOCK_BLK_128x128 : SNIP_BLOCK_COL_128x1, true, true, SR_B>;
+        process_tile<A, B, STATS, false>(d.a, d.b, tl, slot, sh, s32, ts, [&] {
             if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
             prefetch_commit();
         });
@@ -705,16 +810,16 @@ __global__ void row_stats_reduce_kernel(const float2 *row_partials, int64_t rows
 // Launch of a persistent kernel: its dynamic shared memory exceeds the default limit, so the limit is
 // raised first (a per-function, per-device attribute; setting it again is cheap).
 template <typename Kernel, typename Args>
-void launch_persistent(Kernel kernel, const Args &args, dim3 grid, cudaStream_t st)
+void launch_persistent(Kernel kernel, const Args &args, dim3 grid, cudaStream_t st, size_t smem_bytes = kSmemBytes)
 {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) return;  // left in cudaGetLastError
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess) return;  // left in cudaGetLastError
     // Programmatic stream serialization: when the kernel before it on the stream signals its dependents early (the
     // statistics reduction of the previous call does), this grid's CTAs may take their places while that kernel
     // drains; they block in griddepcontrol.wait until it has completed, before they touch global memory.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -746,6 +851,24 @@ void launch_fmt(const QuantArgs &a, int block, bool transposed, bool codes, bool
     } else {
         if (transposed) launch_variant<FMT, SNIP_BLOCK_BLK_128x128, true>(a, codes, stats, rowstats, grid, st);
         else launch_variant<FMT, SNIP_BLOCK_BLK_128x128, false>(a, codes, stats, rowstats, grid, st);
+    }
+}
+
+constexpr size_t kSmemBytes32 = kSmemBytes + sizeof(QuantShared32);
+constexpr int kCtasPerSm32 = 3;   // what the larger shared-memory footprint allows
+
+// 32-long tile kinds: 1x32 tiles as stored, 32x1 tiles transposed.
+template <int FMT>
+void launch_fmt32(const QuantArgs &a, int block, bool codes, bool stats, dim3 grid, cudaStream_t st)
+{
+    if (block == SNIP_BLOCK_ROW_1x32) {
+        if (codes && stats) launch_persistent(quantize_kernel<FMT, SNIP_BLOCK_ROW_1x32, false, true, true, false>, a, grid, st, kSmemBytes32);
+        else if (codes) launch_persistent(quantize_kernel<FMT, SNIP_BLOCK_ROW_1x32, false, true, false, false>, a, grid, st, kSmemBytes32);
+        else launch_persistent(quantize_kernel<FMT, SNIP_BLOCK_ROW_1x32, false, false, true, false>, a, grid, st, kSmemBytes32);
+    } else {
+        if (codes && stats) launch_persistent(quantize_kernel<FMT, SNIP_BLOCK_COL_32x1, true, true, true, false>, a, grid, st, kSmemBytes32);
+        else if (codes) launch_persistent(quantize_kernel<FMT, SNIP_BLOCK_COL_32x1, true, true, false, false>, a, grid, st, kSmemBytes32);
+        else launch_persistent(quantize_kernel<FMT, SNIP_BLOCK_COL_32x1, false, false, true, false>, a, grid, st, kSmemBytes32);
     }
 }
 
@@ -799,7 +922,13 @@ int quantize_impl_full(const void *x, int64_t rows, int64_t cols, int64_t ld, in
         // atoms follow the orientation the GEMM consumes: row tiles as stored, column tiles transposed
         if (!pow2 || !aligned16(sf) || (block == SNIP_BLOCK_ROW_1x128 && tr) || (block == SNIP_BLOCK_COL_128x1 && !tr)) return SNIP_ERR_UNSUPPORTED;
     }
-    if (!x || !valid_fmt(fmt) || !valid_block(block)) return SNIP_ERR_ARG;
+    const bool b32 = block == SNIP_BLOCK_ROW_1x32 || block == SNIP_BLOCK_COL_32x1;
+    if (b32) {
+        // 32-long tiles: power-of-two scales of a quantized format, 1x32 as stored or 32x1 transposed, no per-row sums, RNE
+        const bool tr = (flags & SNIP_Q_TRANSPOSED) != 0;
+        if (!pow2 || sr || row_stats || fmt == SNIP_FMT_BF16 || (block == SNIP_BLOCK_ROW_1x32) == tr) return SNIP_ERR_UNSUPPORTED;
+    }
+    if (!x || !valid_fmt(fmt) || !(valid_block(block) || b32)) return SNIP_ERR_ARG;
     if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
     const bool want_stats = (flags & SNIP_Q_STATS) != 0;
     const bool want_rows = row_stats != nullptr;
@@ -829,8 +958,12 @@ int quantize_impl_full(const void *x, int64_t rows, int64_t cols, int64_t ld, in
     a.partials = any_stats ? static_cast<CtaPartial *>(ws) : nullptr;
     a.row_partials = want_rows ? reinterpret_cast<float2 *>(static_cast<uint8_t *>(ws) + align_up((size_t)(tr * tc) * sizeof(CtaPartial), 256)) : nullptr;
     a.tiles_r = (int32_t)tr; a.tiles_c = (int32_t)tc; a.ntiles = tr * tc;
-    const int64_t nparts = persistent_ctas(tr * tc);
+    const int64_t nparts = persistent_ctas(tr * tc, b32 ? kCtasPerSm32 : kCtasPerSm);
     dim3 grid((unsigned)nparts);
+    if (b32) {
+        if (fmt == SNIP_FMT_FP8_E4M3) launch_fmt32<SNIP_FMT_FP8_E4M3>(a, block, want_codes, any_stats, grid, st);
+        else launch_fmt32<SNIP_FMT_FP4_E2M1>(a, block, want_codes, any_stats, grid, st);
+    } else
     if (sr) {
         const bool row = block == SNIP_BLOCK_ROW_1x128 && !transposed, colt = block == SNIP_BLOCK_COL_128x1 && transposed;
         if (fmt != SNIP_FMT_FP4_E2M1 || !want_codes || want_rows || !(row || colt)) return SNIP_ERR_UNSUPPORTED;
@@ -883,10 +1016,20 @@ static void launch_dual(const DualArgs &d, bool blk, bool stats, dim3 grid, cuda
     else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false>, d, grid, st);
 }
 
-int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bool blk, int pow2, const DualOut &oa, const DualOut &ob,
+template <int FMT_A, int FMT_B>
+static void launch_dual32(const DualArgs &d, bool stats, dim3 grid, cudaStream_t st)
+{
+    if (stats) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, true, false, false, true>, d, grid, st, kSmemBytes32);
+    else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false, false, false, true>, d, grid, st, kSmemBytes32);
+}
+
+// kind: SNIP_DUAL_ROW_COLT, SNIP_DUAL_BLK_BLKT or SNIP_DUAL_ROW32_COL32T (power-of-two scales only).
+int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int kind, int pow2, const DualOut &oa, const DualOut &ob,
                        void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (!x) return SNIP_ERR_ARG;
+    const bool blk = kind == SNIP_DUAL_BLK_BLKT, sub32 = kind == SNIP_DUAL_ROW32_COL32T;
+    if (sub32 && (!pow2 || oa.sr || ob.sr)) return SNIP_ERR_UNSUPPORTED;
     if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
     const DualOut *o[2] = {&oa, &ob};
     for (int i = 0; i < 2; ++i) {
@@ -924,6 +1067,12 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, bo
     dim3 grid((unsigned)nparts);
     const bool a8 = oa.fmt == SNIP_FMT_FP8_E4M3, b8 = ob.fmt == SNIP_FMT_FP8_E4M3;
     constexpr int F8 = SNIP_FMT_FP8_E4M3, F4 = SNIP_FMT_FP4_E2M1;
+    if (sub32) {
+        if (a8 && b8) launch_dual32<F8, F8>(d, stats, grid, st);
+        else if (a8) launch_dual32<F8, F4>(d, stats, grid, st);
+        else if (b8) launch_dual32<F4, F8>(d, stats, grid, st);
+        else launch_dual32<F4, F4>(d, stats, grid, st);
+    } else
     if (oa.sr || ob.sr) {
         if (blk || (oa.sr && a8) || (ob.sr && b8)) return SNIP_ERR_UNSUPPORTED;   // FP4 row / column tiles only
         if (oa.sr && ob.sr) launch_dual_sr<F4, F4, true, true>(d, stats, grid, st);
@@ -959,7 +1108,8 @@ extern "C" int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int bloc
                                    size_t *codes_bytes, size_t *scales_bytes, size_t *ws_bytes)
 {
     using namespace snip;
-    if (!valid_fmt(fmt) || !valid_block(block)) return SNIP_ERR_ARG;
+    const bool b32 = block == SNIP_BLOCK_ROW_1x32 || block == SNIP_BLOCK_COL_32x1;
+    if (!valid_fmt(fmt) || !(valid_block(block) || b32)) return SNIP_ERR_ARG;
     if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
     const bool want_codes = fmt != SNIP_FMT_BF16 && !(flags & SNIP_Q_NO_CODES);
     size_t cb = 0, sb = 0;
@@ -970,6 +1120,8 @@ extern "C" int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int bloc
         if (fmt == SNIP_FMT_FP4_E2M1 && ((rows % 128) || (cols % 128))) cb += 64;
         const int64_t tr = ceil_div(rows, 128), tc = ceil_div(cols, 128);
         int64_t n = block == SNIP_BLOCK_ROW_1x128 ? tc * rows : block == SNIP_BLOCK_COL_128x1 ? tr * cols : tr * tc;
+        if (block == SNIP_BLOCK_ROW_1x32) n = ceil_div(cols, 32) * rows;
+        if (block == SNIP_BLOCK_COL_32x1) n = ceil_div(rows, 32) * cols;
         sb = (size_t)n * sizeof(float);
     }
     if (codes_bytes) *codes_bytes = cb;
@@ -1082,11 +1234,11 @@ extern "C" int snip_quantize_dual(const void *x, int64_t rows, int64_t cols, int
 {
     using namespace snip;
     if (!as_stored || !transposed) return SNIP_ERR_ARG;
-    if (kind != SNIP_DUAL_ROW_COLT && kind != SNIP_DUAL_BLK_BLKT) return SNIP_ERR_ARG;
+    if (kind != SNIP_DUAL_ROW_COLT && kind != SNIP_DUAL_BLK_BLKT && kind != SNIP_DUAL_ROW32_COL32T) return SNIP_ERR_ARG;
     if ((as_stored->rounding & ~1) || (transposed->rounding & ~1)) return SNIP_ERR_ARG;
     const DualOut oa = {as_stored->fmt, as_stored->codes, as_stored->scales, as_stored->sf, as_stored->stats, as_stored->rounding, as_stored->seed};
     const DualOut ob = {transposed->fmt, transposed->codes, transposed->scales, transposed->sf, transposed->stats, transposed->rounding, transposed->seed};
-    return quantize_dual_impl(x, rows, cols, ld, kind == SNIP_DUAL_BLK_BLKT, pow2_scale ? 1 : 0, oa, ob, ws, ws_bytes,
+    return quantize_dual_impl(x, rows, cols, ld, kind, pow2_scale ? 1 : 0, oa, ob, ws, ws_bytes,
                               static_cast<cudaStream_t>(stream));
 }
 
