@@ -210,7 +210,7 @@ class Step:
         dev = self.ws.device
         nbuf = 6 if self.dual else 2
         self.codes = [torch.empty(cb, dtype=torch.uint8, device=dev) for _ in range(nbuf)]
-        self.scales = [torch.empty(sb // 4, dtype=torch.float32, device=dev) for _ in range(nbuf)]
+        self.scales = [torch.empty(sb, dtype=torch.float32, device=dev) for _ in range(nbuf)]   # room for the 32-long tile kinds (4 x the scales)
         self.qws = torch.empty(2 * wb, dtype=torch.uint8, device=dev)
         self.sf = [torch.empty(cb // 32 + 4096, dtype=torch.uint8, device=dev) for _ in range(nbuf)]   # UE8M0 atoms (power-of-two option)
         # GEMM workspace: the size the library reports for a weight-gradient product (room for its contraction slices)
@@ -240,7 +240,7 @@ class Step:
             if qevents is not None:
                 q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 q0.record()
-            api._check("snip_quantize_dual", lib.snip_quantize_dual(p(x), r, c, c, kind, int(mx), outs[0], outs[1], p(self.qws), self.qws.numel(), st))
+            api._check("snip_quantize_dual", lib.snip_quantize_dual(p(x), r, c, c, kind, 1 if mx else 0, outs[0], outs[1], p(self.qws), self.qws.numel(), st))
             if qevents is not None:
                 q1.record()
                 # algorithmic bytes: one bf16 read, two code + scale outputs
@@ -265,6 +265,26 @@ class Step:
                 M, K = x.shape
                 N = w.shape[0]
                 fl = 2.0 * M * N * K
+                # mx == 2: power-of-two scales on 32-long tiles (1x32 as stored, 32x1 transposed, for W as well)
+                R, C, B = (api.BLOCK_ROW32, api.BLOCK_COL32, None) if mx == 2 else (api.BLOCK_ROW, api.BLOCK_COL, api.BLOCK_BLK)
+                if self.dual and mx == 2:
+                    srow = self.stats6[i // 3].view(-1)
+                    i += 3
+                    k32 = api.DUAL_ROW32_COL32T
+                    dual(x, f, k32, 0, srow[0:48]); dual(w, f, k32, 2, srow[48:96])
+                    gemm(api.OP_FWD, f, M, K, R, 0, N, K, R, 0, y, fl, 0, 2)
+                    dual(dy, f, k32, 4, srow[96:144])
+                    gemm(api.OP_DGRAD, f, M, N, R, 0, N, K, C, 1, dx, fl, 4, 3)
+                    gemm(api.OP_WGRAD, f, M, N, C, 1, M, K, C, 1, dw, fl, 5, 1)
+                    continue
+                if mx == 2:
+                    quant(x, f, R, 0, 0, self.stats[2 * i]); quant(w, f, R, 0, 1, self.stats[2 * i + 1]); i += 1
+                    gemm(api.OP_FWD, f, M, K, R, 0, N, K, R, 0, y, fl)
+                    quant(dy, f, R, 0, 0, self.stats[2 * i]); quant(w, f, C, T, 1, self.stats[2 * i + 1]); i += 1
+                    gemm(api.OP_DGRAD, f, M, N, R, 0, N, K, C, 1, dx, fl)
+                    quant(dy, f, C, T, 0, self.stats[2 * i]); quant(x, f, C, T, 1, self.stats[2 * i + 1]); i += 1
+                    gemm(api.OP_WGRAD, f, M, N, C, 1, M, K, C, 1, dw, fl)
+                    continue
                 if self.dual:
                     # slots: 0 X/ROW, 1 X/COL^T, 2 W/BLK, 3 W/BLK^T, 4 dY/ROW, 5 dY/COL^T
                     srow = self.stats6[i // 3].view(-1)
@@ -416,7 +436,8 @@ class KernelTimer:
         api, torch = self.api, self.torch
         g = torch.Generator(device=self.device); g.manual_seed(2)
         xs = [torch.randn(rows, cols, generator=g, device=self.device, dtype=torch.float32).to(torch.bfloat16) for _ in range(3)]
-        bufs = api.snip_quantize_dual(xs[0], kind, fmt, fmt, want_stats=stats)
+        b32 = kind == api.DUAL_ROW32_COL32T    # power-of-two scales per 32-long tile, with the scale-factor atoms
+        bufs = api.snip_quantize_dual(xs[0], kind, fmt, fmt, want_stats=stats, pow2_scale=b32, want_sf=b32)
         ws = torch.empty(api.snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=self.device)
         times = []
         batch = 6
@@ -424,12 +445,12 @@ class KernelTimer:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             for j in range(batch):
-                api.snip_quantize_dual(xs[j % 3], kind, fmt, fmt, bufs=bufs, ws=ws)
+                api.snip_quantize_dual(xs[j % 3], kind, fmt, fmt, bufs=bufs, ws=ws, pow2_scale=b32)
             e1.record()
             torch.cuda.synchronize()
             if i >= warmup:
                 times.append(e0.elapsed_time(e1) / batch)
-        bytes_per_elt = 2.0 + 2.0 * ((1.0 if fmt == FMT_FP8 else 0.5) + 4.0 / 128.0)
+        bytes_per_elt = 2.0 + 2.0 * ((1.0 if fmt == FMT_FP8 else 0.5) + (5.0 / 32.0 if b32 else 4.0 / 128.0))   # FP32 scale (+ 1 atom byte) per tile
         return bytes_per_elt * rows * cols, times
 
 
@@ -489,7 +510,7 @@ def run_profile_case(name):
         parts = parts[:-1]
     if parts[0] == "quantize" and parts[2] == "dual":
         kt = KernelTimer(api, torch, wl.CONFIGS[3], device)
-        kind = api.DUAL_BLK_BLKT if parts[-1] == "blk" else api.DUAL_ROW_COLT
+        kind = api.DUAL_BLK_BLKT if parts[-1] == "blk" else api.DUAL_ROW32_COL32T if parts[-1] == "b32" else api.DUAL_ROW_COLT
         by, times = kt.quantizer_dual(fmt, kind, 16384, 4096, iters=3, warmup=1, stats=not nostats)
         print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
     elif parts[0] == "quantize" and parts[2] == "sr":
@@ -687,7 +708,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-legs", action="store_true")
     ap.add_argument("--profile-case", default=None,
-                    help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t|dual_rowcol|dual_blk> "
+                    help="run one small kernel case a few times and exit (for ncu): quantize_<fp8|fp4>_<row|col_t|blk_t|dual_rowcol|dual_blk|dual_b32> "
                          "or gemm_<fp8|fp4|mxfp8|mxfp4|pairfp8|pairfp4>_<fwd|dgrad|wgrad>[_MxNxK] or layer_stats_<x|w|plain>")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -775,6 +796,29 @@ def main():
                                           "frac_of_sustained_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f]),
                                           "frac_of_burst_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops"] * NOMINAL_RATIO[f])}
                             for f, d in mx_region.items()}}
+
+    # ---- ... and with those scales on 32-long tiles (the tile length of the microscaling formats) ----
+    for _ in range(3):
+        step.run_decomposed(mx=2)
+    barrier()
+    mx32_events = []
+    m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    m0.record()
+    for _ in range(args.steps):
+        step.run_decomposed(mx32_events, mx=2)
+    m1.record()
+    barrier()
+    ms_mx32, flops_mx32 = combine_replicas(m0.elapsed_time(m1), step.flops, dist if world > 1 else None, device)
+    assert api.snip_poll_status(step.gws) == 0, "device-side timeout reported"
+    mx32_region = {}
+    for fmt, op, fl, a, b in mx32_events:
+        d = mx32_region.setdefault(fmt, {"flops": 0.0, "ms": 0.0})
+        d["flops"] += fl; d["ms"] += a.elapsed_time(b)
+    pow2_option["block32"] = {"value": flops_mx32 / (ms_mx32 / args.steps * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_mx32 / args.steps,
+                              "note": "power-of-two scales per 1x32 / 32x1 tile (W included), same hardware-scaled GEMM kernels",
+                              "gemm": {FMT_NAME[f]: {"tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12,
+                                                     "frac_of_sustained_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f])}
+                                       for f, d in mx32_region.items()}}
 
     # ---- end to end: inputs start in pinned host memory, statistics come back -------------------
     e2e = None
@@ -887,7 +931,7 @@ def main():
                 by, times = kt.quantizer(f, block, tr, cfg.M, 4096)
                 avg = sum(times) / len(times)
                 kernels[f"quantize_{FMT_NAME[f]}_{name}"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}
-            for kind, name in ((api.DUAL_ROW_COLT, "row+col_t"), (api.DUAL_BLK_BLKT, "blk+blk_t")):
+            for kind, name in ((api.DUAL_ROW_COLT, "row+col_t"), (api.DUAL_BLK_BLKT, "blk+blk_t"), (api.DUAL_ROW32_COL32T, "row32+col32_t_pow2")):
                 by, times = kt.quantizer_dual(f, kind, cfg.M, 4096)
                 avg = sum(times) / len(times)
                 kernels[f"quantize_dual_{FMT_NAME[f]}_{name}"] = {"gbs": by / (avg * 1e-3) / 1e9, "frac_of_hbm": by / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"], "ms": avg}

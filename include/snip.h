@@ -359,7 +359,9 @@ int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes
  *   W:  128x128 blocks, fmt_fwd (fwd) + the same blocks transposed, fmt_dgrad (dgrad)
  *   dY: 1x128 tiles, fmt_dgrad (dgrad) + 128x1 tiles transposed, fmt_wgrad (wgrad)
  * Results equal those of snip_linear_fwd / _dgrad / _wgrad (pow2_scale = 0) or snip_linear_mx
- * (pow2_scale != 0) called with the same tags.  stats6 (device, may be NULL): six snip_stats_t in the
+ * (pow2_scale = 1) called with the same tags.  pow2_scale = 2: power-of-two scales on 32-long tiles
+ * along each GEMM's contraction for all three tensors (W too: 1x32 tiles for fwd, 32x1 tiles
+ * transposed for dgrad; see the block-32 form of snip_quantize_mx); no stochastic rounding there.  stats6 (device, may be NULL): six snip_stats_t in the
  * order X/1x128, X/128x1, W/fwd format, W/dgrad format, dY/1x128, dY/128x1.  out_dtype applies to all
  * three outputs.  dy_rounding = SNIP_ROUND_STOCHASTIC rounds the FP4 copies of dY stochastically with
  * dy_seed (Sec. 6.1; see snip_quantize_sr), FP8 copies stay nearest-even.  BF16 tags are not offered
