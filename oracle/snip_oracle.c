@@ -422,6 +422,82 @@ static int orc_quantize_impl(const uint16_t *x, int64_t rows, int64_t cols, int 
     return 0;
 }
 
+/*
+ * Two-level block scaling in the style of NVFP4 (added option; the paper lets further quantization methods plug in
+ * as options, Sec. 3.2): E2M1 codes in tiles of 16 along the contraction, one E4M3 scale byte per tile (used
+ * unsigned), one binary32 factor per tensor.  The paper gives no rule for it; this one is fixed here:
+ *   enc   = binary32 quotient 2688 / tensor_amax   (2688 = 448 * 6; enc = 1 if tensor_amax == 0)
+ *   d     = binary32 product of the binary32 quotient amax_tile / 6 with enc
+ *   sf    = d rounded to E4M3 (nearest, ties to even, saturating at 448): a code 0x00 .. 0x7E
+ *   E     = binary32 quotient enc / value(sf)         (a tile with value(sf) == 0 gets all-zero codes)
+ *   t     = binary32 product x * E;  code = t rounded to E2M1 (nearest even, saturating at 6)
+ *   xhat  = value(code) * value(sf) / enc  in binary64  (what the block-scaled tensor core followed by one
+ *           division by enc computes)
+ * col_tiles = 0: 1x16 tiles along the columns, sf[ceil(cols/16)][rows]; 1: 16x1 tiles along the rows,
+ * sf[ceil(rows/16)][cols].  tensor_amax is an input (any positive bound of max|x| works; the exact maximum uses the
+ * scale bytes' range best).  codes / sf / xhat / sumsq may be NULL.  Returns 0, or -1 on a bad argument.
+ */
+int orc_quantize_nvfp4(const uint16_t *x, int64_t rows, int64_t cols, int col_tiles, float tensor_amax,
+                       uint8_t *codes, uint8_t *sf, float *enc_out, double *xhat, double *sumsq)
+{
+    if (!x || rows < 0 || cols < 0 || !(tensor_amax >= 0.0f)) return -1;
+    const int64_t tl = 16;
+    const int64_t nt = col_tiles ? ceil_div(rows, tl) : ceil_div(cols, tl);   /* tiles per line */
+    const int64_t lines = col_tiles ? cols : rows;
+    volatile float enc = tensor_amax == 0.0f ? 1.0f : 2688.0f / tensor_amax;
+    if (isinf(enc)) enc = FLT_MAX;
+    if (enc_out) *enc_out = enc;
+    uint8_t *sfl = (uint8_t *)malloc((size_t)(nt * lines > 0 ? nt * lines : 1));
+    float *am = (float *)calloc((size_t)(nt * lines > 0 ? nt * lines : 1), sizeof(float));
+    if (!sfl || !am) { free(sfl); free(am); return -1; }
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c) {
+            float a = fabsf(orc_bf16_to_float(x[r * cols + c]));
+            int64_t si = col_tiles ? (r / tl) * cols + c : (c / tl) * rows + r;
+            if (a > am[si]) am[si] = a;
+        }
+    for (int64_t i = 0; i < nt * lines; ++i) {
+        volatile float q = am[i] / 6.0f;
+        volatile float d = q * enc;
+        sfl[i] = (uint8_t)orc_encode(&ORC_E4M3, d);
+    }
+    double *rs = (double *)malloc(sizeof(double) * 2 * (size_t)(rows > 0 ? rows : 1));
+    if (!rs) { free(sfl); free(am); return -1; }
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        double tx = 0.0, te = 0.0;
+        for (int64_t c = 0; c < cols; ++c) {
+            float xf = orc_bf16_to_float(x[r * cols + c]);
+            int64_t si = col_tiles ? (r / tl) * cols + c : (c / tl) * rows + r;
+            double sv = orc_decode(&ORC_E4M3, sfl[si]);
+            unsigned code = 0;
+            if (sv != 0.0) {
+                volatile float E = enc / (float)sv;
+                volatile float t = xf * E;
+                code = orc_encode(&ORC_E2M1, t);
+            } else if (signbit(xf)) {
+                code = 0x8;   /* the sign survives, as it does for an underflowing product */
+            }
+            double xh = orc_decode(&ORC_E2M1, code) * sv / (double)enc;
+            if (codes) codes[r * cols + c] = (uint8_t)code;
+            if (xhat) xhat[r * cols + c] = xh;
+            double xd = (double)xf, dd = xd - xh;
+            tx += xd * xd;
+            te += dd * dd;
+        }
+        rs[2 * r] = tx;
+        rs[2 * r + 1] = te;
+    }
+    double tot_x = 0.0, tot_e = 0.0;   /* rows added in ascending order: independent of threading */
+    for (int64_t r = 0; r < rows; ++r) { tot_x += rs[2 * r]; tot_e += rs[2 * r + 1]; }
+    free(rs);
+    if (sf) memcpy(sf, sfl, (size_t)(nt * lines));
+    if (sumsq) { sumsq[0] = tot_x; sumsq[1] = tot_e; }
+    free(sfl);
+    free(am);
+    return 0;
+}
+
 /* Dequantize codes + scales to binary64: xhat = value(code) / S (Sec. 2.3: the scale is removed
  * after the operator by dividing by it). */
 int orc_dequantize(const uint8_t *codes, const float *scales, int64_t rows, int64_t cols,

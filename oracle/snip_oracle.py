@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.orc_quantize.argtypes = [vp, i64, i64, i32, i32, vp, vp, vp, vp, vp]
         L.orc_quantize_rule.restype = i32
         L.orc_quantize_rule.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.orc_quantize_nvfp4.restype = i32
+        L.orc_quantize_nvfp4.argtypes = [vp, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp]
         L.orc_quantize_sr.restype = i32
         L.orc_quantize_sr.argtypes = [vp, i64, i64, i32, i32, i32, ctypes.c_uint64, vp, vp, vp, vp, vp]
         L.orc_philox4x32_10.restype = None
@@ -211,6 +213,75 @@ def quantize(x_bits: np.ndarray, fmt: int, block: int, pow2_scale: bool = False,
         raise ValueError("orc_quantize: bad argument")
     return Quantized(fmt, block, rows, cols, codes, scales, xhat, float(sumsq[0]),
                      float(sumsq[1]), row_sumsq[:, 0].copy(), row_sumsq[:, 1].copy())
+
+
+@dataclass
+class QuantizedNvfp4:
+    """Result of the two-level (NVFP4-style) option: E2M1 codes, one E4M3 scale byte per 16-long tile, one factor per tensor."""
+    rows: int
+    cols: int
+    col_tiles: bool               # False: 1x16 tiles along the columns, sf[ceil(cols/16)][rows]; True: 16x1 tiles, sf[ceil(rows/16)][cols]
+    codes: np.ndarray             # uint8 [rows, cols]
+    sf: np.ndarray                # uint8 E4M3 codes
+    enc: np.float32               # 2688 / tensor_amax: dequantized value = value(code) * value(sf) / enc
+    xhat: np.ndarray              # float64 [rows, cols]
+    sumsq_x: float
+    sumsq_err: float
+
+    def packed(self, transposed: bool = False) -> np.ndarray:
+        return pack_codes(self.codes, FMT_FP4_E2M1, transposed)
+
+
+def quantize_nvfp4(x_bits: np.ndarray, col_tiles: bool = False, tensor_amax: float | None = None) -> QuantizedNvfp4:
+    """tensor_amax = None: the exact maximum magnitude of x."""
+    x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    rows, cols = x.shape
+    if tensor_amax is None:
+        tensor_amax = float(np.abs(bf16_to_float(x)).max()) if x.size else 0.0
+    nt = -(-(rows if col_tiles else cols) // 16)
+    codes = np.zeros((rows, cols), dtype=np.uint8)
+    sf = np.zeros((nt, cols if col_tiles else rows), dtype=np.uint8)
+    enc = np.zeros(1, dtype=np.float32)
+    xhat = np.empty((rows, cols), dtype=np.float64)
+    sumsq = np.zeros(2, dtype=np.float64)
+    rc = lib().orc_quantize_nvfp4(_ptr(x), rows, cols, int(col_tiles), ctypes.c_float(tensor_amax), _ptr(codes), _ptr(sf), _ptr(enc),
+                                  _ptr(xhat), _ptr(sumsq))
+    if rc != 0:
+        raise ValueError("orc_quantize_nvfp4: bad argument")
+    return QuantizedNvfp4(rows, cols, bool(col_tiles), codes, sf, enc[0], xhat, float(sumsq[0]), float(sumsq[1]))
+
+
+def nvfp4_atoms(q: QuantizedNvfp4, transposed: bool) -> np.ndarray:
+    """Scale bytes of a QuantizedNvfp4 in the library's layout: per 128x128 tile and per half (64 elements) of a
+    128-long chunk of the contraction one 512-byte atom, indexed [operand line tile][chunk][half]; inside an atom the
+    word of tile line r (its four 16-long tiles of that half, in order) sits at (r % 32) * 16 + (r // 32) * 4.
+    Lines and tiles beyond the matrix hold 0."""
+    assert transposed == q.col_tiles
+    lines, depth = (q.cols, q.rows) if q.col_tiles else (q.rows, q.cols)
+    lt, ch = -(-lines // TILE), -(-depth // TILE)
+    out = np.zeros((lt, ch, 2, 128, 4), dtype=np.uint8)
+    for i in range(lt):
+        for j in range(ch):
+            for half in range(2):
+                for r in range(min(TILE, lines - i * TILE)):
+                    for k in range(4):
+                        t = 8 * j + 4 * half + k
+                        if t < q.sf.shape[0]:
+                            out[i, j, half, (r % 32) * 4 + r // 32, k] = q.sf[t, i * TILE + r]
+    return out.reshape(-1)
+
+
+def linear_nvfp4(op: str, a_bits, b_bits):
+    """The three GEMMs with both operands under the two-level option: 'fwd' (X, W) -> X W^T with 1x16 tiles along K on
+    both; 'dgrad' (dY, W) -> dY W with 1x16 tiles of dY and 16x1 tiles of W; 'wgrad' (dY, X) -> dY^T X with 16x1 tiles."""
+    if op == "fwd":
+        qa, qb = quantize_nvfp4(a_bits, False), quantize_nvfp4(b_bits, False)
+        return gemm_fwd(qa.xhat, qb.xhat), qa, qb
+    if op == "dgrad":
+        qa, qb = quantize_nvfp4(a_bits, False), quantize_nvfp4(b_bits, True)
+        return gemm_dgrad(qa.xhat, qb.xhat), qa, qb
+    qa, qb = quantize_nvfp4(a_bits, True), quantize_nvfp4(b_bits, True)
+    return gemm_wgrad(qa.xhat, qb.xhat), qa, qb
 
 
 def dequantize(codes: np.ndarray, scales: np.ndarray, fmt: int, block: int) -> np.ndarray:
