@@ -54,7 +54,9 @@ typedef enum { SNIP_FMT_BF16 = 0, SNIP_FMT_FP8_E4M3 = 1, SNIP_FMT_FP4_E2M1 = 2 }
 typedef enum {
     SNIP_BLOCK_ROW_1x128 = 0, SNIP_BLOCK_COL_128x1 = 1, SNIP_BLOCK_BLK_128x128 = 2,
     /* 32-long tiles, power-of-two scales only (snip_quantize_mx, snip_quantize_dual with pow2_scale): an added option */
-    SNIP_BLOCK_ROW_1x32 = 3, SNIP_BLOCK_COL_32x1 = 4
+    SNIP_BLOCK_ROW_1x32 = 3, SNIP_BLOCK_COL_32x1 = 4,
+    /* 16-long tiles of the two-level option (snip_quantize_nvfp4_dual, snip_gemm_nvfp4): an added option */
+    SNIP_BLOCK_ROW_1x16 = 5, SNIP_BLOCK_COL_16x1 = 6
 } snip_block_t;
 
 /* Output element type of a GEMM.  BF16 is the paper's choice (Sec. 2.2 keeps GEMM outputs in
@@ -304,6 +306,39 @@ int snip_gemm_quantized(int op, const snip_qtensor_t *a_host, const snip_qtensor
  */
 int snip_gemm_mx(int op, const snip_qtensor_t *a_host, const void *sf_a, const snip_qtensor_t *b_host,
                  const void *sf_b, void *out, int out_dtype, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Two-level block scaling in the style of NVFP4 (an added option in the sense of paper Sec. 3.2; the paper
+ * does not define it, the rule below is this library's): E2M1 codes in tiles of 16 along the contraction of
+ * the consuming GEMM, one E4M3 scale byte per tile (used unsigned), one binary32 factor per tensor.
+ *   enc  = 2688 / bound (binary32 quotient; 2688 = 448 * 6; enc = 1 if bound == 0), bound = *tensor_amax,
+ *          a device value >= 0: the tensor's maximum magnitude, or an estimate of it (e.g. the amax that an
+ *          earlier call left in a snip_stats_t); values beyond the estimate saturate
+ *   sf   = E4M3 code nearest (ties to even, saturating at 448) to the binary32 value (amax_tile / 6) * enc
+ *   code = E2M1 code nearest to the binary32 product x * (enc / value(sf)); all codes 0 where value(sf) == 0
+ *   dequantized value = value(code) * value(sf) / enc
+ * snip_quantize_nvfp4_dual reads x[rows][ld] once and writes both copies a linear layer needs: as_stored
+ * (1x16 tiles along the columns, codes [rows][cols/2]) and transposed (16x1 tiles along the rows, codes
+ * stored transposed [cols][rows/2]); FP4 packing as in snip_quantize.  Scale bytes come as 512-byte atoms in
+ * the order the tensor core wants them: [operand line tile of 128][128-long chunk of the contraction][half of
+ * the chunk], the word of tile line r (the bytes of its four tiles of that half, in order) at
+ * (r % 32) * 16 + (r / 32) * 4; lines and tiles beyond the matrix hold 0.  snip_quantize_nvfp4_sizes gives
+ * the byte sizes.  stats_* (device, may both be NULL): sum x^2, sum (x - dequantized)^2 and amax of each copy;
+ * ws as for snip_quantize_dual.
+ * snip_gemm_nvfp4: the three products of snip_gemm_quantized over such operands (a / b: codes, rows, cols,
+ * fmt = FP4, block = SNIP_BLOCK_ROW_1x16 or SNIP_BLOCK_COL_16x1 with transposed set, scales unused) on
+ * tcgen05.mma kind::mxf4nvf4 with scale_vec::4X: the tensor core multiplies every 16 products by both scale
+ * bytes and accumulates the whole contraction in FP32 tensor memory; the epilogue divides by enc_a * enc_b
+ * (from the same two bounds) and rounds.  ws: at least 256 bytes, first word = device status word.
+ */
+int snip_quantize_nvfp4_sizes(int64_t rows, int64_t cols, size_t *codes_bytes_host, size_t *sf_bytes_host);
+int snip_quantize_nvfp4_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax,
+                             void *codes_stored, void *sf_stored, snip_stats_t *stats_stored,
+                             void *codes_transposed, void *sf_transposed, snip_stats_t *stats_transposed,
+                             void *ws, size_t ws_bytes, void *stream);
+int snip_gemm_nvfp4(int op, const snip_qtensor_t *a_host, const void *sf_a, const float *amax_a,
+                    const snip_qtensor_t *b_host, const void *sf_b, const float *amax_b, void *out,
+                    int out_dtype, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * One linear layer's forward GEMM under a precision choice: quantize X (1x128 tiles along K)

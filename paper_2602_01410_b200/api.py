@@ -15,6 +15,7 @@ import torch
 FMT_BF16, FMT_FP8_E4M3, FMT_FP4_E2M1 = 0, 1, 2
 BLOCK_ROW, BLOCK_COL, BLOCK_BLK = 0, 1, 2
 BLOCK_ROW32, BLOCK_COL32 = 3, 4   # 32-long tiles, power-of-two scales only
+BLOCK_ROW16, BLOCK_COL16 = 5, 6   # 16-long tiles of the two-level option
 OUT_BF16, OUT_FP32 = 0, 1
 OP_FWD, OP_DGRAD, OP_WGRAD = 0, 1, 2
 Q_TRANSPOSED, Q_STATS, Q_NO_CODES = 1, 2, 4
@@ -25,7 +26,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_linear_fwd",
+    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_quantize_nvfp4_sizes", "snip_quantize_nvfp4_dual", "snip_gemm_nvfp4", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace", "snip_adamw_sensitivity_workspace", "snip_adamw_sensitivity", "snip_loss_divergence", "snip_weight_divergence", "snip_select_scheme",
     "snip_poll_status", "snip_debug_set",
 )
@@ -82,6 +83,9 @@ def _load():
     lib.snip_workspace_size.argtypes = [i32, i64, i64, i64, i32, i32, psz, psz]
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
     lib.snip_gemm_mx.argtypes = [i32, ctypes.POINTER(QTensor), vp, ctypes.POINTER(QTensor), vp, vp, i32, vp, sz, vp]
+    lib.snip_quantize_nvfp4_sizes.argtypes = [i64, i64, psz, psz]
+    lib.snip_quantize_nvfp4_dual.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.snip_gemm_nvfp4.argtypes = [i32, ctypes.POINTER(QTensor), vp, vp, ctypes.POINTER(QTensor), vp, vp, vp, i32, vp, sz, vp]
     lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_fwd.argtypes = lin
     lib.snip_linear_dgrad.argtypes = lin
@@ -295,6 +299,41 @@ def snip_gemm_mx(op, a: QTensor, sf_a, b: QTensor, sf_b, out_shape, out_dtype=OU
         ws = torch.zeros(256, dtype=torch.uint8, device=out.device)
     _check("snip_gemm_mx", _lib.snip_gemm_mx(op, ctypes.byref(a), _p(sf_a), ctypes.byref(b), _p(sf_b), _p(out), out_dtype, _p(ws),
                                              ws.numel(), _stream()))
+    return out
+
+
+def snip_quantize_nvfp4_sizes(rows, cols):
+    cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
+    _check("snip_quantize_nvfp4_sizes", _lib.snip_quantize_nvfp4_sizes(rows, cols, ctypes.byref(cb), ctypes.byref(sb)))
+    return cb.value, sb.value
+
+
+def snip_quantize_nvfp4_dual(x: torch.Tensor, tensor_amax: torch.Tensor, *, want_stats=True, bufs=None, ws=None):
+    """Two-level option, both copies from one read.  tensor_amax: float32 CUDA tensor with one element (the bound of |x|).
+    Returns two dicts (as stored, transposed) with codes / sf / stats tensors."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    assert tensor_amax.is_cuda and tensor_amax.dtype == torch.float32
+    rows, cols = x.shape
+    dev = x.device
+    if bufs is None:
+        cb, sb = snip_quantize_nvfp4_sizes(rows, cols)
+        bufs = tuple({"codes": torch.empty(cb, dtype=torch.uint8, device=dev), "sf": torch.empty(sb, dtype=torch.uint8, device=dev),
+                      "stats": torch.empty(32, dtype=torch.uint8, device=dev) if want_stats else None} for _ in range(2))
+    if ws is None and bufs[0]["stats"] is not None:
+        ws = torch.empty(snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=dev)
+    a, b = bufs
+    _check("snip_quantize_nvfp4_dual", _lib.snip_quantize_nvfp4_dual(_p(x), rows, cols, x.stride(0), _p(tensor_amax), _p(a["codes"]), _p(a["sf"]),
+                                                                     _p(a["stats"]), _p(b["codes"]), _p(b["sf"]), _p(b["stats"]), _p(ws),
+                                                                     0 if ws is None else ws.numel(), _stream()))
+    return a, b
+
+
+def snip_gemm_nvfp4(op, a: QTensor, sf_a, amax_a, b: QTensor, sf_b, amax_b, out_shape, out_dtype=OUT_BF16, *, out=None, ws=None, device="cuda"):
+    out = _out(out_shape, out_dtype, device, out)
+    if ws is None:
+        ws = torch.zeros(256, dtype=torch.uint8, device=out.device)
+    _check("snip_gemm_nvfp4", _lib.snip_gemm_nvfp4(op, ctypes.byref(a), _p(sf_a), _p(amax_a), ctypes.byref(b), _p(sf_b), _p(amax_b), _p(out), out_dtype,
+                                                   _p(ws), ws.numel(), _stream()))
     return out
 
 

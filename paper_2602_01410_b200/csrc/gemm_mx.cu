@@ -12,6 +12,7 @@
 // Every wait is bounded, as in gemm.cu.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <float.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -30,6 +31,7 @@ constexpr int kThreads = 384;
 constexpr int kNumEpiWarps = 8;
 constexpr int kSfaCol = 256;   // tensor-memory columns: accumulator 0..255, SFA 256..259, SFB 260..267
 constexpr int kSfbCol = 260;
+constexpr int kNvSfbCol = 264; // two-level option: a word per line and MMA: SFA 256..263 (two MMAs), SFB 264..279
 constexpr int kTmemCols = 512;
 
 struct MxArgs {
@@ -39,16 +41,20 @@ struct MxArgs {
     int32_t n_atoms_b;         // ceil(No/128)
     uint32_t stage_tx_bytes;   // bytes reported to a stage's barrier (operands + scale-factor atoms)
     uint32_t *status;
+    const float *amax_a, *amax_b;   // two-level option: the tensors' magnitude bounds (device); else null
 };
 
 template <MmaKind KIND>
 struct MxCfg {
-    static constexpr int kChunksPerStage = (KIND == MmaKind::MXF4) ? 2 : 1;   // packed FP4: 256 elements per 128-byte row
+    static constexpr bool kNv = KIND == MmaKind::NVF4;
+    static constexpr int kChunksPerStage = (KIND == MmaKind::MXF4 || kNv) ? 2 : 1;   // packed FP4: 256 elements per 128-byte row
     static constexpr int kABytes = BM * 128;
     static constexpr int kBBytes = BN * 128;
-    static constexpr int kSfBytes = 2048 * kChunksPerStage;                   // per chunk: SFA 512 + SFB 2 x 512 (+ pad)
+    // per chunk: SFA 512 + SFB 2 x 512 (+ pad); two-level option: an atom per 64 elements, SFA 2 x 512 + SFB 4 x 512
+    static constexpr int kSfChunkBytes = kNv ? 3072 : 2048;
+    static constexpr int kSfBytes = kSfChunkBytes * kChunksPerStage;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfBytes;
-    static constexpr int kStages = 4;
+    static constexpr int kStages = kNv ? 3 : 4;
     static constexpr int kOutStageBytes = kNumEpiWarps * 2048;
     static constexpr int kSmemBytes = kStages * kStageBytes + kOutStageBytes + 256 + 1024;
     static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -140,10 +146,16 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int h = 0; h < CPS; ++h) {
                         const int c = min(ks * CPS + h, num_chunks - 1);   // a stage's unused second chunk reloads a valid atom
-                        const uint32_t dst = sf_tile(s) + h * 2048;
-                        bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 512, 512, full_bar(s));
-                        bulk_load_1d(dst + 512, g.sfb + ((int64_t)nb0 * num_chunks + c) * 512, 512, full_bar(s));
-                        bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb1 * num_chunks + c) * 512, 512, full_bar(s));
+                        const uint32_t dst = sf_tile(s) + h * C::kSfChunkBytes;
+                        if (C::kNv) {   // [A: two halves][B rows 0-127: two halves][B rows 128-255: two halves]
+                            bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 1024, 1024, full_bar(s));
+                            bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb0 * num_chunks + c) * 1024, 1024, full_bar(s));
+                            bulk_load_1d(dst + 2048, g.sfb + ((int64_t)nb1 * num_chunks + c) * 1024, 1024, full_bar(s));
+                        } else {
+                            bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 512, 512, full_bar(s));
+                            bulk_load_1d(dst + 512, g.sfb + ((int64_t)nb0 * num_chunks + c) * 512, 512, full_bar(s));
+                            bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb1 * num_chunks + c) * 512, 512, full_bar(s));
+                        }
                     }
                 }
             }
@@ -153,7 +165,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             uint32_t it = 0, tiles_done = 0;
             bool ok = true;
-            const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + kSfbCol;
+            const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + (C::kNv ? kNvSfbCol : kSfbCol);
             for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tiles_done) {
                 // the single accumulator must have been drained by the epilogue of the previous tile
                 if (!mbar_wait(tempty_bar, (tiles_done & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -167,10 +179,17 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int h = 0; h < CPS; ++h) {
                         if (ks * CPS + h < num_chunks) {
-                            const uint32_t sf = sf_tile(s) + h * 2048;
-                            tmem_cp_sf_atom(sfa, sf);
-                            tmem_cp_sf_atom(sfb, sf + 512);
-                            tmem_cp_sf_atom(sfb + 4, sf + 1024);
+                            const uint32_t sf = sf_tile(s) + h * C::kSfChunkBytes;
+                            if (C::kNv) {
+                                // MMA k of the chunk reads a whole word per line: SFA columns 4k.., SFB columns 8k.. (two 128-line groups)
+                                tmem_cp_sf_atom(sfa, sf);             tmem_cp_sf_atom(sfa + 4, sf + 512);
+                                tmem_cp_sf_atom(sfb, sf + 1024);      tmem_cp_sf_atom(sfb + 8, sf + 1536);
+                                tmem_cp_sf_atom(sfb + 4, sf + 2048);  tmem_cp_sf_atom(sfb + 12, sf + 2560);
+                            } else {
+                                tmem_cp_sf_atom(sfa, sf);
+                                tmem_cp_sf_atom(sfb, sf + 512);
+                                tmem_cp_sf_atom(sfb + 4, sf + 1024);
+                            }
                             constexpr int kMmas = 4 / CPS;   // 32 bytes of K per MMA: four per 128-byte row
 #pragma unroll
                             for (int k = 0; k < kMmas; ++k) {
@@ -178,9 +197,9 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 // which of the line's four scale bytes this MMA applies: byte k for the 32-long blocks of
                                 // kind::mxf8f6f4, bytes 2k and 2k+1 for the two halves of kind::mxf4's 64-long step
                                 // (descriptor fields b_sf_id at bit 4, a_sf_id at bit 29)
-                                const uint32_t sf_id = (KIND == MmaKind::MXF4) ? 2u * k : (uint32_t)k;
+                                const uint32_t sf_id = C::kNv ? 0u : (KIND == MmaKind::MXF4) ? 2u * k : (uint32_t)k;
                                 mma_ss<KIND, false>(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc | (sf_id << 4) | (sf_id << 29),
-                                                    (ks > 0 || kk > 0) ? 1u : 0u, sfa, sfb);
+                                                    (ks > 0 || kk > 0) ? 1u : 0u, sfa + (C::kNv ? 4 * k : 0), sfb + (C::kNv ? 8 * k : 0));
                             }
                         }
                     }
@@ -195,6 +214,13 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t stage_u32 = out_stage0 + e * 2048;
         uint32_t tiles_done = 0;
         bool ok = true;
+        // two-level option: the sums carry both tensors' factors 2688 / bound; they are divided out here, once per output
+        float out_scale = 1.0f;
+        if (C::kNv) {
+            const float ba = *g.amax_a, bb = *g.amax_b;
+            const float ea = ba == 0.0f ? 1.0f : fminf(__fdiv_rn(2688.0f, ba), FLT_MAX), eb = bb == 0.0f ? 1.0f : fminf(__fdiv_rn(2688.0f, bb), FLT_MAX);
+            out_scale = __fdiv_rn(1.0f, ea * eb);
+        }
         for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tiles_done) {
             int m_idx, n_idx;
             mx_tile_coords(t, num_m, num_n, m_idx, n_idx);
@@ -211,6 +237,12 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar);   // the next tile's MMAs may start
+            if (C::kNv) {
+#pragma unroll
+                for (int gi = 0; gi < 4; ++gi)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[gi][i] = __float_as_uint(__uint_as_float(v[gi][i]) * out_scale);
+            }
             constexpr int kPerBox = OUT_F32 ? 16 : 32;   // output columns per 64-byte box row
 #pragma unroll
             for (int b = 0; b < HALF / kPerBox; ++b) {
@@ -298,6 +330,7 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
     g.sfb = static_cast<const uint8_t *>(sfb);
     g.n_atoms_b = (int32_t)ceil_div(No, 128);
     g.status = static_cast<uint32_t *>(ws);
+    g.amax_a = g.amax_b = nullptr;
 
     CUtensorMap tmA, tmB, tmO;
     rc = f32 ? make_tiled_map_2d(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Mo, No, No * 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_64B)
@@ -324,6 +357,42 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
     g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128) + 1536;
     const uint32_t idesc = make_idesc_block_scaled(a4 ? 5 : 0, b4 ? 5 : 0, BM, BN);
     return f32 ? launch_mx<MmaKind::MXF8, true>(tmA, tmB, tmO, g, idesc, sms, st) : launch_mx<MmaKind::MXF8, false>(tmA, tmB, tmO, g, idesc, sms, st);
+}
+
+// Two-level option: packed E2M1 codes, E4M3 scale bytes per 16-long tile as atoms [line tile][chunk][half][512], and the
+// two tensors' magnitude bounds (device pointers).  out = (sum of block-scaled products) / (enc_a * enc_b), enc = 2688 / bound.
+int gemm_nvfp4_impl(const void *a_codes, const void *b_codes, const void *sfa, const void *sfb, const float *amax_a, const float *amax_b,
+                    int64_t Mo, int64_t No, int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status)
+{
+    if (!a_codes || !b_codes || !sfa || !sfb || !amax_a || !amax_b || !out) return SNIP_ERR_ARG;
+    if (!valid_dim(Mo) || !valid_dim(No) || !valid_dim(Kc) || Mo > INT32_MAX || No > INT32_MAX || Kc > INT32_MAX) return SNIP_ERR_SHAPE;
+    if (out_dtype != SNIP_OUT_BF16 && out_dtype != SNIP_OUT_FP32) return SNIP_ERR_ARG;
+    if (!ws || ws_bytes < 256) return SNIP_ERR_WORKSPACE;
+    if (!aligned16(a_codes) || !aligned16(b_codes) || !aligned16(sfa) || !aligned16(sfb) || !aligned16(out) || !aligned16(ws)) return SNIP_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(amax_a) & 3u) || (reinterpret_cast<uintptr_t>(amax_b) & 3u)) return SNIP_ERR_ALIGN;
+    int rc = require_sm100();
+    if (rc != SNIP_OK) return rc;
+    if (clear_status) { rc = gemm_clear_status(ws, st); if (rc) return rc; }
+    const bool f32 = out_dtype == SNIP_OUT_FP32;
+    MxArgs g;
+    g.Mo = (int32_t)Mo; g.No = (int32_t)No; g.Kc = (int32_t)Kc;
+    g.sfa = static_cast<const uint8_t *>(sfa);
+    g.sfb = static_cast<const uint8_t *>(sfb);
+    g.n_atoms_b = (int32_t)ceil_div(No, 128);
+    g.status = static_cast<uint32_t *>(ws);
+    g.amax_a = amax_a; g.amax_b = amax_b;
+    CUtensorMap tmA, tmB, tmO;
+    rc = f32 ? make_tiled_map_2d(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Mo, No, No * 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_64B)
+             : make_tiled_map_2d(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Mo, No, No * 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (rc) return rc;
+    rc = make_tiled_map_2d(&tmA, a_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, Mo, Kc / 2, Kc / 2, 128, BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    rc = make_tiled_map_2d(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+    g.stage_tx_bytes = (BM + BN) * 128 + 2 * 3072;
+    const uint32_t idesc = make_idesc_block_scaled_e4m3(1, 1, BM, BN);
+    const int sms = gemm_sm_count();
+    return f32 ? launch_mx<MmaKind::NVF4, true>(tmA, tmB, tmO, g, idesc, sms, st) : launch_mx<MmaKind::NVF4, false>(tmA, tmB, tmO, g, idesc, sms, st);
 }
 
 }  // namespace snip
@@ -354,4 +423,27 @@ extern "C" int snip_gemm_mx(int op, const snip_qtensor_t *a, const void *sf_a, c
         Mo = a->cols; No = b->cols; Kc = a->rows;
     }
     return gemm_mx_impl(a->fmt, b->fmt, a->codes, b->codes, sf_a, sf_b, Mo, No, Kc, out, out_dtype, ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
+}
+
+extern "C" int snip_gemm_nvfp4(int op, const snip_qtensor_t *a, const void *sf_a, const float *amax_a, const snip_qtensor_t *b, const void *sf_b,
+                               const float *amax_b, void *out, int out_dtype, void *ws, size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    if (!a || !b || op < SNIP_OP_FWD || op > SNIP_OP_WGRAD) return SNIP_ERR_ARG;
+    if (a->fmt != SNIP_FMT_FP4_E2M1 || b->fmt != SNIP_FMT_FP4_E2M1) return SNIP_ERR_UNSUPPORTED;
+    int64_t Mo, No, Kc;
+    if (op == SNIP_OP_FWD) {
+        if (a->cols != b->cols || a->transposed || b->transposed) return SNIP_ERR_SHAPE;
+        if (a->block != SNIP_BLOCK_ROW_1x16 || b->block != SNIP_BLOCK_ROW_1x16) return SNIP_ERR_UNSUPPORTED;
+        Mo = a->rows; No = b->rows; Kc = a->cols;
+    } else if (op == SNIP_OP_DGRAD) {
+        if (a->cols != b->rows || a->transposed || !b->transposed) return SNIP_ERR_SHAPE;
+        if (a->block != SNIP_BLOCK_ROW_1x16 || b->block != SNIP_BLOCK_COL_16x1) return SNIP_ERR_UNSUPPORTED;
+        Mo = a->rows; No = b->cols; Kc = a->cols;
+    } else {
+        if (a->rows != b->rows || !a->transposed || !b->transposed) return SNIP_ERR_SHAPE;
+        if (a->block != SNIP_BLOCK_COL_16x1 || b->block != SNIP_BLOCK_COL_16x1) return SNIP_ERR_UNSUPPORTED;
+        Mo = a->cols; No = b->cols; Kc = a->rows;
+    }
+    return gemm_nvfp4_impl(a->codes, b->codes, sf_a, sf_b, amax_a, amax_b, Mo, No, Kc, out, out_dtype, ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
 }

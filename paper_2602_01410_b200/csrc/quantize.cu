@@ -46,6 +46,8 @@ struct QuantArgs {
     uint64_t seed;        // stochastic rounding: key of the generator
     int pow2;             // 1: power-of-two scale rule (largest 2^e with amax * 2^e <= FPX_MAX)
     uint32_t *sf;         // optional: UE8M0 bytes of 1/S in 512-byte atoms for hardware block scaling; null if unused
+                          // (two-level option: the E4M3 scale bytes, two atoms per 128x128 tile)
+    const float *tensor_amax;   // two-level option: bound of the tensor's magnitudes (device); else unused
 };
 
 // Scratch shared memory of one CTA (next to the tile slot).
@@ -65,6 +67,17 @@ struct QuantShared {
 struct QuantShared32 {
     __align__(16) float row_scale[4][kTile];
     __align__(16) float col_scale[4][kTile];
+};
+
+// Scratch of the 16-long tile kinds (two-level option): the scale byte of every 1x16 / 16x1 tile of the 128x128 tile,
+// [line][tile along the contraction], so that a line's four bytes of a half are one word.
+struct QuantShared16 {
+    __align__(16) uint8_t row_sf[kTile][8];
+    __align__(16) uint8_t col_sf[kTile][8];
+};
+// Per-tensor factors of the two-level option: enc = 2688 / bound and its reciprocal.
+struct TwoLevel {
+    float enc = 1.0f, inv_enc = 1.0f;
 };
 
 // Tile (r, c) of an nr x nc grid of 128x128 tiles.
@@ -274,15 +287,15 @@ struct SubScales {
 template <class O>
 __device__ __forceinline__ float2 scale_pair(const SubScales &sc, int p, int i)
 {
-    if (O::BLOCK == SNIP_BLOCK_ROW_1x128 || O::BLOCK == SNIP_BLOCK_ROW_1x32) return make_float2(sc.s_row[p], sc.s_row[p]);
-    if (O::BLOCK == SNIP_BLOCK_COL_128x1 || O::BLOCK == SNIP_BLOCK_COL_32x1) return make_float2(sc.s_col[2 * i], sc.s_col[2 * i + 1]);
+    if (O::BLOCK == SNIP_BLOCK_ROW_1x128 || O::BLOCK == SNIP_BLOCK_ROW_1x32 || O::BLOCK == SNIP_BLOCK_ROW_1x16) return make_float2(sc.s_row[p], sc.s_row[p]);
+    if (O::BLOCK == SNIP_BLOCK_COL_128x1 || O::BLOCK == SNIP_BLOCK_COL_32x1 || O::BLOCK == SNIP_BLOCK_COL_16x1) return make_float2(sc.s_col[2 * i], sc.s_col[2 * i + 1]);
     return make_float2(sc.s_blk, sc.s_blk);
 }
 template <class O>
 __device__ __forceinline__ float2 ninv_pair(const SubScales &sc, int p, int i)
 {
-    if (O::BLOCK == SNIP_BLOCK_ROW_1x128 || O::BLOCK == SNIP_BLOCK_ROW_1x32) return make_float2(sc.n_row[p], sc.n_row[p]);
-    if (O::BLOCK == SNIP_BLOCK_COL_128x1 || O::BLOCK == SNIP_BLOCK_COL_32x1) return make_float2(sc.n_col[2 * i], sc.n_col[2 * i + 1]);
+    if (O::BLOCK == SNIP_BLOCK_ROW_1x128 || O::BLOCK == SNIP_BLOCK_ROW_1x32 || O::BLOCK == SNIP_BLOCK_ROW_1x16) return make_float2(sc.n_row[p], sc.n_row[p]);
+    if (O::BLOCK == SNIP_BLOCK_COL_128x1 || O::BLOCK == SNIP_BLOCK_COL_32x1 || O::BLOCK == SNIP_BLOCK_COL_16x1) return make_float2(sc.n_col[2 * i], sc.n_col[2 * i + 1]);
     return make_float2(sc.n_blk, sc.n_blk);
 }
 
@@ -452,6 +465,81 @@ __device__ __forceinline__ void col32_scales(const QuantArgs &a, const Tile &tl,
     }
 }
 
+// Two-level option: scale byte, encode factor and (negated) decode factor of two tiles from their maxima.
+//   d = (amax / 6) * enc in binary32;  sf = E4M3(d), nearest even, saturating;  E = enc / value(sf);  -value(sf) / enc
+__device__ __forceinline__ uint32_t two_level_pair(float am0, float am1, const TwoLevel &tw, float &e0, float &e1, float &n0, float &n1)
+{
+    const float d0 = __fmul_rn(__fdiv_rn(am0, 6.0f), tw.enc), d1 = __fmul_rn(__fdiv_rn(am1, 6.0f), tw.enc);
+    const uint32_t c = cvt_e4m3x2(d0, d1);          // low byte: first tile
+    const float2 sv = dec_e4m3x2(c);
+    e0 = sv.x == 0.0f ? 0.0f : __fdiv_rn(tw.enc, sv.x);
+    e1 = sv.y == 0.0f ? 0.0f : __fdiv_rn(tw.enc, sv.y);
+    n0 = -sv.x * tw.inv_enc;
+    n1 = -sv.y * tw.inv_enc;
+    return c;
+}
+
+// 1x16 tiles of the two-level option: a tile is the 8 columns of this lane and of its neighbour (lane ^ 1).  Both derive
+// the eight rows' factors; the even lane stages the scale bytes, and after a warp barrier lane tx of the row group
+// writes the atom word of row 8*ty + tx%8, half tx/8 (the bytes of that half's four tiles in order).
+template <class O>
+__device__ __forceinline__ void row16_scales(const QuantArgs &a, const Tile &tl, QuantShared16 &s16, const TwoLevel &tw, const uint32_t (&rmax)[8],
+                                             int tx, int ty, int64_t rbase, SubScales &sc, float &amax_acc)
+{
+    float am[8];
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        const uint32_t m = rmax[p] & 0x7FFF7FFFu;
+        uint32_t mm = max(m & 0xFFFFu, m >> 16);                 // non-negative bf16: integer order
+        mm = max(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, 1));
+        am[p] = __uint_as_float(mm << 16);
+        amax_acc = fmaxf(amax_acc, am[p]);
+    }
+#pragma unroll
+    for (int p = 0; p < 8; p += 2) {
+        const uint32_t c = two_level_pair(am[p], am[p + 1], tw, sc.s_row[p], sc.s_row[p + 1], sc.n_row[p], sc.n_row[p + 1]);
+        if (O::CODES && a.sf && !(tx & 1)) {
+            s16.row_sf[8 * ty + p][tx >> 1] = (uint8_t)(c & 0xFFu);
+            s16.row_sf[8 * ty + p + 1][tx >> 1] = (uint8_t)(c >> 8);
+        }
+    }
+    if (O::CODES && a.sf) {
+        __syncwarp();
+        const int r = 8 * ty + (tx & 7), half = tx >> 3;
+        const uint32_t word = *reinterpret_cast<const uint32_t *>(&s16.row_sf[r][4 * half]);
+        a.sf[(((int64_t)tl.r * tl.nc + tl.c) * 2 + half) * 128 + (r & 31) * 4 + (r >> 5)] = (rbase + (tx & 7) < a.rows) ? word : 0u;
+    }
+}
+
+// 16x1 tiles of the two-level option: a warp holds 16 rows, so after the exchange with lane ^ 16 (done by the caller)
+// cm holds the tile maxima of this lane's eight columns; the tile's index along the contraction is the warp's.
+// The scale bytes are staged for write_col16_atoms, which runs after the CTA barrier of the transposed output.
+template <class O>
+__device__ __forceinline__ void col16_scales(const QuantArgs &a, QuantShared16 &s16, const TwoLevel &tw, const uint32_t (&cm)[4], int lane, int tx,
+                                             int warp, SubScales &sc)
+{
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t m = cm[q] & 0x7FFF7FFFu;
+        const uint32_t c = two_level_pair(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u), tw, sc.s_col[2 * q], sc.s_col[2 * q + 1],
+                                          sc.n_col[2 * q], sc.n_col[2 * q + 1]);
+        if (O::CODES && a.sf && lane < 16) {
+            s16.col_sf[8 * tx + 2 * q][warp] = (uint8_t)(c & 0xFFu);
+            s16.col_sf[8 * tx + 2 * q + 1][warp] = (uint8_t)(c >> 8);
+        }
+    }
+}
+template <class O>
+__device__ __forceinline__ void write_col16_atoms(const QuantArgs &a, const Tile &tl, const QuantShared16 &s16, int tid, int64_t c0)
+{
+    if (O::CODES && a.sf) {
+        const int col = tid & (kTile - 1), half = tid >> 7;
+        const uint32_t word = *reinterpret_cast<const uint32_t *>(&s16.col_sf[col][4 * half]);
+        // atoms [column tile][row tile][half] (the operand is consumed transposed): one word per column and half
+        a.sf[(((int64_t)tl.c * tl.nr + tl.r) * 2 + half) * 128 + (col & 31) * 4 + (col >> 5)] = (c0 + col < a.cols) ? word : 0u;
+    }
+}
+
 template <class O>
 __device__ __forceinline__ void blk_scales(const QuantArgs &a, const Tile &tl, float blk_am, int tid, SubScales &sc)
 {
@@ -469,14 +557,18 @@ __device__ __forceinline__ void blk_scales(const QuantArgs &a, const Tile &tl, f
 // the last read of the slot has been issued (the caller starts the next tile's fetch there).
 template <class A, class B, bool STATS, bool ROWSTATS, class AfterReads>
 __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArgs &qb, const Tile &tl, const uint4 *slot, QuantShared &sh,
-                                             QuantShared32 *s32, ThreadStats &ts, AfterReads after_reads)
+                                             QuantShared32 *s32, ThreadStats &ts, AfterReads after_reads, const TwoLevel &tw = TwoLevel())
 {
+    QuantShared16 *s16 = reinterpret_cast<QuantShared16 *>(s32);   // the same place: a kernel uses one of the two
     static_assert(!(A::TRANSPOSED && B::TRANSPOSED), "one transposed output per pass");
     constexpr bool kRow = (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128) || (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128);
     constexpr bool kCol = (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_128x1) || (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_128x1);
     constexpr bool kRow32 = (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x32) || (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x32);
     constexpr bool kCol32 = (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_32x1) || (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_32x1);
+    constexpr bool kRow16 = (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x16) || (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x16);
+    constexpr bool kCol16 = (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_16x1) || (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_16x1);
     static_assert(!((kRow && kRow32) || (kCol && kCol32)), "one row-tiled and one column-tiled output per pass");
+    static_assert(!(kRow16 && (kRow || kRow32)) && !(kCol16 && (kCol || kCol32)), "one row-tiled and one column-tiled output per pass");
     constexpr bool kBlk = (A::kQuant && A::BLOCK == SNIP_BLOCK_BLK_128x128) || (B::kQuant && B::BLOCK == SNIP_BLOCK_BLK_128x128);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tx = tid & 15, ty = tid >> 4;
@@ -491,13 +583,25 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
             const uint4 vp = slot[p * kThreads];
-            if (kRow || kRow32) rmax[p] = absmax2x(absmax2x(vp.x, vp.y), absmax2x(vp.z, vp.w));
-            if (kCol || kCol32 || kBlk || !(kRow || kRow32)) {
+            if (kRow || kRow32 || kRow16) rmax[p] = absmax2x(absmax2x(vp.x, vp.y), absmax2x(vp.z, vp.w));
+            if (kCol || kCol32 || kCol16 || kBlk || !(kRow || kRow32 || kRow16)) {
                 cm[0] = absmax2x(cm[0], vp.x);
                 cm[1] = absmax2x(cm[1], vp.y);
                 cm[2] = absmax2x(cm[2], vp.z);
                 cm[3] = absmax2x(cm[3], vp.w);
             }
+        }
+        if (kRow16) {
+            float am = 0.0f;
+            if (A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x16) row16_scales<A>(qa, tl, *s16, tw, rmax, tx, ty, rbase, sa, am);
+            if (B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x16) row16_scales<B>(qb, tl, *s16, tw, rmax, tx, ty, rbase, sb, am);
+            if (STATS) ts.amax = fmaxf(ts.amax, am);
+        }
+        if (kCol16) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) cm[q] = absmax2x(cm[q], __shfl_xor_sync(0xFFFFFFFFu, cm[q], 16));
+            if (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_16x1) col16_scales<A>(qa, *s16, tw, cm, lane, tx, warp, sa);
+            if (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_16x1) col16_scales<B>(qb, *s16, tw, cm, lane, tx, warp, sb);
         }
         if (kRow || kRow32) {
             static_assert(!(A::kQuant && A::BLOCK == SNIP_BLOCK_ROW_1x128 && B::kQuant && B::BLOCK == SNIP_BLOCK_ROW_1x128), "one row-tiled output per pass");
@@ -519,10 +623,10 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
             if (A::kQuant && A::BLOCK == SNIP_BLOCK_COL_32x1) col32_scales<A>(qa, tl, sh, *s32, tid, tx, ty, r0, c0, sa);
             if (B::kQuant && B::BLOCK == SNIP_BLOCK_COL_32x1) col32_scales<B>(qb, tl, sh, *s32, tid, tx, ty, r0, c0, sb);
         }
-        if (kBlk || (!(kRow || kRow32) && STATS)) {
+        if (kBlk || (!(kRow || kRow32 || kRow16) && STATS)) {
             uint32_t m = absmax2x(absmax2x(cm[0], cm[1]), absmax2x(cm[2], cm[3])) & 0x7FFF7FFFu;
             m = max(m & 0xFFFFu, m >> 16);
-            if (!(kRow || kRow32) && STATS) ts.amax = fmaxf(ts.amax, __uint_as_float(m << 16));
+            if (!(kRow || kRow32 || kRow16) && STATS) ts.amax = fmaxf(ts.amax, __uint_as_float(m << 16));
             if (kBlk) {
                 m = __reduce_max_sync(0xFFFFFFFFu, m);
                 if (lane == 0) sh.red_m[warp] = m;
@@ -625,6 +729,7 @@ __device__ __forceinline__ void process_tile(const QuantArgs &qa, const QuantArg
         stage_transposed<B::FMT>(sh.stage, tx, ty, keep);
         __syncthreads();
         write_transposed<B::FMT>(qb, sh.stage, r0, c0);
+        if (B::BLOCK == SNIP_BLOCK_COL_16x1) write_col16_atoms<B>(qb, tl, *s16, tid, c0);
     }
 }
 
@@ -741,6 +846,41 @@ __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel
             if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
             prefetch_commit();
         });
+        __syncthreads();
+    }
+    if (STATS) finish_stats<true>(ts, sh, d.a.partials, d.b.partials);
+}
+
+// Two-level option, both copies from one read: a = 1x16 tiles as stored, b = 16x1 tiles transposed, E2M1 codes.
+template <bool STATS>
+__global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_nvfp4_dual_kernel(const DualArgs d)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    QuantShared &sh = *reinterpret_cast<QuantShared *>(smem + kStageBytes);
+    QuantShared32 *s32 = reinterpret_cast<QuantShared32 *>(smem + kSmemBytes);   // holds this kernel's QuantShared16
+    const uint4 *slot = reinterpret_cast<const uint4 *>(smem) + threadIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (STATS) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    TwoLevel tw;
+    {
+        const float bound = *d.a.tensor_amax;
+        tw.enc = bound == 0.0f ? 1.0f : fminf(__fdiv_rn(2688.0f, bound), FLT_MAX);
+        tw.inv_enc = __fdiv_rn(1.0f, tw.enc);
+    }
+    ThreadStats ts;
+    TileWalk w((int)d.a.tiles_r, (int)d.a.tiles_c);
+    if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
+    prefetch_commit();
+    while (w.valid()) {
+        prefetch_wait<0>();
+        const Tile tl = {w.r, w.c, w.nr, w.nc};
+        w.next();
+        using A = Out<SNIP_FMT_FP4_E2M1, SNIP_BLOCK_ROW_1x16, false, true>;
+        using B = Out<SNIP_FMT_FP4_E2M1, SNIP_BLOCK_COL_16x1, true, true>;
+        process_tile<A, B, STATS, false>(d.a, d.b, tl, slot, sh, s32, ts, [&] {
+            if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
+            prefetch_commit();
+        }, tw);
         __syncthreads();
     }
     if (STATS) finish_stats<true>(ts, sh, d.a.partials, d.b.partials);
@@ -1102,7 +1242,79 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, in
     return SNIP_OK;
 }
 
+// Two-level option (see include/snip.h): both copies of a tensor from one read.
+int quantize_nvfp4_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax, void *codes_a, void *sf_a,
+                             snip_stats_t *stats_a, void *codes_b, void *sf_b, snip_stats_t *stats_b, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    if (!x || !tensor_amax || !codes_a || !sf_a || !codes_b || !sf_b) return SNIP_ERR_ARG;
+    if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
+    if ((stats_a == nullptr) != (stats_b == nullptr)) return SNIP_ERR_ARG;
+    if (!aligned16(x) || !aligned16(codes_a) || !aligned16(sf_a) || !aligned16(codes_b) || !aligned16(sf_b) ||
+        (reinterpret_cast<uintptr_t>(tensor_amax) & 3u) || (stats_a && ((reinterpret_cast<uintptr_t>(stats_a) | reinterpret_cast<uintptr_t>(stats_b)) & 7u)))
+        return SNIP_ERR_ALIGN;
+    const bool stats = stats_a != nullptr;
+    const size_t one = stats_ws_bytes(rows, cols, false);
+    if (stats && (!ws || ws_bytes < 2 * one)) return SNIP_ERR_WORKSPACE;
+    if (stats && !aligned16(ws)) return SNIP_ERR_ALIGN;
+    int rc = require_sm100();
+    if (rc != SNIP_OK) return rc;
+    const int64_t tr = ceil_div(rows, kTile), tc = ceil_div(cols, kTile);
+    DualArgs d;
+    void *codes[2] = {codes_a, codes_b}, *sf[2] = {sf_a, sf_b};
+    for (int i = 0; i < 2; ++i) {
+        QuantArgs &q = i ? d.b : d.a;
+        q.x = static_cast<const uint16_t *>(x);
+        q.rows = (int32_t)rows; q.cols = (int32_t)cols; q.ld = (int32_t)ld;
+        q.codes = static_cast<uint8_t *>(codes[i]);
+        q.scales = nullptr;
+        q.partials = stats ? reinterpret_cast<CtaPartial *>(static_cast<uint8_t *>(ws) + i * one) : nullptr;
+        q.row_partials = nullptr;
+        q.pow2 = 0;
+        q.seed = 0;
+        q.sf = static_cast<uint32_t *>(sf[i]);
+        q.tensor_amax = tensor_amax;
+        q.tiles_r = (int32_t)tr; q.tiles_c = (int32_t)tc; q.ntiles = tr * tc;
+    }
+    const int64_t nparts = persistent_ctas(tr * tc, kDualCtasPerSm);
+    dim3 grid((unsigned)nparts);
+    if (stats) launch_persistent(quantize_nvfp4_dual_kernel<true>, d, grid, st, kSmemBytes32);
+    else launch_persistent(quantize_nvfp4_dual_kernel<false>, d, grid, st, kSmemBytes32);
+    SNIP_CUDA_TRY(cudaGetLastError());
+    if (stats) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2);
+        cfg.blockDim = dim3(1024);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const ReduceSets sets = {{d.a.partials, d.b.partials}, {stats_a, stats_b}};
+        SNIP_CUDA_TRY(cudaLaunchKernelEx(&cfg, stats_reduce_kernel, sets, nparts));
+    }
+    return SNIP_OK;
+}
+
 }  // namespace snip
+
+extern "C" int snip_quantize_nvfp4_sizes(int64_t rows, int64_t cols, size_t *codes_bytes, size_t *sf_bytes)
+{
+    using namespace snip;
+    if (!valid_dim(rows) || !valid_dim(cols)) return SNIP_ERR_SHAPE;
+    // 64 bytes of tail slack after the codes of a ragged shape, as in snip_quantize_sizes
+    if (codes_bytes) *codes_bytes = (size_t)(rows * cols) / 2 + (((rows % 128) || (cols % 128)) ? 64 : 0);
+    if (sf_bytes) *sf_bytes = (size_t)(ceil_div(rows, 128) * ceil_div(cols, 128)) * 1024;
+    return SNIP_OK;
+}
+
+extern "C" int snip_quantize_nvfp4_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax, void *codes_stored,
+                                        void *sf_stored, snip_stats_t *stats_stored, void *codes_transposed, void *sf_transposed,
+                                        snip_stats_t *stats_transposed, void *ws, size_t ws_bytes, void *stream)
+{
+    return snip::quantize_nvfp4_dual_impl(x, rows, cols, ld, tensor_amax, codes_stored, sf_stored, stats_stored, codes_transposed, sf_transposed,
+                                          stats_transposed, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
 
 extern "C" int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int block, uint32_t flags,
                                    size_t *codes_bytes, size_t *scales_bytes, size_t *ws_bytes)

@@ -326,8 +326,13 @@ __host__ __device__ constexpr uint32_t make_idesc_block_scaled(uint32_t a_fmt, u
 {
     return (a_fmt << 7) | (b_fmt << 10) | ((N >> 3) << 17) | (1u << 23) | ((M >> 4) << 24);
 }
+// The same with E4M3 scale factors (bit 23 clear), as kind::mxf4nvf4 with scale_vec::4X takes them.
+__host__ __device__ constexpr uint32_t make_idesc_block_scaled_e4m3(uint32_t a_fmt, uint32_t b_fmt, uint32_t M, uint32_t N)
+{
+    return (a_fmt << 7) | (b_fmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
 
-enum class MmaKind { F16, F8F6F4, MXF4, MXF8 };   // MXF8 = kind::mxf8f6f4 with hardware block scales
+enum class MmaKind { F16, F8F6F4, MXF4, MXF8, NVF4 };   // MXF8 = kind::mxf8f6f4 with hardware block scales; NVF4 = kind::mxf4nvf4, E4M3 scale per 16
 
 template <MmaKind KIND, bool PAIR>
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
@@ -345,6 +350,11 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
     } else if constexpr (KIND == MmaKind::MXF8) {                                                                              \
         asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                                                       \
                      "tcgen05.mma.cta_group::" GROUP ".kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"        \
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)         \
+                     : "memory");                                                                                              \
+    } else if constexpr (KIND == MmaKind::NVF4) {                                                                              \
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"                                                       \
+                     "tcgen05.mma.cta_group::" GROUP ".kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}" \
                      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)         \
                      : "memory");                                                                                              \
     } else {                                                                                                                   \
