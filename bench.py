@@ -303,6 +303,58 @@ class Step:
                 gemm(api.OP_WGRAD, f, M, N, api.BLOCK_COL, 1, M, K, api.BLOCK_COL, 1, dw, fl)
 
 
+def run_two_level(step, events=None, qevents=None):
+    """The FP4 half of the step under the two-level (NVFP4-style) option: per linear three one-read two-output
+    quantizer calls (statistics on) and the three block-scaled GEMMs; the per-tensor bounds are the tensors' maxima,
+    computed once outside the timed region (a training loop would carry them over from the previous step)."""
+    api, torch = step.api, step.torch
+    if not hasattr(step, "codes"):
+        step._alloc_decomposed()
+    if not hasattr(step, "nv_bounds"):
+        step.nv_bounds = [tuple(t.float().abs().max().reshape(1).contiguous() for t in trip) for trip in step.inputs]
+        step.nv_sf = [torch.empty(api.snip_quantize_nvfp4_sizes(step.cfg.M, max(max(L.N, L.K) for L in step.cfg.linears))[1] + 4096, dtype=torch.uint8,
+                                  device=step.ws.device) for _ in range(6)]
+    lib, p, st = api._lib, api._p, api._stream()
+    F4 = api.FMT_FP4_E2M1
+    R, C = api.BLOCK_ROW16, api.BLOCK_COL16
+
+    def dual(x, bound, slot, stats_row):
+        r, c = x.shape
+        if qevents is not None:
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q0.record()
+        api._check("snip_quantize_nvfp4_dual", lib.snip_quantize_nvfp4_dual(p(x), r, c, c, p(bound), p(step.codes[slot]), p(step.nv_sf[slot]), p(stats_row[0:24]),
+                                                                         p(step.codes[slot + 1]), p(step.nv_sf[slot + 1]), p(stats_row[24:48]),
+                                                                         p(step.qws), step.qws.numel(), st))
+        if qevents is not None:
+            q1.record()
+            qevents.append((F4, (2.0 + 2.0 * (0.5 + 1.0 / 16.0)) * r * c, q0, q1))   # one bf16 read, two code + scale-byte outputs
+
+    def gemm(op, ra, ca, blka, ta, sa, ba, rb, cb_, blkb, tb, sb_, bb, out, flops):
+        a = api.make_qtensor(step.codes[sa], None, ra, ca, F4, blka, ta)
+        b = api.make_qtensor(step.codes[sb_], None, rb, cb_, F4, blkb, tb)
+        if events is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        api._check("snip_gemm_nvfp4", lib.snip_gemm_nvfp4(op, a, p(step.nv_sf[sa]), p(ba), b, p(step.nv_sf[sb_]), p(bb), p(out), api.OUT_BF16,
+                                                       p(step.gws), step.gws.numel(), st))
+        if events is not None:
+            e1.record()
+            events.append((F4, op, flops, e0, e1))
+
+    for i, (((x, w, dy), (y, dx, dw)), (bx, bw, bdy)) in enumerate(zip(zip(step.inputs, step.out), step.nv_bounds)):
+        M, K = x.shape
+        N = w.shape[0]
+        fl = 2.0 * M * N * K
+        srow = step.stats6[i].view(-1)
+        # slots: 0 X/1x16, 1 X/16x1^T, 2 W/1x16, 3 W/16x1^T, 4 dY/1x16, 5 dY/16x1^T
+        dual(x, bx, 0, srow[0:48]); dual(w, bw, 2, srow[48:96])
+        gemm(api.OP_FWD, M, K, R, 0, 0, bx, N, K, R, 0, 2, bw, y, fl)
+        dual(dy, bdy, 4, srow[96:144])
+        gemm(api.OP_DGRAD, M, N, R, 0, 4, bdy, N, K, C, 1, 3, bw, dx, fl)
+        gemm(api.OP_WGRAD, M, N, C, 1, 5, bdy, M, K, C, 1, 1, bx, dw, fl)
+
+
 class TaggedStep:
     """A table-driven workload (3B: each GEMM drawn FP4 / FP8 / BF16; 70B slice: at least 80 % of the linear-layer
     FLOPs in FP4, the rest FP8): `layers` layers resident, every linear's forward, input-gradient and weight-gradient
@@ -480,6 +532,55 @@ def run_profile_case(name):
     torch.cuda.set_device(0)
     device = torch.device("cuda", 0)
     parts = name.split("_")
+    if len(parts) > 1 and parts[1] == "nvfp4":
+        # two-level (NVFP4-style) option: quantize_nvfp4_dual | gemm_nvfp4_<fwd|dgrad|wgrad> on the 7B QKV shape
+        M, K, N = 16384, 4096, 12288
+        g = torch.Generator(device=device); g.manual_seed(3)
+        rnd = lambda r, c, sc: (torch.randn(r, c, generator=g, device=device, dtype=torch.float32) * sc).to(torch.bfloat16)
+        bound = lambda t: t.float().abs().max().reshape(1).contiguous()
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        times = []
+        if parts[0] == "quantize":
+            xs = [rnd(M, K, 1.0) for _ in range(3)]
+            bs = [bound(t) for t in xs]
+            bufs = api.snip_quantize_nvfp4_dual(xs[0], bs[0])
+            ws = torch.empty(api.snip_quantize_dual_workspace(M, K), dtype=torch.uint8, device=device)
+            for i in range(4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for j in range(6):
+                    api.snip_quantize_nvfp4_dual(xs[j % 3], bs[j % 3], bufs=bufs, ws=ws)
+                e1.record(); torch.cuda.synchronize()
+                if i >= 1: times.append(e0.elapsed_time(e1) / 6)
+            by = (2.0 + 2.0 * (0.5 + 1.0 / 16.0)) * M * K
+            print(f"{name}: {by / (min(times) * 1e-3) / 1e9:.0f} GB/s best of {len(times)}")
+            return
+        op = {"fwd": api.OP_FWD, "dgrad": api.OP_DGRAD, "wgrad": api.OP_WGRAD}[parts[2]]
+        R, C, F4 = api.BLOCK_ROW16, api.BLOCK_COL16, api.FMT_FP4_E2M1
+        if op == api.OP_FWD:
+            A, B, oshape = rnd(M, K, 1.0), rnd(N, K, 0.02), (M, N)
+            (qa, _), (qb, _) = api.snip_quantize_nvfp4_dual(A, bound(A), want_stats=False), api.snip_quantize_nvfp4_dual(B, bound(B), want_stats=False)
+            a, b = api.make_qtensor(qa["codes"], None, M, K, F4, R), api.make_qtensor(qb["codes"], None, N, K, F4, R)
+        elif op == api.OP_DGRAD:
+            A, B, oshape = rnd(M, N, 1e-3), rnd(N, K, 0.02), (M, K)
+            (qa, _), (_, qb) = api.snip_quantize_nvfp4_dual(A, bound(A), want_stats=False), api.snip_quantize_nvfp4_dual(B, bound(B), want_stats=False)
+            a, b = api.make_qtensor(qa["codes"], None, M, N, F4, R), api.make_qtensor(qb["codes"], None, N, K, F4, C, True)
+        else:
+            A, B, oshape = rnd(M, N, 1e-3), rnd(M, K, 1.0), (N, K)
+            (_, qa), (_, qb) = api.snip_quantize_nvfp4_dual(A, bound(A), want_stats=False), api.snip_quantize_nvfp4_dual(B, bound(B), want_stats=False)
+            a, b = api.make_qtensor(qa["codes"], None, M, N, F4, C, True), api.make_qtensor(qb["codes"], None, M, K, F4, C, True)
+        out = torch.empty(oshape, dtype=torch.bfloat16, device=device)
+        ws = torch.zeros(1024, dtype=torch.uint8, device=device)
+        ba, bb = bound(A), bound(B)
+        for i in range(4):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            api.snip_gemm_nvfp4(op, a, qa["sf"], ba, b, qb["sf"], bb, oshape, api.OUT_BF16, out=out, ws=ws)
+            e1.record(); torch.cuda.synchronize()
+            if i >= 1: times.append(e0.elapsed_time(e1))
+        print(f"{name}: {2.0 * M * N * K / (min(times) * 1e-3) / 1e12:.0f} TFLOP/s best of {len(times)}")
+        return
     if name.startswith("adamw"):
         n = 12288 * 4096
         ms_ = [torch.randn(n, device=device) * 1e-3 for _ in range(2)]
@@ -819,6 +920,28 @@ def main():
                               "gemm": {FMT_NAME[f]: {"tflops": d["flops"] / (d["ms"] * 1e-3) / 1e12,
                                                      "frac_of_sustained_peak": d["flops"] / (d["ms"] * 1e-3) / 1e12 / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[f])}
                                        for f, d in mx32_region.items()}}
+
+    # ---- the FP4 half of the step under the two-level (NVFP4-style) option ------------------------
+    for _ in range(3):
+        run_two_level(step)
+    barrier()
+    nv_events, nv_q = [], []
+    m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    m0.record()
+    for _ in range(args.steps):
+        run_two_level(step, nv_events, nv_q)
+    m1.record()
+    barrier()
+    flops_half = step.flops / len(step.formats)
+    ms_nv, flops_nv = combine_replicas(m0.elapsed_time(m1), flops_half, dist if world > 1 else None, device)
+    assert api.snip_poll_status(step.gws) == 0, "device-side timeout reported"
+    nv_g = sum(fl for _, _, fl, _, _ in nv_events) / (sum(a.elapsed_time(b) for _, _, _, a, b in nv_events) * 1e-3) / 1e12
+    nv_qgbs = sum(by for _, by, _, _ in nv_q) / (sum(a.elapsed_time(b) for _, _, a, b in nv_q) * 1e-3) / 1e9
+    pow2_option["two_level_fp4"] = {"value": flops_nv / (ms_nv / args.steps * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_nv / args.steps,
+                                    "note": "the FP4 half of the step (15 GEMMs) with E2M1 codes in 16-long tiles, E4M3 scale bytes and a per-tensor bound "
+                                            "(snip_quantize_nvfp4_dual + snip_gemm_nvfp4, kind::mxf4nvf4); an added option",
+                                    "gemm": {"tflops": nv_g, "frac_of_sustained_peak": nv_g / (peaks["bf16_tflops_sustained"] * NOMINAL_RATIO[FMT_FP4])},
+                                    "quantizer": {"gbs": nv_qgbs, "frac_of_hbm": nv_qgbs / peaks["hbm_gbs"]}}
 
     # ---- end to end: inputs start in pinned host memory, statistics come back -------------------
     e2e = None
