@@ -130,7 +130,8 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (warp == 0) {
         // ================= producer: operand tiles and scale-factor atoms =================
-        if (lane == 0) {
+        // (whole warp in the loop, one elected lane issues: see the MMA warp)
+        {
             uint32_t it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
@@ -139,73 +140,83 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int nb0 = 2 * n_idx, nb1 = min(2 * n_idx + 1, g.n_atoms_b - 1);
                 for (int ks = 0; ks < num_kstages; ++ks, ++it) {
                     const int s = it % S;
-                    if (!mbar_wait(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
-                    tma_load_2d(a_tile(s), &tmA, full_bar(s), ks * 128, m_idx * BM);
-                    tma_load_2d(b_tile(s), &tmB, full_bar(s), ks * 128, n_idx * BN);
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
+                    if (elect_one()) {
+                        mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
+                        tma_load_2d(a_tile(s), &tmA, full_bar(s), ks * 128, m_idx * BM);
+                        tma_load_2d(b_tile(s), &tmB, full_bar(s), ks * 128, n_idx * BN);
 #pragma unroll
-                    for (int h = 0; h < CPS; ++h) {
-                        const int c = min(ks * CPS + h, num_chunks - 1);   // a stage's unused second chunk reloads a valid atom
-                        const uint32_t dst = sf_tile(s) + h * C::kSfChunkBytes;
-                        if (C::kNv) {   // [A: two halves][B rows 0-127: two halves][B rows 128-255: two halves]
-                            bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 1024, 1024, full_bar(s));
-                            bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb0 * num_chunks + c) * 1024, 1024, full_bar(s));
-                            bulk_load_1d(dst + 2048, g.sfb + ((int64_t)nb1 * num_chunks + c) * 1024, 1024, full_bar(s));
-                        } else {
-                            bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 512, 512, full_bar(s));
-                            bulk_load_1d(dst + 512, g.sfb + ((int64_t)nb0 * num_chunks + c) * 512, 512, full_bar(s));
-                            bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb1 * num_chunks + c) * 512, 512, full_bar(s));
+                        for (int h = 0; h < CPS; ++h) {
+                            const int c = min(ks * CPS + h, num_chunks - 1);   // a stage's unused second chunk reloads a valid atom
+                            const uint32_t dst = sf_tile(s) + h * C::kSfChunkBytes;
+                            if (C::kNv) {   // [A: two halves][B rows 0-127: two halves][B rows 128-255: two halves]
+                                bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 1024, 1024, full_bar(s));
+                                bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb0 * num_chunks + c) * 1024, 1024, full_bar(s));
+                                bulk_load_1d(dst + 2048, g.sfb + ((int64_t)nb1 * num_chunks + c) * 1024, 1024, full_bar(s));
+                            } else {
+                                bulk_load_1d(dst, g.sfa + ((int64_t)m_idx * num_chunks + c) * 512, 512, full_bar(s));
+                                bulk_load_1d(dst + 512, g.sfb + ((int64_t)nb0 * num_chunks + c) * 512, 512, full_bar(s));
+                                bulk_load_1d(dst + 1024, g.sfb + ((int64_t)nb1 * num_chunks + c) * 512, 512, full_bar(s));
+                            }
                         }
                     }
+                    __syncwarp();
                 }
             }
         }
     } else if (warp == 1) {
         // ================= scale-factor copies and MMA issue =================
-        if (lane == 0) {
+        // The whole warp walks the loop and one elected lane issues: under `elect.sync` the operands of the tcgen05
+        // instructions stay in uniform registers, which makes each of them several times cheaper for the issuing thread than
+        // under a `lane == 0` branch; with up to seventeen of them per stage that thread is what the tensor core waits for.
+        {
             uint32_t it = 0, tiles_done = 0;
             bool ok = true;
             const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + (C::kNv ? kNvSfbCol : kSfbCol);
+            auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag)); };
             for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tiles_done) {
                 // the single accumulator must have been drained by the epilogue of the previous tile
-                if (!mbar_wait(tempty_bar, (tiles_done & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                if (!wait_all(tempty_bar, (tiles_done & 1u) ^ 1u)) { ok = false; break; }
                 tc_fence_after_sync();
                 for (int ks = 0; ks < num_kstages && ok; ++ks, ++it) {
                     const int s = it % S;
-                    if (!mbar_wait(full_bar(s), (it / S) & 1u, abort_flag)) { ok = false; break; }
+                    if (!wait_all(full_bar(s), (it / S) & 1u)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint64_t adesc = make_smem_desc_k128(a_tile(s));
                     const uint64_t bdesc = make_smem_desc_k128(b_tile(s));
+                    if (elect_one()) {
 #pragma unroll
-                    for (int h = 0; h < CPS; ++h) {
-                        if (ks * CPS + h < num_chunks) {
-                            const uint32_t sf = sf_tile(s) + h * C::kSfChunkBytes;
-                            if (C::kNv) {
-                                // MMA k of the chunk reads a whole word per line: SFA columns 4k.., SFB columns 8k.. (two 128-line groups)
-                                tmem_cp_sf_atom(sfa, sf);             tmem_cp_sf_atom(sfa + 4, sf + 512);
-                                tmem_cp_sf_atom(sfb, sf + 1024);      tmem_cp_sf_atom(sfb + 8, sf + 1536);
-                                tmem_cp_sf_atom(sfb + 4, sf + 2048);  tmem_cp_sf_atom(sfb + 12, sf + 2560);
-                            } else {
-                                tmem_cp_sf_atom(sfa, sf);
-                                tmem_cp_sf_atom(sfb, sf + 512);
-                                tmem_cp_sf_atom(sfb + 4, sf + 1024);
-                            }
-                            constexpr int kMmas = 4 / CPS;   // 32 bytes of K per MMA: four per 128-byte row
+                        for (int h = 0; h < CPS; ++h) {
+                            if (ks * CPS + h < num_chunks) {
+                                const uint32_t sf = sf_tile(s) + h * C::kSfChunkBytes;
+                                if (C::kNv) {
+                                    // MMA k of the chunk reads a whole word per line: SFA columns 4k.., SFB columns 8k.. (two 128-line groups)
+                                    tmem_cp_sf_atom(sfa, sf);             tmem_cp_sf_atom(sfa + 4, sf + 512);
+                                    tmem_cp_sf_atom(sfb, sf + 1024);      tmem_cp_sf_atom(sfb + 8, sf + 1536);
+                                    tmem_cp_sf_atom(sfb + 4, sf + 2048);  tmem_cp_sf_atom(sfb + 12, sf + 2560);
+                                } else {
+                                    tmem_cp_sf_atom(sfa, sf);
+                                    tmem_cp_sf_atom(sfb, sf + 512);
+                                    tmem_cp_sf_atom(sfb + 4, sf + 1024);
+                                }
+                                constexpr int kMmas = 4 / CPS;   // 32 bytes of K per MMA: four per 128-byte row
 #pragma unroll
-                            for (int k = 0; k < kMmas; ++k) {
-                                const int kk = h * kMmas + k;
-                                // which of the line's four scale bytes this MMA applies: byte k for the 32-long blocks of
-                                // kind::mxf8f6f4, bytes 2k and 2k+1 for the two halves of kind::mxf4's 64-long step
-                                // (descriptor fields b_sf_id at bit 4, a_sf_id at bit 29)
-                                const uint32_t sf_id = C::kNv ? 0u : (KIND == MmaKind::MXF4) ? 2u * k : (uint32_t)k;
-                                mma_ss<KIND, false>(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc | (sf_id << 4) | (sf_id << 29),
-                                                    (ks > 0 || kk > 0) ? 1u : 0u, sfa + (C::kNv ? 4 * k : 0), sfb + (C::kNv ? 8 * k : 0));
+                                for (int k = 0; k < kMmas; ++k) {
+                                    const int kk = h * kMmas + k;
+                                    // which of the line's four scale bytes this MMA applies: byte k for the 32-long blocks of
+                                    // kind::mxf8f6f4, bytes 2k and 2k+1 for the two halves of kind::mxf4's 64-long step
+                                    // (descriptor fields b_sf_id at bit 4, a_sf_id at bit 29); the two-level option reads whole words
+                                    const uint32_t sf_id = C::kNv ? 0u : (KIND == MmaKind::MXF4) ? 2u * k : (uint32_t)k;
+                                    mma_ss<KIND, false>(tmem_base, adesc + 2 * kk, bdesc + 2 * kk, idesc | (sf_id << 4) | (sf_id << 29),
+                                                        (ks > 0 || kk > 0) ? 1u : 0u, sfa + (C::kNv ? 4 * k : 0), sfb + (C::kNv ? 8 * k : 0));
+                                }
                             }
                         }
+                        tc_commit<false>(empty_bar(s));
+                        if (ks == num_kstages - 1) tc_commit<false>(tfull_bar);
                     }
-                    tc_commit<false>(empty_bar(s));
+                    __syncwarp();
                 }
-                if (ok) tc_commit<false>(tfull_bar);
             }
         }
     } else if (warp >= 4) {
