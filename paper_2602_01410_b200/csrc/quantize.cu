@@ -479,9 +479,10 @@ __device__ __forceinline__ uint32_t two_level_pair(float am0, float am1, const T
     return c;
 }
 
-// 1x16 tiles of the two-level option: a tile is the 8 columns of this lane and of its neighbour (lane ^ 1).  Both derive
-// the eight rows' factors; the even lane stages the scale bytes, and after a warp barrier lane tx of the row group
-// writes the atom word of row 8*ty + tx%8, half tx/8 (the bytes of that half's four tiles in order).
+// 1x16 tiles of the two-level option: a tile is the 8 columns of this lane and of its neighbour (lane ^ 1).  The two
+// share the work (four IEEE divisions per pair of tiles): the even lane derives the factors of rows 0..3, the odd lane
+// those of rows 4..7, each stages its scale bytes, and they swap the factors.  After a warp barrier lane tx of the row
+// group writes the atom word of row 8*ty + tx%8, half tx/8 (the bytes of that half's four tiles in order).
 template <class O>
 __device__ __forceinline__ void row16_scales(const QuantArgs &a, const Tile &tl, QuantShared16 &s16, const TwoLevel &tw, const uint32_t (&rmax)[8],
                                              int tx, int ty, int64_t rbase, SubScales &sc, float &amax_acc)
@@ -495,13 +496,22 @@ __device__ __forceinline__ void row16_scales(const QuantArgs &a, const Tile &tl,
         am[p] = __uint_as_float(mm << 16);
         amax_acc = fmaxf(amax_acc, am[p]);
     }
+    const bool odd = (tx & 1) != 0;
+    float e[4], n[4];
 #pragma unroll
-    for (int p = 0; p < 8; p += 2) {
-        const uint32_t c = two_level_pair(am[p], am[p + 1], tw, sc.s_row[p], sc.s_row[p + 1], sc.n_row[p], sc.n_row[p + 1]);
-        if (O::CODES && a.sf && !(tx & 1)) {
-            s16.row_sf[8 * ty + p][tx >> 1] = (uint8_t)(c & 0xFFu);
-            s16.row_sf[8 * ty + p + 1][tx >> 1] = (uint8_t)(c >> 8);
+    for (int i = 0; i < 4; i += 2) {
+        const uint32_t c = two_level_pair(odd ? am[4 + i] : am[i], odd ? am[5 + i] : am[i + 1], tw, e[i], e[i + 1], n[i], n[i + 1]);
+        if (O::CODES && a.sf) {
+            const int r = 8 * ty + (odd ? 4 : 0) + i;
+            s16.row_sf[r][tx >> 1] = (uint8_t)(c & 0xFFu);
+            s16.row_sf[r + 1][tx >> 1] = (uint8_t)(c >> 8);
         }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float eo = __shfl_xor_sync(0xFFFFFFFFu, e[i], 1), no = __shfl_xor_sync(0xFFFFFFFFu, n[i], 1);
+        sc.s_row[i] = odd ? eo : e[i];      sc.n_row[i] = odd ? no : n[i];
+        sc.s_row[4 + i] = odd ? e[i] : eo;  sc.n_row[4 + i] = odd ? n[i] : no;
     }
     if (O::CODES && a.sf) {
         __syncwarp();
@@ -513,20 +523,29 @@ __device__ __forceinline__ void row16_scales(const QuantArgs &a, const Tile &tl,
 
 // 16x1 tiles of the two-level option: a warp holds 16 rows, so after the exchange with lane ^ 16 (done by the caller)
 // cm holds the tile maxima of this lane's eight columns; the tile's index along the contraction is the warp's.
-// The scale bytes are staged for write_col16_atoms, which runs after the CTA barrier of the transposed output.
+// The two lanes share the work: lanes 0..15 derive the factors of columns 0..3, lanes 16..31 those of columns 4..7, and
+// they swap.  The scale bytes are staged for write_col16_atoms, which runs after the CTA barrier of the transposed output.
 template <class O>
 __device__ __forceinline__ void col16_scales(const QuantArgs &a, QuantShared16 &s16, const TwoLevel &tw, const uint32_t (&cm)[4], int lane, int tx,
                                              int warp, SubScales &sc)
 {
+    const bool upper = lane >= 16;
+    float e[4], n[4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const uint32_t m = cm[q] & 0x7FFF7FFFu;
-        const uint32_t c = two_level_pair(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u), tw, sc.s_col[2 * q], sc.s_col[2 * q + 1],
-                                          sc.n_col[2 * q], sc.n_col[2 * q + 1]);
-        if (O::CODES && a.sf && lane < 16) {
-            s16.col_sf[8 * tx + 2 * q][warp] = (uint8_t)(c & 0xFFu);
-            s16.col_sf[8 * tx + 2 * q + 1][warp] = (uint8_t)(c >> 8);
+    for (int q = 0; q < 2; ++q) {
+        const uint32_t m = (upper ? cm[2 + q] : cm[q]) & 0x7FFF7FFFu;
+        const uint32_t c = two_level_pair(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u), tw, e[2 * q], e[2 * q + 1], n[2 * q], n[2 * q + 1]);
+        if (O::CODES && a.sf) {
+            const int col = 8 * tx + (upper ? 4 : 0) + 2 * q;
+            s16.col_sf[col][warp] = (uint8_t)(c & 0xFFu);
+            s16.col_sf[col + 1][warp] = (uint8_t)(c >> 8);
         }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float eo = __shfl_xor_sync(0xFFFFFFFFu, e[i], 16), no = __shfl_xor_sync(0xFFFFFFFFu, n[i], 16);
+        sc.s_col[i] = upper ? eo : e[i];      sc.n_col[i] = upper ? no : n[i];
+        sc.s_col[4 + i] = upper ? e[i] : eo;  sc.n_col[4 + i] = upper ? n[i] : no;
     }
 }
 template <class O>
