@@ -325,7 +325,7 @@ def run_two_level(step, events=None, qevents=None):
             q0.record()
         api._check("snip_quantize_nvfp4_dual", lib.snip_quantize_nvfp4_dual(p(x), r, c, c, p(bound), p(step.codes[slot]), p(step.nv_sf[slot]), p(stats_row[0:24]),
                                                                          p(step.codes[slot + 1]), p(step.nv_sf[slot + 1]), p(stats_row[24:48]),
-                                                                         p(step.qws), step.qws.numel(), st))
+                                                                         0, 0, p(step.qws), step.qws.numel(), st))
         if qevents is not None:
             q1.record()
             qevents.append((F4, (2.0 + 2.0 * (0.5 + 1.0 / 16.0)) * r * c, q0, q1))   # one bf16 read, two code + scale-byte outputs

@@ -208,7 +208,8 @@ int snip_quantize_noalloc(const void *x, int64_t rows, int64_t cols, int64_t ld,
  * with independent formats, so codes, scales and statistics are bit-identical to those calls.
  * pow2_scale != 0 selects the power-of-two rule of snip_quantize_mx (and allows sf != NULL).
  * kind ROW32_COL32T (needs pow2_scale != 0): as_stored = (fmt, SNIP_BLOCK_ROW_1x32), transposed =
- * (fmt, SNIP_BLOCK_COL_32x1, SNIP_Q_TRANSPOSED), the block-32 form of snip_quantize_mx.
+ * (fmt, SNIP_BLOCK_COL_32x1, SNIP_Q_TRANSPOSED), the block-32 form of snip_quantize_mx; FP4 outputs of
+ * this kind may be rounded stochastically like those of kind ROW_COLT.
  * Algorithmic bytes per element: 2 + the two outputs' code and scale bytes, instead of 4 + those.
  * The paper does not prescribe how the copies are produced; it only fixes what they contain (Sec. 2.3).
  * ws_bytes >= snip_quantize_dual_workspace() when statistics are requested (else ws may be NULL).
@@ -324,7 +325,9 @@ int snip_gemm_mx(int op, const snip_qtensor_t *a_host, const void *sf_a, const s
  * the chunk], the word of tile line r (the bytes of its four tiles of that half, in order) at
  * (r % 32) * 16 + (r / 32) * 4; lines and tiles beyond the matrix hold 0.  snip_quantize_nvfp4_sizes gives
  * the byte sizes.  stats_* (device, may both be NULL): sum x^2, sum (x - dequantized)^2 and amax of each copy;
- * ws as for snip_quantize_dual.
+ * ws as for snip_quantize_dual.  rounding = SNIP_ROUND_STOCHASTIC rounds the E2M1 codes of both copies
+ * stochastically with `seed` (paper Sec. 6.1, meant for output gradients; rule and generator of snip_quantize_sr,
+ * applied to the same binary32 product); the scale bytes are not affected.
  * snip_gemm_nvfp4: the three products of snip_gemm_quantized over such operands (a / b: codes, rows, cols,
  * fmt = FP4, block = SNIP_BLOCK_ROW_1x16 or SNIP_BLOCK_COL_16x1 with transposed set, scales unused) on
  * tcgen05.mma kind::mxf4nvf4 with scale_vec::4X: the tensor core multiplies every 16 products by both scale
@@ -335,7 +338,7 @@ int snip_quantize_nvfp4_sizes(int64_t rows, int64_t cols, size_t *codes_bytes_ho
 int snip_quantize_nvfp4_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax,
                              void *codes_stored, void *sf_stored, snip_stats_t *stats_stored,
                              void *codes_transposed, void *sf_transposed, snip_stats_t *stats_transposed,
-                             void *ws, size_t ws_bytes, void *stream);
+                             int rounding, uint64_t seed, void *ws, size_t ws_bytes, void *stream);
 int snip_gemm_nvfp4(int op, const snip_qtensor_t *a_host, const void *sf_a, const float *amax_a,
                     const snip_qtensor_t *b_host, const void *sf_b, const float *amax_b, void *out,
                     int out_dtype, void *ws, size_t ws_bytes, void *stream);
@@ -396,7 +399,7 @@ int snip_layer_stats_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes
  * Results equal those of snip_linear_fwd / _dgrad / _wgrad (pow2_scale = 0) or snip_linear_mx
  * (pow2_scale = 1) called with the same tags.  pow2_scale = 2: power-of-two scales on 32-long tiles
  * along each GEMM's contraction for all three tensors (W too: 1x32 tiles for fwd, 32x1 tiles
- * transposed for dgrad; see the block-32 form of snip_quantize_mx); no stochastic rounding there.  stats6 (device, may be NULL): six snip_stats_t in the
+ * transposed for dgrad; see the block-32 form of snip_quantize_mx).  stats6 (device, may be NULL): six snip_stats_t in the
  * order X/1x128, X/128x1, W/fwd format, W/dgrad format, dY/1x128, dY/128x1.  out_dtype applies to all
  * three outputs.  dy_rounding = SNIP_ROUND_STOCHASTIC rounds the FP4 copies of dY stochastically with
  * dy_seed (Sec. 6.1; see snip_quantize_sr), FP8 copies stay nearest-even.  BF16 tags are not offered

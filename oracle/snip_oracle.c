@@ -437,8 +437,19 @@ static int orc_quantize_impl(const uint16_t *x, int64_t rows, int64_t cols, int 
  * sf[ceil(rows/16)][cols].  tensor_amax is an input (any positive bound of max|x| works; the exact maximum uses the
  * scale bytes' range best).  codes / sf / xhat / sumsq may be NULL.  Returns 0, or -1 on a bad argument.
  */
+int orc_quantize_nvfp4_sr(const uint16_t *x, int64_t rows, int64_t cols, int col_tiles, float tensor_amax, int stochastic, uint64_t seed,
+                          uint8_t *codes, uint8_t *sf, float *enc_out, double *xhat, double *sumsq);
+
 int orc_quantize_nvfp4(const uint16_t *x, int64_t rows, int64_t cols, int col_tiles, float tensor_amax,
                        uint8_t *codes, uint8_t *sf, float *enc_out, double *xhat, double *sumsq)
+{
+    return orc_quantize_nvfp4_sr(x, rows, cols, col_tiles, tensor_amax, 0, 0, codes, sf, enc_out, xhat, sumsq);
+}
+
+/* The same with the codes rounded stochastically (Sec. 6.1: FP4 output gradients), by the rule and generator of
+ * orc_quantize_sr applied to the product t; the scale bytes do not change. */
+int orc_quantize_nvfp4_sr(const uint16_t *x, int64_t rows, int64_t cols, int col_tiles, float tensor_amax, int stochastic, uint64_t seed,
+                          uint8_t *codes, uint8_t *sf, float *enc_out, double *xhat, double *sumsq)
 {
     if (!x || rows < 0 || cols < 0 || !(tensor_amax >= 0.0f)) return -1;
     const int64_t tl = 16;
@@ -474,7 +485,7 @@ int orc_quantize_nvfp4(const uint16_t *x, int64_t rows, int64_t cols, int col_ti
             if (sv != 0.0) {
                 volatile float E = enc / (float)sv;
                 volatile float t = xf * E;
-                code = orc_encode(&ORC_E2M1, t);
+                code = stochastic ? orc_encode_sr_fmt(&ORC_E2M1, t, orc_sr_uniform16(seed, (uint64_t)(r * cols + c))) : orc_encode(&ORC_E2M1, t);
             } else if (signbit(xf)) {
                 code = 0x8;   /* the sign survives, as it does for an underflowing product */
             }

@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.orc_quantize_rule.argtypes = [vp, i64, i64, i32, i32, i32, vp, vp, vp, vp, vp]
         L.orc_quantize_nvfp4.restype = i32
         L.orc_quantize_nvfp4.argtypes = [vp, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp]
+        L.orc_quantize_nvfp4_sr.restype = i32
+        L.orc_quantize_nvfp4_sr.argtypes = [vp, i64, i64, i32, ctypes.c_float, i32, ctypes.c_uint64, vp, vp, vp, vp, vp]
         L.orc_quantize_sr.restype = i32
         L.orc_quantize_sr.argtypes = [vp, i64, i64, i32, i32, i32, ctypes.c_uint64, vp, vp, vp, vp, vp]
         L.orc_philox4x32_10.restype = None
@@ -232,8 +234,8 @@ class QuantizedNvfp4:
         return pack_codes(self.codes, FMT_FP4_E2M1, transposed)
 
 
-def quantize_nvfp4(x_bits: np.ndarray, col_tiles: bool = False, tensor_amax: float | None = None) -> QuantizedNvfp4:
-    """tensor_amax = None: the exact maximum magnitude of x."""
+def quantize_nvfp4(x_bits: np.ndarray, col_tiles: bool = False, tensor_amax: float | None = None, sr_seed: int | None = None) -> QuantizedNvfp4:
+    """tensor_amax = None: the exact maximum magnitude of x.  sr_seed = an integer: codes rounded stochastically (Sec. 6.1)."""
     x = np.ascontiguousarray(x_bits, dtype=np.uint16)
     rows, cols = x.shape
     if tensor_amax is None:
@@ -244,8 +246,8 @@ def quantize_nvfp4(x_bits: np.ndarray, col_tiles: bool = False, tensor_amax: flo
     enc = np.zeros(1, dtype=np.float32)
     xhat = np.empty((rows, cols), dtype=np.float64)
     sumsq = np.zeros(2, dtype=np.float64)
-    rc = lib().orc_quantize_nvfp4(_ptr(x), rows, cols, int(col_tiles), ctypes.c_float(tensor_amax), _ptr(codes), _ptr(sf), _ptr(enc),
-                                  _ptr(xhat), _ptr(sumsq))
+    rc = lib().orc_quantize_nvfp4_sr(_ptr(x), rows, cols, int(col_tiles), ctypes.c_float(tensor_amax), int(sr_seed is not None),
+                                     0 if sr_seed is None else sr_seed, _ptr(codes), _ptr(sf), _ptr(enc), _ptr(xhat), _ptr(sumsq))
     if rc != 0:
         raise ValueError("orc_quantize_nvfp4: bad argument")
     return QuantizedNvfp4(rows, cols, bool(col_tiles), codes, sf, enc[0], xhat, float(sumsq[0]), float(sumsq[1]))

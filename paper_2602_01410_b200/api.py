@@ -84,7 +84,7 @@ def _load():
     lib.snip_gemm_quantized.argtypes = [i32, ctypes.POINTER(QTensor), ctypes.POINTER(QTensor), vp, i32, i32, vp, sz, vp]
     lib.snip_gemm_mx.argtypes = [i32, ctypes.POINTER(QTensor), vp, ctypes.POINTER(QTensor), vp, vp, i32, vp, sz, vp]
     lib.snip_quantize_nvfp4_sizes.argtypes = [i64, i64, psz, psz]
-    lib.snip_quantize_nvfp4_dual.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.snip_quantize_nvfp4_dual.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, i32, ctypes.c_uint64, vp, sz, vp]
     lib.snip_gemm_nvfp4.argtypes = [i32, ctypes.POINTER(QTensor), vp, vp, ctypes.POINTER(QTensor), vp, vp, vp, i32, vp, sz, vp]
     lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_fwd.argtypes = lin
@@ -308,7 +308,7 @@ def snip_quantize_nvfp4_sizes(rows, cols):
     return cb.value, sb.value
 
 
-def snip_quantize_nvfp4_dual(x: torch.Tensor, tensor_amax: torch.Tensor, *, want_stats=True, bufs=None, ws=None):
+def snip_quantize_nvfp4_dual(x: torch.Tensor, tensor_amax: torch.Tensor, *, want_stats=True, bufs=None, ws=None, sr_seed=None):
     """Two-level option, both copies from one read.  tensor_amax: float32 CUDA tensor with one element (the bound of |x|).
     Returns two dicts (as stored, transposed) with codes / sf / stats tensors."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
@@ -323,8 +323,9 @@ def snip_quantize_nvfp4_dual(x: torch.Tensor, tensor_amax: torch.Tensor, *, want
         ws = torch.empty(snip_quantize_dual_workspace(rows, cols), dtype=torch.uint8, device=dev)
     a, b = bufs
     _check("snip_quantize_nvfp4_dual", _lib.snip_quantize_nvfp4_dual(_p(x), rows, cols, x.stride(0), _p(tensor_amax), _p(a["codes"]), _p(a["sf"]),
-                                                                     _p(a["stats"]), _p(b["codes"]), _p(b["sf"]), _p(b["stats"]), _p(ws),
-                                                                     0 if ws is None else ws.numel(), _stream()))
+                                                                     _p(a["stats"]), _p(b["codes"]), _p(b["sf"]), _p(b["stats"]),
+                                                                     ROUND_NEAREST_EVEN if sr_seed is None else ROUND_STOCHASTIC, 0 if sr_seed is None else sr_seed,
+                                                                     _p(ws), 0 if ws is None else ws.numel(), _stream()))
     return a, b
 
 

@@ -274,7 +274,6 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
     const bool mx = pow2_scale != 0;
     const int fmt[6] = {fmt_fwd, fmt_wgrad, fmt_fwd, fmt_dgrad, fmt_dgrad, fmt_wgrad};
     const FwdBwdCarve f = carve_fwd_bwd(ws, M, N, K, fmt, pow2_scale);
-    if (pow2_scale == 2 && dy_rounding == SNIP_ROUND_STOCHASTIC) return SNIP_ERR_UNSUPPORTED;
     const int kind_xdy = pow2_scale == 2 ? SNIP_DUAL_ROW32_COL32T : SNIP_DUAL_ROW_COLT;
     const int kind_w = pow2_scale == 2 ? SNIP_DUAL_ROW32_COL32T : SNIP_DUAL_BLK_BLKT;
     if (dy_rounding != SNIP_ROUND_NEAREST_EVEN && dy_rounding != SNIP_ROUND_STOCHASTIC) return SNIP_ERR_ARG;

@@ -871,7 +871,7 @@ __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_dual_kernel
 }
 
 // Two-level option, both copies from one read: a = 1x16 tiles as stored, b = 16x1 tiles transposed, E2M1 codes.
-template <bool STATS>
+template <bool STATS, bool SR = false>
 __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_nvfp4_dual_kernel(const DualArgs d)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -894,8 +894,8 @@ __global__ void __launch_bounds__(kThreads, kDualCtasPerSm) quantize_nvfp4_dual_
         prefetch_wait<0>();
         const Tile tl = {w.r, w.c, w.nr, w.nc};
         w.next();
-        using A = Out<SNIP_FMT_FP4_E2M1, SNIP_BLOCK_ROW_1x16, false, true>;
-        using B = Out<SNIP_FMT_FP4_E2M1, SNIP_BLOCK_COL_16x1, true, true>;
+        using A = Out<SNIP_FMT_FP4_E2M1, SNIP_BLOCK_ROW_1x16, false, true, SR>;
+        using B = Out<SNIP_FMT_FP4_E2M1, SNIP_BLOCK_COL_16x1, true, true, SR>;
         process_tile<A, B, STATS, false>(d.a, d.b, tl, slot, sh, s32, ts, [&] {
             if (w.valid()) prefetch_tile(d.a, w.r, w.c, smem);
             prefetch_commit();
@@ -1175,11 +1175,11 @@ static void launch_dual(const DualArgs &d, bool blk, bool stats, dim3 grid, cuda
     else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false>, d, grid, st);
 }
 
-template <int FMT_A, int FMT_B>
+template <int FMT_A, int FMT_B, bool SR_A = false, bool SR_B = false>
 static void launch_dual32(const DualArgs &d, bool stats, dim3 grid, cudaStream_t st)
 {
-    if (stats) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, true, false, false, true>, d, grid, st, kSmemBytes32);
-    else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false, false, false, true>, d, grid, st, kSmemBytes32);
+    if (stats) launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, true, SR_A, SR_B, true>, d, grid, st, kSmemBytes32);
+    else launch_persistent(quantize_dual_kernel<FMT_A, FMT_B, false, false, SR_A, SR_B, true>, d, grid, st, kSmemBytes32);
 }
 
 // kind: SNIP_DUAL_ROW_COLT, SNIP_DUAL_BLK_BLKT or SNIP_DUAL_ROW32_COL32T (power-of-two scales only).
@@ -1188,7 +1188,7 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, in
 {
     if (!x) return SNIP_ERR_ARG;
     const bool blk = kind == SNIP_DUAL_BLK_BLKT, sub32 = kind == SNIP_DUAL_ROW32_COL32T;
-    if (sub32 && (!pow2 || oa.sr || ob.sr)) return SNIP_ERR_UNSUPPORTED;
+    if (sub32 && !pow2) return SNIP_ERR_UNSUPPORTED;
     if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
     const DualOut *o[2] = {&oa, &ob};
     for (int i = 0; i < 2; ++i) {
@@ -1226,7 +1226,14 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, in
     dim3 grid((unsigned)nparts);
     const bool a8 = oa.fmt == SNIP_FMT_FP8_E4M3, b8 = ob.fmt == SNIP_FMT_FP8_E4M3;
     constexpr int F8 = SNIP_FMT_FP8_E4M3, F4 = SNIP_FMT_FP4_E2M1;
-    if (sub32) {
+    if (sub32 && (oa.sr || ob.sr)) {
+        if ((oa.sr && a8) || (ob.sr && b8)) return SNIP_ERR_UNSUPPORTED;   // stochastic rounding is offered for FP4 codes
+        if (oa.sr && ob.sr) launch_dual32<F4, F4, true, true>(d, stats, grid, st);
+        else if (oa.sr && b8) launch_dual32<F4, F8, true, false>(d, stats, grid, st);
+        else if (oa.sr) launch_dual32<F4, F4, true, false>(d, stats, grid, st);
+        else if (a8) launch_dual32<F8, F4, false, true>(d, stats, grid, st);
+        else launch_dual32<F4, F4, false, true>(d, stats, grid, st);
+    } else if (sub32) {
         if (a8 && b8) launch_dual32<F8, F8>(d, stats, grid, st);
         else if (a8) launch_dual32<F8, F4>(d, stats, grid, st);
         else if (b8) launch_dual32<F4, F8>(d, stats, grid, st);
@@ -1263,8 +1270,11 @@ int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, in
 
 // Two-level option (see include/snip.h): both copies of a tensor from one read.
 int quantize_nvfp4_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax, void *codes_a, void *sf_a,
-                             snip_stats_t *stats_a, void *codes_b, void *sf_b, snip_stats_t *stats_b, void *ws, size_t ws_bytes, cudaStream_t st)
+                             snip_stats_t *stats_a, void *codes_b, void *sf_b, snip_stats_t *stats_b, int rounding, uint64_t seed, void *ws,
+                             size_t ws_bytes, cudaStream_t st)
 {
+    if (rounding != SNIP_ROUND_NEAREST_EVEN && rounding != SNIP_ROUND_STOCHASTIC) return SNIP_ERR_ARG;
+    const bool sr = rounding == SNIP_ROUND_STOCHASTIC;
     if (!x || !tensor_amax || !codes_a || !sf_a || !codes_b || !sf_b) return SNIP_ERR_ARG;
     if (!valid_dim(rows) || !valid_dim(cols) || ld < cols || (ld % 8) != 0 || rows > INT32_MAX || ld > INT32_MAX) return SNIP_ERR_SHAPE;
     if ((stats_a == nullptr) != (stats_b == nullptr)) return SNIP_ERR_ARG;
@@ -1289,15 +1299,17 @@ int quantize_nvfp4_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t 
         q.partials = stats ? reinterpret_cast<CtaPartial *>(static_cast<uint8_t *>(ws) + i * one) : nullptr;
         q.row_partials = nullptr;
         q.pow2 = 0;
-        q.seed = 0;
+        q.seed = seed;
         q.sf = static_cast<uint32_t *>(sf[i]);
         q.tensor_amax = tensor_amax;
         q.tiles_r = (int32_t)tr; q.tiles_c = (int32_t)tc; q.ntiles = tr * tc;
     }
     const int64_t nparts = persistent_ctas(tr * tc, kDualCtasPerSm);
     dim3 grid((unsigned)nparts);
-    if (stats) launch_persistent(quantize_nvfp4_dual_kernel<true>, d, grid, st, kSmemBytes32);
-    else launch_persistent(quantize_nvfp4_dual_kernel<false>, d, grid, st, kSmemBytes32);
+    if (stats && sr) launch_persistent(quantize_nvfp4_dual_kernel<true, true>, d, grid, st, kSmemBytes32);
+    else if (stats) launch_persistent(quantize_nvfp4_dual_kernel<true, false>, d, grid, st, kSmemBytes32);
+    else if (sr) launch_persistent(quantize_nvfp4_dual_kernel<false, true>, d, grid, st, kSmemBytes32);
+    else launch_persistent(quantize_nvfp4_dual_kernel<false, false>, d, grid, st, kSmemBytes32);
     SNIP_CUDA_TRY(cudaGetLastError());
     if (stats) {
         cudaLaunchConfig_t cfg = {};
@@ -1329,10 +1341,10 @@ extern "C" int snip_quantize_nvfp4_sizes(int64_t rows, int64_t cols, size_t *cod
 
 extern "C" int snip_quantize_nvfp4_dual(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax, void *codes_stored,
                                         void *sf_stored, snip_stats_t *stats_stored, void *codes_transposed, void *sf_transposed,
-                                        snip_stats_t *stats_transposed, void *ws, size_t ws_bytes, void *stream)
+                                        snip_stats_t *stats_transposed, int rounding, uint64_t seed, void *ws, size_t ws_bytes, void *stream)
 {
     return snip::quantize_nvfp4_dual_impl(x, rows, cols, ld, tensor_amax, codes_stored, sf_stored, stats_stored, codes_transposed, sf_transposed,
-                                          stats_transposed, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+                                          stats_transposed, rounding, seed, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int snip_quantize_sizes(int64_t rows, int64_t cols, int fmt, int block, uint32_t flags,

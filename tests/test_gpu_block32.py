@@ -151,3 +151,20 @@ def test_7b_activation_tensor_bit_exact(api):
     torch.cuda.synchronize()
     check_output(api, a["codes"], a["scales"], a["sf"], a["stats"], orc.quantize(x, FP4, orc.BLOCK_ROW32, True), False)
     check_output(api, b["codes"], b["scales"], b["sf"], b["stats"], orc.quantize(x, FP8, orc.BLOCK_COL32, True), True)
+
+
+@pytest.mark.parametrize("shape", [(256, 384), (320, 448)])
+def test_stochastic_rounding_of_fp4_outputs(api, shape):
+    # Sec. 6.1: FP4 output gradients are rounded stochastically; the 32-long tile kinds take the same rule and generator
+    rows, cols = shape
+    x = spread_inputs(np.random.default_rng(rows + 3 * cols), rows, cols)
+    seeds = (77, 0xFEEDFACE1)
+    a, b = api.snip_quantize_dual(to_dev(x), api.DUAL_ROW32_COL32T, FP4, FP4, pow2_scale=True, want_sf=True, sr_seeds=seeds)
+    torch.cuda.synchronize()
+    check_output(api, a["codes"], a["scales"], a["sf"], a["stats"], orc.quantize(x, FP4, orc.BLOCK_ROW32, True, sr_seed=seeds[0]), False)
+    check_output(api, b["codes"], b["scales"], b["sf"], b["stats"], orc.quantize(x, FP4, orc.BLOCK_COL32, True, sr_seed=seeds[1]), True)
+    # one stochastic FP4 output next to a nearest-even FP8 output
+    a, b = api.snip_quantize_dual(to_dev(x), api.DUAL_ROW32_COL32T, FP8, FP4, pow2_scale=True, want_sf=True, sr_seeds=(None, 5))
+    torch.cuda.synchronize()
+    check_output(api, a["codes"], a["scales"], a["sf"], a["stats"], orc.quantize(x, FP8, orc.BLOCK_ROW32, True), False)
+    check_output(api, b["codes"], b["scales"], b["sf"], b["stats"], orc.quantize(x, FP4, orc.BLOCK_COL32, True, sr_seed=5), True)

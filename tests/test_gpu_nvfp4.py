@@ -142,3 +142,19 @@ def test_7b_activation_tensor_bit_exact(api):
     torch.cuda.synchronize()
     check_copy(api, a, orc.quantize_nvfp4(x, False), False)
     check_copy(api, b, orc.quantize_nvfp4(x, True), True)
+
+
+@pytest.mark.parametrize("shape", [(256, 384), (320, 448)])
+def test_stochastic_rounding_bit_exact(api, shape):
+    # Sec. 6.1: output gradients in FP4 are rounded stochastically; same rule and generator as snip_quantize_sr
+    rows, cols = shape
+    x = spread(np.random.default_rng(rows + 5 * cols), rows, cols, 1e-3)
+    seed = 0x1234ABCD5
+    a, b = api.snip_quantize_nvfp4_dual(to_dev(x), dev_f32(amax_of(x)), sr_seed=seed)
+    torch.cuda.synchronize()
+    check_copy(api, a, orc.quantize_nvfp4(x, False, sr_seed=seed), False)
+    check_copy(api, b, orc.quantize_nvfp4(x, True, sr_seed=seed), True)
+    a2, b2 = api.snip_quantize_nvfp4_dual(to_dev(x), dev_f32(amax_of(x)), sr_seed=seed + 1)
+    torch.cuda.synchronize()
+    n = rows * cols // 2
+    assert not torch.equal(a["codes"][:n], a2["codes"][:n]) and torch.equal(a["sf"], a2["sf"])

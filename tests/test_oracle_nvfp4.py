@@ -187,3 +187,35 @@ def test_gemms_match_explicit_sums_over_tiles():
     assert qdyc.col_tiles and qxc.col_tiles
     ref = qdyc.xhat.T @ qxc.xhat
     assert np.abs(dw - ref).max() <= 1e-12 * np.abs(ref).max()
+
+
+def test_stochastic_codes_follow_the_rule_and_are_unbiased():
+    # Sec. 6.1: the product t = x * E goes to one of its two neighbours on the E2M1 grid, up iff (t - lo)/(hi - lo) > (u + 1/2)/2^16
+    rng = np.random.default_rng(36)
+    x = data(rng, 6, 64, 0.05)
+    xf = orc.bf16_to_float(x).astype(np.float64)
+    q0 = orc.quantize_nvfp4(x)
+    grid = [0, 0.5, 1, 1.5, 2, 3, 4, 6]
+    seed = 1234
+    q = orc.quantize_nvfp4(x, sr_seed=seed)
+    assert np.array_equal(q.sf, q0.sf) and q.enc == q0.enc          # the scale bytes do not depend on the rounding
+    for r in range(6):
+        for c in range(64):
+            sv = orc.decode_code(FP8, int(q.sf[c // 16, r]))
+            t = f32(xf[r, c]) * (q.enc / f32(sv))
+            a = min(abs(float(t)), 6.0)
+            lo = max(g for g in grid if g <= a)
+            hi = min([g for g in grid if g > a], default=lo)
+            u = orc.sr_uniform16(seed, r * 64 + c)
+            up = hi > lo and (Fraction(a) - Fraction(lo)) / (Fraction(hi) - Fraction(lo)) > Fraction(2 * u + 1, 131072)
+            want = (hi if up else lo) * (-1.0 if np.signbit(t) else 1.0)
+            assert orc.decode_code(FP4, int(q.codes[r, c])) == want, (r, c)
+    # the mean over seeds approaches x wherever the value does not saturate
+    acc = np.zeros_like(xf)
+    n = 400
+    for s in range(n):
+        acc += orc.quantize_nvfp4(x, sr_seed=1000 + s).xhat
+    v8 = np.vectorize(lambda c: orc.decode_code(FP8, int(c)))
+    unit = v8(q0.sf).T.repeat(16, axis=1) / float(q0.enc)
+    inside = np.abs(xf) <= 6.0 * unit
+    assert (np.abs(acc / n - xf)[inside] <= 2.0 * unit[inside] * 4.0 / np.sqrt(n)).all()   # 4 sigma of a step of at most 2 units
