@@ -342,6 +342,18 @@ int snip_quantize_nvfp4_dual(const void *x, int64_t rows, int64_t cols, int64_t 
 int snip_gemm_nvfp4(int op, const snip_qtensor_t *a_host, const void *sf_a, const float *amax_a,
                     const snip_qtensor_t *b_host, const void *sf_b, const float *amax_b, void *out,
                     int out_dtype, void *ws, size_t ws_bytes, void *stream);
+/*
+ * One linear layer, forward and both gradients, under the two-level option (the composition of
+ * snip_linear_fwd_bwd): X, W and dY each go through snip_quantize_nvfp4_dual once, then Y = X W^T, dX = dY W,
+ * dW = dY^T X through snip_gemm_nvfp4.  bounds3 (device): the magnitude bounds of X, W and dY, in this order.
+ * dy_rounding / dy_seed: stochastic rounding of both copies of dY (Sec. 6.1).  stats6 (device, may be NULL):
+ * X/1x16, X/16x1, W/1x16, W/16x1, dY/1x16, dY/16x1.
+ */
+int snip_linear_fwd_bwd_nvfp4_workspace(int64_t M, int64_t N, int64_t K, size_t *ws_bytes_host);
+int snip_linear_fwd_bwd_nvfp4(const void *X, const void *W, const void *dY, void *Y, void *dX, void *dW,
+                              int64_t M, int64_t N, int64_t K, int out_dtype, const float *bounds3,
+                              int dy_rounding, uint64_t dy_seed, snip_stats_t *stats6, void *ws,
+                              size_t ws_bytes, void *stream);
 
 /*
  * One linear layer's forward GEMM under a precision choice: quantize X (1x128 tiles along K)

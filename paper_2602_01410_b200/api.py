@@ -26,7 +26,7 @@ LIB_PATH = os.environ.get("SNIP_B200_LIB") or os.path.join(os.path.dirname(os.pa
 
 EXPORTS = (
     "snip_version", "snip_status_string", "snip_last_cuda_error", "snip_quantize_sizes",
-    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_quantize_nvfp4_sizes", "snip_quantize_nvfp4_dual", "snip_gemm_nvfp4", "snip_linear_fwd",
+    "snip_quantize", "snip_quantize_noalloc", "snip_quantize_mx_sizes", "snip_quantize_mx", "snip_quantize_dual_workspace", "snip_quantize_dual", "snip_quantize_sr", "snip_workspace_size", "snip_gemm_quantized", "snip_gemm_mx", "snip_quantize_nvfp4_sizes", "snip_quantize_nvfp4_dual", "snip_gemm_nvfp4", "snip_linear_fwd_bwd_nvfp4_workspace", "snip_linear_fwd_bwd_nvfp4", "snip_linear_fwd",
     "snip_linear_dgrad", "snip_linear_wgrad", "snip_linear_mx", "snip_linear_mx_workspace", "snip_linear_fwd_bwd_workspace", "snip_linear_fwd_bwd", "snip_layer_stats", "snip_layer_stats_workspace", "snip_adamw_sensitivity_workspace", "snip_adamw_sensitivity", "snip_loss_divergence", "snip_weight_divergence", "snip_select_scheme",
     "snip_poll_status", "snip_debug_set",
 )
@@ -86,6 +86,8 @@ def _load():
     lib.snip_quantize_nvfp4_sizes.argtypes = [i64, i64, psz, psz]
     lib.snip_quantize_nvfp4_dual.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, i32, ctypes.c_uint64, vp, sz, vp]
     lib.snip_gemm_nvfp4.argtypes = [i32, ctypes.POINTER(QTensor), vp, vp, ctypes.POINTER(QTensor), vp, vp, vp, i32, vp, sz, vp]
+    lib.snip_linear_fwd_bwd_nvfp4_workspace.argtypes = [i64, i64, i64, psz]
+    lib.snip_linear_fwd_bwd_nvfp4.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i32, vp, i32, ctypes.c_uint64, vp, vp, sz, vp]
     lin = [vp, vp, vp, i64, i64, i64, i32, i32, i32, vp, vp, vp, sz, vp]
     lib.snip_linear_fwd.argtypes = lin
     lib.snip_linear_dgrad.argtypes = lin
@@ -428,6 +430,25 @@ def snip_linear_fwd_bwd(x, w, dy, fmt_fwd, fmt_dgrad, fmt_wgrad, out_dtype=OUT_B
     _check("snip_linear_fwd_bwd", _lib.snip_linear_fwd_bwd(_p(x), _p(w), _p(dy), _p(y), _p(dx), _p(dw), M, N, K, fmt_fwd, fmt_dgrad, fmt_wgrad,
                                                            out_dtype, int(pow2_scale), ROUND_NEAREST_EVEN if dy_sr_seed is None else ROUND_STOCHASTIC,
                                                            0 if dy_sr_seed is None else dy_sr_seed, _p(stats), _p(ws), ws.numel(), _stream()))
+    return y, dx, dw, stats
+
+
+def snip_linear_fwd_bwd_nvfp4(x, w, dy, bounds3, out_dtype=OUT_BF16, *, dy_sr_seed=None, stats=None, ws=None):
+    """Forward and both gradients under the two-level option.  bounds3: float32 CUDA tensor [3] (bounds of |X|, |W|, |dY|).
+    Returns (y, dx, dw, stats) with stats a uint8 tensor holding six 24-byte snip_stats_t."""
+    M, K = x.shape
+    N = w.shape[0]
+    dev = x.device
+    y, dx, dw = _out((M, N), out_dtype, dev, None), _out((M, K), out_dtype, dev, None), _out((N, K), out_dtype, dev, None)
+    if stats is None:
+        stats = torch.zeros(6 * 24, dtype=torch.uint8, device=dev)
+    if ws is None:
+        n = ctypes.c_size_t()
+        _check("snip_linear_fwd_bwd_nvfp4_workspace", _lib.snip_linear_fwd_bwd_nvfp4_workspace(M, N, K, ctypes.byref(n)))
+        ws = torch.zeros(n.value, dtype=torch.uint8, device=dev)
+    _check("snip_linear_fwd_bwd_nvfp4", _lib.snip_linear_fwd_bwd_nvfp4(_p(x), _p(w), _p(dy), _p(y), _p(dx), _p(dw), M, N, K, out_dtype, _p(bounds3),
+                                                                       ROUND_NEAREST_EVEN if dy_sr_seed is None else ROUND_STOCHASTIC,
+                                                                       0 if dy_sr_seed is None else dy_sr_seed, _p(stats), _p(ws), ws.numel(), _stream()))
     return y, dx, dw, stats
 
 

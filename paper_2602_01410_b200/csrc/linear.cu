@@ -20,6 +20,12 @@ size_t gemm_ws_bytes();
 size_t gemm_ws_bytes_sliced();   // with room for the weight-gradient product's contraction slices
 int quantize_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, int kind, int pow2, const DualOut &oa, const DualOut &ob,
                        void *ws, size_t ws_bytes, cudaStream_t st);
+int quantize_nvfp4_dual_impl(const void *x, int64_t rows, int64_t cols, int64_t ld, const float *tensor_amax, void *codes_a, void *sf_a,
+                             snip_stats_t *stats_a, void *codes_b, void *sf_b, snip_stats_t *stats_b, int rounding, uint64_t seed, void *ws,
+                             size_t ws_bytes, cudaStream_t st);
+int gemm_nvfp4_impl(const void *a_codes, const void *b_codes, const void *sfa, const void *sfb, const float *amax_a, const float *amax_b,
+                    int64_t Mo, int64_t No, int64_t Kc, void *out, int out_dtype, void *ws, size_t ws_bytes, cudaStream_t st, bool clear_status);
+int gemm_clear_status(void *ws, cudaStream_t st);
 
 namespace {
 
@@ -308,4 +314,81 @@ extern "C" int snip_linear_fwd_bwd(const void *X, const void *W, const void *dY,
     rc = gemm(SNIP_OP_DGRAD, 4, 3, dX);
     if (rc) return rc;
     return gemm(SNIP_OP_WGRAD, 5, 1, dW);
+}
+
+// ---- the same composition under the two-level (NVFP4-style) option ---------------------------------
+
+namespace snip {
+namespace {
+struct NvCarve {
+    void *gws;
+    void *codes[6];
+    void *sf[6];
+    void *stats_ws;
+    size_t stats_ws_bytes, total;
+};
+NvCarve carve_nvfp4(void *ws, int64_t M, int64_t N, int64_t K)
+{
+    // index: 0 X/1x16, 1 X/16x1^T, 2 W/1x16, 3 W/16x1^T, 4 dY/1x16, 5 dY/16x1^T
+    const int64_t rows[6] = {M, M, N, N, M, M}, cols[6] = {K, K, K, K, N, N};
+    NvCarve f{};
+    Carve c(ws, 0);
+    f.gws = c.take(gemm_ws_bytes());
+    size_t sb = 0;
+    for (int i = 0; i < 6; ++i) {
+        size_t cb = 0, fb = 0;
+        snip_quantize_nvfp4_sizes(rows[i], cols[i], &cb, &fb);
+        f.codes[i] = c.take(cb);
+        f.sf[i] = c.take(fb);
+        size_t w = 0;
+        snip_quantize_dual_workspace(rows[i], cols[i], &w);
+        if (w > sb) sb = w;
+    }
+    f.stats_ws = c.take(sb);
+    f.stats_ws_bytes = sb;
+    f.total = c.off;
+    return f;
+}
+}  // namespace
+}  // namespace snip
+
+extern "C" int snip_linear_fwd_bwd_nvfp4_workspace(int64_t M, int64_t N, int64_t K, size_t *bytes)
+{
+    using namespace snip;
+    if (!bytes) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    *bytes = carve_nvfp4(nullptr, M, N, K).total;
+    return SNIP_OK;
+}
+
+extern "C" int snip_linear_fwd_bwd_nvfp4(const void *X, const void *W, const void *dY, void *Y, void *dX, void *dW, int64_t M, int64_t N, int64_t K,
+                                         int out_dtype, const float *bounds3, int dy_rounding, uint64_t dy_seed, snip_stats_t *stats6, void *ws,
+                                         size_t ws_bytes, void *stream)
+{
+    using namespace snip;
+    if (!X || !W || !dY || !Y || !dX || !dW || !bounds3) return SNIP_ERR_ARG;
+    if (!valid_dim(M) || !valid_dim(N) || !valid_dim(K)) return SNIP_ERR_SHAPE;
+    if (dy_rounding != SNIP_ROUND_NEAREST_EVEN && dy_rounding != SNIP_ROUND_STOCHASTIC) return SNIP_ERR_ARG;
+    const NvCarve f = carve_nvfp4(ws, M, N, K);
+    if (!ws || ws_bytes < f.total) return SNIP_ERR_WORKSPACE;
+    if (!aligned16(ws) || (stats6 && (reinterpret_cast<uintptr_t>(stats6) & 7u))) return SNIP_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float *bx = bounds3, *bw = bounds3 + 1, *bdy = bounds3 + 2;
+    auto stat = [&](int i) { return stats6 ? stats6 + i : nullptr; };
+    int rc = gemm_clear_status(f.gws, st);   // one status word for the three GEMMs
+    if (rc) return rc;
+    rc = quantize_nvfp4_dual_impl(X, M, K, K, bx, f.codes[0], f.sf[0], stat(0), f.codes[1], f.sf[1], stat(1), SNIP_ROUND_NEAREST_EVEN, 0, f.stats_ws,
+                                  f.stats_ws_bytes, st);
+    if (rc) return rc;
+    rc = quantize_nvfp4_dual_impl(W, N, K, K, bw, f.codes[2], f.sf[2], stat(2), f.codes[3], f.sf[3], stat(3), SNIP_ROUND_NEAREST_EVEN, 0, f.stats_ws,
+                                  f.stats_ws_bytes, st);
+    if (rc) return rc;
+    rc = gemm_nvfp4_impl(f.codes[0], f.codes[2], f.sf[0], f.sf[2], bx, bw, M, N, K, Y, out_dtype, f.gws, gemm_ws_bytes(), st, false);
+    if (rc) return rc;
+    rc = quantize_nvfp4_dual_impl(dY, M, N, N, bdy, f.codes[4], f.sf[4], stat(4), f.codes[5], f.sf[5], stat(5), dy_rounding, dy_seed, f.stats_ws,
+                                  f.stats_ws_bytes, st);
+    if (rc) return rc;
+    rc = gemm_nvfp4_impl(f.codes[4], f.codes[3], f.sf[4], f.sf[3], bdy, bw, M, K, N, dX, out_dtype, f.gws, gemm_ws_bytes(), st, false);
+    if (rc) return rc;
+    return gemm_nvfp4_impl(f.codes[5], f.codes[1], f.sf[5], f.sf[1], bdy, bx, N, K, M, dW, out_dtype, f.gws, gemm_ws_bytes(), st, false);
 }

@@ -158,3 +158,26 @@ def test_stochastic_rounding_bit_exact(api, shape):
     torch.cuda.synchronize()
     n = rows * cols // 2
     assert not torch.equal(a["codes"][:n], a2["codes"][:n]) and torch.equal(a["sf"], a2["sf"])
+
+
+def test_fwd_bwd_composition(api):
+    M, K, N = 384, 640, 448
+    rng = np.random.default_rng(78)
+    x, w, dy = spread(rng, M, K, 1.0), spread(rng, N, K, 0.02), spread(rng, M, N, 1e-3)
+    bounds = torch.tensor([amax_of(x), amax_of(w), amax_of(dy)], dtype=torch.float32, device="cuda")
+    y, dx, dw, stats = api.snip_linear_fwd_bwd_nvfp4(to_dev(x), to_dev(w), to_dev(dy), bounds, api.OUT_FP32)
+    torch.cuda.synchronize()
+    ref_y, qx, qw = orc.linear_nvfp4("fwd", x, w)
+    ref_dx, qdy, qwt = orc.linear_nvfp4("dgrad", dy, w)
+    ref_dw, qdyc, qxc = orc.linear_nvfp4("wgrad", dy, x)
+    assert rel_fro(y.cpu().numpy(), ref_y) <= 1e-5
+    assert rel_fro(dx.cpu().numpy(), ref_dx) <= 1e-5
+    assert rel_fro(dw.cpu().numpy(), ref_dw) <= 1e-5
+    for i, q in enumerate((qx, qxc, qw, qwt, qdy, qdyc)):
+        assert api.stats_to_host(stats[24 * i:24 * i + 24])["sumsq_err"] == pytest.approx(q.sumsq_err, rel=1e-4), i
+    # stochastic rounding of dY changes dX and dW only
+    y2, dx2, dw2, _ = api.snip_linear_fwd_bwd_nvfp4(to_dev(x), to_dev(w), to_dev(dy), bounds, api.OUT_FP32, dy_sr_seed=11)
+    torch.cuda.synchronize()
+    assert torch.equal(y2, y) and not torch.equal(dx2, dx)
+    want_dx = orc.gemm_dgrad(orc.quantize_nvfp4(dy, False, sr_seed=11).xhat, qwt.xhat)
+    assert rel_fro(dx2.cpu().numpy(), want_dx) <= 1e-5
