@@ -484,7 +484,8 @@ int snip_select_scheme(int m, int n, const double *q, const int64_t *w, int64_t 
 
 /*
  * Testing hooks, process-wide and off by default.  (No counterpart in the paper.)
- *   SNIP_DEBUG_WAIT_LIMIT_NS : bound of every device-side wait of the GEMM kernels (default 2e9).
+ *   SNIP_DEBUG_WAIT_LIMIT_NS : bound of every device-side wait of the GEMM kernels, the hardware-scaled
+ *                              ones (snip_gemm_mx, snip_gemm_nvfp4) included (default 2e9).
  *   SNIP_DEBUG_TX_SKEW_BYTES : a multiple of 16 added to the byte count a pipeline stage's barrier
  *                              expects.  Non-zero makes the first stage of every GEMM incomplete for
  *                              ever while every copy still lands: the kernel's waits run out, it

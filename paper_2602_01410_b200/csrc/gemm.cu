@@ -781,6 +781,13 @@ std::atomic<int> g_slicing{1};                           // 0: the weight-gradie
 std::atomic<int> g_kernel_choice{0};                     // 0, 1 = single-CTA kernels, 2 = CTA-pair kernels for quantized operands
 }  // namespace
 
+// The hooks' current values, for the other GEMM families (gemm_mx.cu).
+void gemm_debug_hooks(uint64_t *wait_limit_ns, int *tx_skew)
+{
+    *wait_limit_ns = (uint64_t)g_wait_limit_ns.load();
+    *tx_skew = g_tx_skew.load();
+}
+
 int gemm_pair_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, int64_t Mo, int64_t No, int64_t Kc, const float *sa,
                    int64_t sa_chunk_stride, const float *sb, int64_t sb_chunk_stride, int64_t sb_blk_stride, int scale_mode, void *out,
                    int out_dtype, int accumulate, uint32_t *status, uint64_t wait_limit_ns, int tx_skew, cudaStream_t st);

@@ -42,6 +42,7 @@ struct MxArgs {
     uint32_t stage_tx_bytes;   // bytes reported to a stage's barrier (operands + scale-factor atoms)
     uint32_t *status;
     const float *amax_a, *amax_b;   // two-level option: the tensors' magnitude bounds (device); else null
+    uint64_t wait_limit_ns;    // bound of every device-side wait
 };
 
 template <MmaKind KIND>
@@ -140,7 +141,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int nb0 = 2 * n_idx, nb1 = min(2 * n_idx + 1, g.n_atoms_b - 1);
                 for (int ks = 0; ks < num_kstages; ++ks, ++it) {
                     const int s = it % S;
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag))) { ok = false; break; }
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / S) & 1u) ^ 1u, abort_flag, g.wait_limit_ns))) { ok = false; break; }
                     if (elect_one()) {
                         mbar_arrive_expect_tx(full_bar(s), g.stage_tx_bytes);
                         tma_load_2d(a_tile(s), &tmA, full_bar(s), ks * 128, m_idx * BM);
@@ -173,7 +174,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t it = 0, tiles_done = 0;
             bool ok = true;
             const uint32_t sfa = tmem_base + kSfaCol, sfb = tmem_base + (C::kNv ? kNvSfbCol : kSfbCol);
-            auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag)); };
+            auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, g.wait_limit_ns)); };
             for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tiles_done) {
                 // the single accumulator must have been drained by the epilogue of the previous tile
                 if (!wait_all(tempty_bar, (tiles_done & 1u) ^ 1u)) { ok = false; break; }
@@ -237,7 +238,7 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mx_tile_coords(t, num_m, num_n, m_idx, n_idx);
             const int row0 = m_idx * BM + q * 32;
             const int col0 = n_idx * BN + h * HALF;
-            const bool got = mbar_wait(tfull_bar, tiles_done & 1u, abort_flag);
+            const bool got = mbar_wait(tfull_bar, tiles_done & 1u, abort_flag, g.wait_limit_ns);
             if (!__all_sync(0xFFFFFFFFu, got)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + h * HALF;
@@ -318,6 +319,7 @@ int make_tiled_map_2d(CUtensorMap *map, const void *ptr, int dtype, int64_t rows
                       int box_rows, int swizzle);
 int gemm_clear_status(void *ws, cudaStream_t st);
 int gemm_sm_count();
+void gemm_debug_hooks(uint64_t *wait_limit_ns, int *tx_skew);   // testing hooks of snip_debug_set (gemm.cu)
 
 // a_codes [Mo][Kc], b_codes [No][Kc] contraction-major; sfa / sfb: UE8M0 atoms [line tile][chunk][512].
 int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes, const void *sfa, const void *sfb, int64_t Mo, int64_t No,
@@ -341,6 +343,8 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
     g.sfb = static_cast<const uint8_t *>(sfb);
     g.n_atoms_b = (int32_t)ceil_div(No, 128);
     g.status = static_cast<uint32_t *>(ws);
+    int tx_skew = 0;
+    gemm_debug_hooks(&g.wait_limit_ns, &tx_skew);
     g.amax_a = g.amax_b = nullptr;
 
     CUtensorMap tmA, tmB, tmO;
@@ -354,7 +358,7 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
         if (rc) return rc;
         rc = make_tiled_map_2d(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN, CU_TENSOR_MAP_SWIZZLE_128B);
         if (rc) return rc;
-        g.stage_tx_bytes = (BM + BN) * 128 + 2 * 1536;
+        g.stage_tx_bytes = (BM + BN) * 128 + 2 * 1536 + tx_skew;
         const uint32_t idesc = make_idesc_block_scaled(1, 1, BM, BN);
         return f32 ? launch_mx<MmaKind::MXF4, true>(tmA, tmB, tmO, g, idesc, sms, st) : launch_mx<MmaKind::MXF4, false>(tmA, tmB, tmO, g, idesc, sms, st);
     }
@@ -365,7 +369,7 @@ int gemm_mx_impl(int fmt_a, int fmt_b, const void *a_codes, const void *b_codes,
     rc = make_tiled_map_2d(&tmB, b_codes, b4 ? CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B : CU_TENSOR_MAP_DATA_TYPE_UINT8, No, b4 ? kpad : Kc,
                            b4 ? Kc / 2 : Kc, 128, BN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128) + 1536;
+    g.stage_tx_bytes = BM * (a4 ? 64 : 128) + BN * (b4 ? 64 : 128) + 1536 + tx_skew;
     const uint32_t idesc = make_idesc_block_scaled(a4 ? 5 : 0, b4 ? 5 : 0, BM, BN);
     return f32 ? launch_mx<MmaKind::MXF8, true>(tmA, tmB, tmO, g, idesc, sms, st) : launch_mx<MmaKind::MXF8, false>(tmA, tmB, tmO, g, idesc, sms, st);
 }
@@ -391,6 +395,8 @@ int gemm_nvfp4_impl(const void *a_codes, const void *b_codes, const void *sfa, c
     g.sfb = static_cast<const uint8_t *>(sfb);
     g.n_atoms_b = (int32_t)ceil_div(No, 128);
     g.status = static_cast<uint32_t *>(ws);
+    int tx_skew = 0;
+    gemm_debug_hooks(&g.wait_limit_ns, &tx_skew);
     g.amax_a = amax_a; g.amax_b = amax_b;
     CUtensorMap tmA, tmB, tmO;
     rc = f32 ? make_tiled_map_2d(&tmO, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Mo, No, No * 4, 16, 32, CU_TENSOR_MAP_SWIZZLE_64B)
@@ -400,7 +406,7 @@ int gemm_nvfp4_impl(const void *a_codes, const void *b_codes, const void *sfa, c
     if (rc) return rc;
     rc = make_tiled_map_2d(&tmB, b_codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, No, Kc / 2, Kc / 2, 128, BN, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc) return rc;
-    g.stage_tx_bytes = (BM + BN) * 128 + 2 * 3072;
+    g.stage_tx_bytes = (BM + BN) * 128 + 2 * 3072 + tx_skew;
     const uint32_t idesc = make_idesc_block_scaled_e4m3(1, 1, BM, BN);
     const int sms = gemm_sm_count();
     return f32 ? launch_mx<MmaKind::NVF4, true>(tmA, tmB, tmO, g, idesc, sms, st) : launch_mx<MmaKind::NVF4, false>(tmA, tmB, tmO, g, idesc, sms, st);

@@ -89,3 +89,57 @@ def test_gemm_outputs_stay_inside_their_buffers(choice, fa, fb, out_dtype):
         api.snip_debug_set(api.DEBUG_GEMM_KERNEL, api.GEMM_KERNEL_AUTO)
     assert intact(wy, M * N * esz) and intact(wdx, M * K * esz) and intact(wdw, N * K * esz)
     assert torch.isfinite(y.float()).all() and torch.isfinite(dw.float()).all()
+
+
+@pytest.mark.parametrize("shape", [(320, 448), (192, 320), (64, 704)])
+def test_added_quantizer_forms_stay_inside_their_buffers(shape):
+    # 32-long tiles with power-of-two scales (codes, scales, atoms) and the two-level form (codes, atoms), two outputs each
+    from paper_2602_01410_b200 import api
+    rows, cols = shape
+    x = to_dev(wl.make_x(np.random.default_rng(6), rows, cols, 0.01, 20.0))
+    n = api.ctypes.c_size_t()
+    api._check("snip_quantize_mx_sizes", api._lib.snip_quantize_mx_sizes(rows, cols, api.ctypes.byref(n)))
+    for fmt in (FP8, FP4):
+        bufs, wholes = [], []
+        for i, blk in enumerate((api.BLOCK_ROW32, api.BLOCK_COL32)):
+            cb, sb, _ = api.snip_quantize_sizes(rows, cols, fmt, blk, api.Q_TRANSPOSED if i else 0)
+            wc, codes = guarded(cb); wsc, scales = guarded(sb, torch.float32); wsf, sf = guarded(n.value); wst, stats = guarded(32)
+            bufs.append({"codes": codes, "scales": scales, "sf": sf, "stats": stats[:24]})
+            wholes += [(wc, cb), (wsc, sb), (wsf, n.value), (wst, 32)]
+        wb = api.snip_quantize_dual_workspace(rows, cols)
+        ww, ws = guarded(wb)
+        api.snip_quantize_dual(x, api.DUAL_ROW32_COL32T, fmt, fmt, pow2_scale=True, bufs=tuple(bufs), ws=ws)
+        torch.cuda.synchronize()
+        assert all(intact(w, nb) for w, nb in wholes) and intact(ww, wb)
+        assert not (bufs[0]["sf"].cpu().numpy() == CANARY).all()
+    cb, fb = api.snip_quantize_nvfp4_sizes(rows, cols)
+    bufs, wholes = [], []
+    for i in range(2):
+        wc, codes = guarded(cb); wsf, sf = guarded(fb); wst, stats = guarded(32)
+        bufs.append({"codes": codes, "sf": sf, "stats": stats[:24]})
+        wholes += [(wc, cb), (wsf, fb), (wst, 32)]
+    wb = api.snip_quantize_dual_workspace(rows, cols)
+    ww, ws = guarded(wb)
+    bound = x.float().abs().max().reshape(1).contiguous()
+    api.snip_quantize_nvfp4_dual(x, bound, bufs=tuple(bufs), ws=ws)
+    torch.cuda.synchronize()
+    assert all(intact(w, nb) for w, nb in wholes) and intact(ww, wb)
+    assert not (bufs[1]["sf"].cpu().numpy() == CANARY).all()
+
+
+@pytest.mark.parametrize("shape", [(320, 448, 192), (64, 192, 320)])
+def test_hardware_scaled_gemm_outputs_stay_inside_their_buffers(shape):
+    from paper_2602_01410_b200 import api
+    M, K, N = shape
+    rng = np.random.default_rng(8)
+    x, w = to_dev(wl.make_x(rng, M, K, 0.01, 20.0)), to_dev(wl.make_w(rng, N, K))
+    bx, bw = x.float().abs().max().reshape(1).contiguous(), w.float().abs().max().reshape(1).contiguous()
+    xa, _ = api.snip_quantize_nvfp4_dual(x, bx, want_stats=False)
+    wa, _ = api.snip_quantize_nvfp4_dual(w, bw, want_stats=False)
+    a = api.make_qtensor(xa["codes"], None, M, K, FP4, api.BLOCK_ROW16)
+    b = api.make_qtensor(wa["codes"], None, N, K, FP4, api.BLOCK_ROW16)
+    for dt, esz in ((api.OUT_BF16, 2), (api.OUT_FP32, 4)):
+        wo, out = guarded(M * N * esz, torch.bfloat16 if esz == 2 else torch.float32)
+        api.snip_gemm_nvfp4(api.OP_FWD, a, xa["sf"], bx, b, wa["sf"], bw, (M, N), dt, out=out.view(M, N))
+        torch.cuda.synchronize()
+        assert intact(wo, M * N * esz)

@@ -100,3 +100,31 @@ def test_7b_qkv_sampled_rows_hardware_scaled():
     qw = orc.quantize(w, FP4, orc.BLOCK_BLK, True)
     ref16 = orc.bf16_to_float(orc.round_to_bf16(orc.gemm_fwd(qx.xhat, qw.xhat)))
     assert rel_fro(bf16_out_to_f64(y[torch.from_numpy(rows).cuda()]), ref16) <= 1e-3
+
+
+@pytest.mark.parametrize("fmt", [FP8, FP4])
+def test_a_wait_that_runs_out_in_the_hardware_scaled_gemm(fmt):
+    # Host-made condition (see test_gpu_gemm_kernels.py): the first stage's barrier expects 16 bytes more than the copies
+    # deliver, every copy lands, the phase never completes.  With a 20 ms wait limit the kernel gives up by itself, releases
+    # its tensor memory and raises the status word; nothing traps, faults or spins without a bound.
+    from paper_2602_01410_b200 import api
+    M, K, N = 512, 512, 256
+    rng = np.random.default_rng(19)
+    x, w = wl.make_x(rng, M, K), wl.make_w(rng, N, K)
+    cx, sx, fx, _ = api.snip_quantize_mx(to_dev(x), fmt, api.BLOCK_ROW)
+    cw, sw, fw, _ = api.snip_quantize_mx(to_dev(w), fmt, api.BLOCK_BLK)
+    a = api.make_qtensor(cx, sx, M, K, fmt, api.BLOCK_ROW); b = api.make_qtensor(cw, sw, N, K, fmt, api.BLOCK_BLK)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    try:
+        api.snip_debug_set(api.DEBUG_WAIT_LIMIT_NS, 20_000_000)
+        api.snip_debug_set(api.DEBUG_TX_SKEW_BYTES, 16)
+        api.snip_gemm_mx(api.OP_FWD, a, fx, b, fw, (M, N), api.OUT_FP32, ws=ws)
+        torch.cuda.synchronize()
+        assert api.snip_poll_status(ws) == api.ERR_TIMEOUT
+    finally:
+        api.snip_debug_set(api.DEBUG_TX_SKEW_BYTES, 0)
+        api.snip_debug_set(api.DEBUG_WAIT_LIMIT_NS, 2_000_000_000)
+    y = api.snip_gemm_mx(api.OP_FWD, a, fx, b, fw, (M, N), api.OUT_FP32, ws=ws)
+    torch.cuda.synchronize()
+    assert api.snip_poll_status(ws) == api.OK
+    assert rel_fro(y.cpu().numpy(), orc.linear_fwd(x, w, fmt, fmt, True)[0]) <= 1e-5

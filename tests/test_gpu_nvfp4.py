@@ -181,3 +181,29 @@ def test_fwd_bwd_composition(api):
     assert torch.equal(y2, y) and not torch.equal(dx2, dx)
     want_dx = orc.gemm_dgrad(orc.quantize_nvfp4(dy, False, sr_seed=11).xhat, qwt.xhat)
     assert rel_fro(dx2.cpu().numpy(), want_dx) <= 1e-5
+
+
+def test_a_wait_that_runs_out_reports_timeout(api):
+    # the host-made condition of test_gpu_gemm_kernels.py (a stage barrier that expects 16 bytes too many, a 20 ms wait limit)
+    M, K, N = 512, 512, 256
+    rng = np.random.default_rng(79)
+    x, w = spread(rng, M, K, 1.0), spread(rng, N, K, 0.02)
+    ax, aw = dev_f32(amax_of(x)), dev_f32(amax_of(w))
+    xa, _ = api.snip_quantize_nvfp4_dual(to_dev(x), ax, want_stats=False)
+    wa, _ = api.snip_quantize_nvfp4_dual(to_dev(w), aw, want_stats=False)
+    a = api.make_qtensor(xa["codes"], None, M, K, FP4, api.BLOCK_ROW16)
+    b = api.make_qtensor(wa["codes"], None, N, K, FP4, api.BLOCK_ROW16)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    try:
+        api.snip_debug_set(api.DEBUG_WAIT_LIMIT_NS, 20_000_000)
+        api.snip_debug_set(api.DEBUG_TX_SKEW_BYTES, 16)
+        api.snip_gemm_nvfp4(api.OP_FWD, a, xa["sf"], ax, b, wa["sf"], aw, (M, N), api.OUT_FP32, ws=ws)
+        torch.cuda.synchronize()
+        assert api.snip_poll_status(ws) == api.ERR_TIMEOUT
+    finally:
+        api.snip_debug_set(api.DEBUG_TX_SKEW_BYTES, 0)
+        api.snip_debug_set(api.DEBUG_WAIT_LIMIT_NS, 2_000_000_000)
+    y = api.snip_gemm_nvfp4(api.OP_FWD, a, xa["sf"], ax, b, wa["sf"], aw, (M, N), api.OUT_FP32, ws=ws)
+    torch.cuda.synchronize()
+    assert api.snip_poll_status(ws) == api.OK
+    assert rel_fro(y.cpu().numpy(), orc.linear_nvfp4("fwd", x, w)[0]) <= 1e-5
