@@ -8,8 +8,13 @@
 // One CTA per SM, persistent, 384 threads: warp 0 streams operand tiles (TMA) and 512-byte
 // scale-factor atoms (bulk copies) into a shared-memory ring; warp 1 copies each stage's atoms into
 // tensor memory (tcgen05.cp) and issues the MMAs; warps 4-11 drain the 128x256 FP32 accumulator
-// (one buffer: 256 columns, next to 12 scale-factor columns), round, and store through the TMA unit.
-// Every wait is bounded, as in gemm.cu.
+// (one buffer: 256 columns, next to 12 or 24 scale-factor columns), round, and store through the TMA unit.
+// Warps 0 and 1 walk their loops as whole warps and one elected lane issues.  Every wait is bounded, as in gemm.cu.
+//
+// The bytes may differ within a chunk (32-long tiles: byte k belongs to the k-th 32 elements; the MMA of that step
+// selects it through the descriptor's scale-factor id).  A third instantiation serves the two-level option in the
+// style of NVFP4: E2M1 codes, an E4M3 scale byte per 16 elements (a word per line and 64-long MMA step, two atoms per
+// chunk), tcgen05.mma kind::mxf4nvf4 with scale_vec::4X, and one division by the two per-tensor factors at the end.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <float.h>

@@ -12,6 +12,12 @@
 // for COL, both for BLK).  Codes as stored leave straight from registers; transposed codes go through
 // byte-permute 8x8 transposes and an XOR-swizzled shared-memory tile so that the global stores stay coalesced.
 // The two-output form (quantize_dual_kernel) encodes each element under two scales in the same pass.
+//
+// Added options (paper Sec. 3.2 lets further quantization methods join the per-layer choices): the power-of-two scale
+// rule on the same tiles or on 32-long tiles (ROW_1x32 / COL_32x1: the maxima are combined over 4 lanes / 2 warps
+// instead of 16 lanes / 8 warps), with the scale exponents also written as the 512-byte atoms the block-scaled MMA
+// reads; and the two-level form in the style of NVFP4 (quantize_nvfp4_dual_kernel: 16-long tiles = two neighbouring
+// lanes / the two row groups of a warp, an E4M3 scale byte per tile, a per-tensor factor from a caller-supplied bound).
 #include <cuda_bf16.h>
 #include <float.h>
 
