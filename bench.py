@@ -358,7 +358,9 @@ def run_two_level(step, events=None, qevents=None):
 class TaggedStep:
     """A table-driven workload (3B: each GEMM drawn FP4 / FP8 / BF16; 70B slice: at least 80 % of the linear-layer
     FLOPs in FP4, the rest FP8): `layers` layers resident, every linear's forward, input-gradient and weight-gradient
-    GEMM through snip_linear_fwd / dgrad / wgrad with the tag of that GEMM on both operands, statistics on."""
+    GEMM with the tag of that GEMM on both operands, statistics on.  A linear whose three tags are all quantized formats
+    goes through snip_linear_fwd_bwd (each tensor read once, both of its copies and their statistics written); one with a
+    BF16 tag through snip_linear_fwd / dgrad / wgrad."""
 
     def __init__(self, api, torch, cfg, device, layers):
         from paper_2602_01410_b200 import workloads as wl
@@ -373,9 +375,12 @@ class TaggedStep:
             for op in (api.OP_FWD, api.OP_DGRAD, api.OP_WGRAD):
                 for f in (FMT_BF16, FMT_FP8, FMT_FP4):
                     ws_bytes = max(ws_bytes, api.snip_workspace_size(op, M, L.N, L.K, f, f)[1])
+        for L in cfg.linears:
+            ws_bytes = max(ws_bytes, api.snip_linear_fwd_bwd_workspace(M, L.N, L.K, FMT_FP8, FMT_FP8, FMT_FP8, 0))
         self.ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
         n_gemm = layers * len(cfg.linears) * 3
         self.stats = torch.zeros(n_gemm * 2, 32, dtype=torch.uint8, device=device)
+        self.stats6 = torch.zeros(layers * len(cfg.linears), 6 * 24, dtype=torch.uint8, device=device)
         self.flops = layers * sum(2.0 * M * L.N * L.K * 3 for L in cfg.linears)
         self.flops_by_fmt = {}
         for l in range(layers):
@@ -383,8 +388,10 @@ class TaggedStep:
                 for gi in range(3):
                     f = int(self.tags[l, j, gi])
                     self.flops_by_fmt[f] = self.flops_by_fmt.get(f, 0.0) + 2.0 * M * L.N * L.K
-        # per GEMM: quantized tags: 2 quantizers + 2 reductions + 1 GEMM; BF16 tags: statistics kernels + reductions + GEMM (+ transposes)
-        self.launches_per_step = n_gemm * 5
+        # a linear through snip_linear_fwd_bwd: 3 two-output quantizers + 3 reductions + 3 GEMMs; through the three separate calls, per GEMM:
+        # 2 quantizers (BF16 tags: statistics kernels, transposes) + 2 reductions + 1 GEMM
+        n_fused = sum(1 for l in range(layers) for j in range(len(cfg.linears)) if FMT_BF16 not in [int(t) for t in self.tags[l, j]])
+        self.launches_per_step = n_fused * 9 + (layers * len(cfg.linears) - n_fused) * 15
 
     def run(self, events=None, inputs=None, before=None):
         api, torch = self.api, self.torch
@@ -397,6 +404,19 @@ class TaggedStep:
                     before(l, j)
                 M, K = x.shape
                 N = w.shape[0]
+                t3 = [int(self.tags[l, j, gi]) for gi in range(3)]
+                if FMT_BF16 not in t3:
+                    if events is not None:
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                    api._check("snip_linear_fwd_bwd", lib.snip_linear_fwd_bwd(p(x), p(w), p(dy), p(y), p(dx), p(dw), M, N, K, t3[0], t3[1], t3[2], api.OUT_BF16,
+                                                                              0, 0, 0, p(self.stats6[l * len(self.out) + j]), p(self.ws), self.ws.numel(), st))
+                    if events is not None:
+                        e1.record()
+                        for f in t3:   # one call, three GEMMs of equal size: a third of its time to each tag
+                            events.append((f, 2.0 * M * N * K, e0, e1, 1.0 / 3.0))
+                    i += 3
+                    continue
                 calls = (("snip_linear_fwd", lambda f, sa, sb: lib.snip_linear_fwd(p(x), p(w), p(y), M, N, K, f, f, api.OUT_BF16, p(sa), p(sb), p(self.ws), self.ws.numel(), st)),
                          ("snip_linear_dgrad", lambda f, sa, sb: lib.snip_linear_dgrad(p(dy), p(w), p(dx), M, N, K, f, f, api.OUT_BF16, p(sa), p(sb), p(self.ws), self.ws.numel(), st)),
                          ("snip_linear_wgrad", lambda f, sa, sb: lib.snip_linear_wgrad(p(dy), p(x), p(dw), M, N, K, f, f, api.OUT_BF16, 0, p(sa), p(sb), p(self.ws), self.ws.numel(), st)))
@@ -729,9 +749,10 @@ def run_tagged(args, api, torch, dist, wl, cfg, device, world, rank, local_rank,
     value = flops_job / (ms_per_step * 1e-3) / 1e12
     # per operand format: the linear calls (quantizers + GEMM) of the timed region against the GEMM's tensor peak
     per_format = {}
-    for f, fl, a, b in events:
+    for ev in events:
+        f, fl, a, b = ev[:4]
         d = per_format.setdefault(f, {"flops": 0.0, "ms": 0.0, "calls": 0})
-        d["flops"] += fl; d["ms"] += a.elapsed_time(b); d["calls"] += 1
+        d["flops"] += fl; d["ms"] += a.elapsed_time(b) * (ev[4] if len(ev) > 4 else 1.0); d["calls"] += 1
     pf = {}
     for f, d in per_format.items():
         ach = d["flops"] / (d["ms"] * 1e-3) / 1e12
@@ -739,7 +760,7 @@ def run_tagged(args, api, torch, dist, wl, cfg, device, world, rank, local_rank,
         pf[FMT_NAME[f]] = {"achieved": ach, "peak": pk, "frac": ach / pk, "calls": d["calls"], "share_of_step": d["ms"] / ms_total,
                            "share_of_flops": step.flops_by_fmt.get(f, 0.0) / step.flops}
     worst = min(pf, key=lambda k: pf[k]["frac"])
-    roofline = {"kernel": f"snip_linear_fwd/dgrad/wgrad calls (two quantizer passes with statistics + GEMM), headline = {worst} tags",
+    roofline = {"kernel": f"snip_linear_fwd_bwd / snip_linear_fwd/dgrad/wgrad calls (quantizer passes with statistics + GEMMs), headline = {worst} tags",
                 "bound": "tensor", "achieved": pf[worst]["achieved"], "peak": pf[worst]["peak"], "unit": "TFLOP/s", "frac": pf[worst]["frac"],
                 "traffic": None, "per_format": pf,
                 "peak_source": f"{peaks['source']} cuBLAS bf16 sustained x nominal format ratio (x1 bf16, x2 fp8, x4 fp4)"}
