@@ -178,7 +178,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     using C = Cfg<KIND, BN, SCALE>;
     constexpr int S = C::kStages;
     constexpr int HALF = BN / 2;     // columns handled by one epilogue warp
-    constexpr int GC = 32;           // columns per tensor-memory load
+    // columns per tensor-memory load: 16 in vector mode (wgrad: the promotion loop holds the column reciprocals next to the
+    // staging registers and runs 1.5-4 % faster with the smaller groups), 32 otherwise (fwd / dgrad: 2.5 % faster than 16)
+    constexpr int GC = (SCALE == SCALE_VEC_B) ? 16 : 32;
     constexpr int G = HALF / GC;     // groups handled by one epilogue warp per chunk
 
     extern __shared__ uint8_t smem_raw[];
