@@ -549,20 +549,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 };
                 // Two loads are in flight from the start; each group's FMAs free its registers for the load two groups
-                // on.  The buffer goes back to the MMA warp as soon as the last load has landed, so that the stretch in
-                // which that warp may be waiting holds the FMAs of only G-2 groups; the last two groups follow the release.
+                // on.  A load is waited for one group after it was issued, before the next one is issued (the wait covers
+                // every outstanding load of the thread), so that its latency lies under that group's FMAs and no group is
+                // consumed before its load has been waited for.  The buffer goes back to the MMA warp when the last load
+                // has landed; the last group follows the release.
                 tmem_ld_wait();
                 if (G <= 2) release_buffer();
 #pragma unroll
                 for (int gi = 0; gi < G; ++gi) {
                     consume_group(gi, v[gi & 1]);
-                    if (gi + 2 < G) {
-                        tmem_ld_cols(taddr + GC * (gi + 2), v[gi & 1]);
-                        if (gi + 3 >= G) {   // that was the chunk's last load
-                            tmem_ld_wait();
-                            release_buffer();
-                        }
-                    }
+                    if (gi >= 1 && gi + 1 < G) tmem_ld_wait();                   // group gi+1 has landed
+                    if (gi + 2 < G) tmem_ld_cols(taddr + GC * (gi + 2), v[gi & 1]);
+                    if (G > 2 && gi + 2 == G) release_buffer();                  // ... and it was the chunk's last load
                 }
                 if (SCALE == SCALE_VEC_B && (cc % C::kVecBlock) == C::kVecBlock - 1) {
                     __syncwarp();                        // every lane has read the block's slots
